@@ -1,0 +1,238 @@
+/*
+ * dsq.h - C ABI of the B200 (sm_100a) library for the deployed form of
+ * Differentiable Soft Quantization (arXiv 1908.05033): 2-4 bit uniform-
+ * quantised convolution with integer contraction and a fused
+ * dequantise / requantise epilogue.
+ *
+ * Quantiser (paper Sec. 3.1 Eq. 2; Algorithm 1 feed-forward steps 1, 3, 4):
+ * bit width b, clip bounds l < u, interval Delta = (u - l) / (2^b - 1).
+ * A value x becomes the unsigned code
+ *       q = floor((clip(x, l, u) - l) / Delta + 1/2),   0 <= q <= 2^b - 1,
+ * a value on an interval midpoint taking the upper code (sgn(0) = +1, Eq. 1);
+ * its dequantised value is l + q * Delta.  This is the limit the soft
+ * quantiser (Eq. 3-5) reaches as alpha -> 0, and what sgn(phi(x)) yields for
+ * any alpha.  Weights are stored as signed codes c = q - 2^(b-1).
+ * The binary32 operation sequence is fixed:
+ *       inv = (float)(2^b - 1) / (u - l);  xc = fminf(fmaxf(x, l), u);
+ *       r = fmaf(xc - l, inv, 0.5f);       q = min((int)floorf(r), 2^b - 1)
+ * (NaN quantises to code 0, +-inf to the nearest end).
+ *
+ * Packed code format ("packed rows"): each row is a little-endian dense bit
+ * stream, element j in bits [j*b, j*b + b); unsigned codes in plain binary,
+ * signed codes in b-bit two's complement; the row pitch is
+ * dsq_row_pitch(k, b) = ceil(k*b/8) rounded up to 16 bytes; spare bits are 0.
+ * An activation tensor is NHWC with one packed row per pixel (k = C).
+ *
+ * Conventions for every entry point
+ *  - All data pointers are DEVICE pointers unless a parameter says "host".
+ *    Descriptor structs (dsq_*_t) are read on the host during the call.
+ *  - Every buffer is allocated and owned by the caller and must be 16-byte
+ *    aligned.  The library allocates no device memory.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the legacy default
+ *    stream).  Work is enqueued asynchronously; no entry point synchronises
+ *    except dsq_workspace_status.
+ *  - Return value: DSQ_OK (0) or a negative dsq_status code.  Arguments are
+ *    validated on the host before anything is launched; nothing is launched
+ *    when an error is returned.  No entry point throws, aborts or prints.
+ *  - `workspace`: at least dsq_workspace_bytes() bytes of device memory,
+ *    cleared once with dsq_workspace_init.  The tensor-core kernels bound
+ *    every wait on a barrier; a wait that runs out records DSQ_ERR_TIMEOUT
+ *    in the workspace, the kernel releases its tensor memory and returns, and
+ *    dsq_workspace_status reports it.  Calls that share a workspace must be
+ *    ordered on one stream.
+ */
+#ifndef DSQ_H_
+#define DSQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum dsq_status {
+    DSQ_OK = 0,
+    DSQ_ERR_NULL = -1,        /* a required pointer is NULL                   */
+    DSQ_ERR_ALIGN = -2,       /* a buffer is not 16-byte aligned              */
+    DSQ_ERR_BITS = -3,        /* bit width outside 2..4                       */
+    DSQ_ERR_SHAPE = -4,       /* non-positive or inconsistent dimensions      */
+    DSQ_ERR_SIZE = -5,        /* an output / workspace buffer is too small    */
+    DSQ_ERR_RANGE = -6,       /* hi <= lo, or a bound is not finite           */
+    DSQ_ERR_OVERFLOW = -7,    /* K * 2^7 * (2^b - 1) would exceed int32       */
+    DSQ_ERR_UNSUPPORTED = -8, /* valid request this build does not implement  */
+    DSQ_ERR_CUDA = -9,        /* a CUDA runtime / driver call failed          */
+    DSQ_ERR_TIMEOUT = -10     /* a bounded device-side wait ran out           */
+} dsq_status;
+
+/* Quantiser parameters (b, l, u) of one tensor. */
+typedef struct dsq_quant_t {
+    int32_t bits;
+    float lo, hi;
+} dsq_quant_t;
+
+/* Activation tensor shape, NHWC. */
+typedef struct dsq_nhwc_t {
+    int32_t N, H, W, C;
+} dsq_nhwc_t;
+
+/* Convolution geometry.  groups = 1: dense, weights [Cout][KH][KW][Cin].
+ * groups = Cin = Cout: depthwise, weights [C][KH][KW].  Dilation is 1. */
+typedef struct dsq_conv_t {
+    int32_t Cout, KH, KW, Cin;
+    int32_t stride, pad;
+    int32_t groups;
+} dsq_conv_t;
+
+/* Epilogue applied to the int32 accumulator acc[m][co] (Algorithm 1 steps
+ * 4-5 folded onto integers, then steps 1 and 3 of the next layer):
+ *   w_offset = 0   : y = fmaf((float)acc, scale[co], bias[co])
+ *   w_offset = 0.5 : y = fmaf((float)(2*acc + S_a), scale[co]*0.5f, bias[co])
+ *                    where S_a = sum of the activation codes under the
+ *                    in-image filter taps.  This is the paper's weight grid
+ *                    l_w + Delta_w*q_w with a symmetric clip l_w = -u_w, for
+ *                    which w^ = Delta_w * (c + 1/2); scale = Delta_a*Delta_w.
+ *   residual_codes : y = y + fmaf((float)q_r, Delta_r, l_r), q_r the unsigned
+ *                    code at the same output position (packed NHWC, same
+ *                    shape as the output), (l_r, Delta_r) from residual_q
+ *   requant.bits>0 : codes = quantise(y; requant)  (ReLU is the clip at lo=0)
+ * Other w_offset values return DSQ_ERR_UNSUPPORTED. */
+typedef struct dsq_epilogue_t {
+    const float *scale;          /* [Cout], required */
+    const float *bias;           /* [Cout], required */
+    float w_offset;
+    const void *residual_codes;  /* nullable */
+    dsq_quant_t residual_q;      /* bits must equal the layer's when used */
+    dsq_quant_t requant;         /* bits = 0: no code output */
+} dsq_epilogue_t;
+
+/* ---- sizes ------------------------------------------------------------- */
+
+/* Row pitch in bytes of k codes of `bits` bits: ceil(k*bits/8) rounded up to
+ * a multiple of 16.  0 on invalid arguments. */
+size_t dsq_row_pitch(int64_t k, int bits);
+
+/* rows * dsq_row_pitch(k, bits). */
+size_t dsq_packed_bytes(int64_t rows, int64_t k, int bits);
+
+/* Size of the blob dsq_pack_weights writes for this geometry. */
+size_t dsq_weight_bytes(const dsq_conv_t *conv, int bits);
+
+/* Minimum workspace size. */
+size_t dsq_workspace_bytes(void);
+
+/* ---- workspace --------------------------------------------------------- */
+
+/* Clear a workspace (asynchronous memset on `stream`). */
+int dsq_workspace_init(void *workspace, size_t ws_bytes, void *stream);
+
+/* Synchronise `stream`, read the status word of the workspace and clear it.
+ * Returns DSQ_OK, DSQ_ERR_TIMEOUT (a kernel gave up on a wait; its outputs
+ * are undefined) or DSQ_ERR_RANGE (dsq_pack_weights met a bad clip range). */
+int dsq_workspace_status(void *workspace, void *stream);
+
+/* ---- Algorithm 1 steps 1, 3 for weights (offline) ---------------------- */
+
+/* Quantise fp32 weights to signed b-bit codes and write the layout the
+ * convolution kernels read.
+ *   w          fp32, [Cout][KH][KW][Cin] (dense) or [C][KH][KW] (depthwise)
+ *   lo, hi     device arrays of clip bounds: one element each, or Cout
+ *              elements when per_channel != 0
+ *   packed_out dsq_weight_bytes(conv, bits) bytes.  Dense: Cout rows, each
+ *              the KH*KW filter taps in order, every tap a packed row of Cin
+ *              signed codes at the activation pixel pitch
+ *              dsq_row_pitch(Cin, bits).  Depthwise: KH*KW packed rows of C
+ *              signed codes.  Treat as opaque; dsq_unpack can read it.
+ * A clip range with hi <= lo or a non-finite bound cannot be seen from the
+ * host: the kernel writes code 0 for that channel and records DSQ_ERR_RANGE
+ * in the workspace. */
+int dsq_pack_weights(const float *w, const dsq_conv_t *conv, int bits,
+                     const float *lo, const float *hi, int per_channel,
+                     void *packed_out, size_t packed_bytes, void *workspace,
+                     size_t ws_bytes, void *stream);
+
+/* ---- Algorithm 1 steps 1, 3 for activations ---------------------------- */
+
+/* fp32 NHWC -> packed unsigned codes, one packed row per pixel.
+ * codes_out: dsq_packed_bytes(N*H*W, C, q->bits) bytes.  HBM-bound:
+ * 4 + bits/8 bytes per element. */
+int dsq_quantize_act(const float *x, const dsq_nhwc_t *shape,
+                     const dsq_quant_t *q, void *codes_out, size_t bytes,
+                     void *stream);
+
+/* ---- Algorithm 1 step 5 on codes + epilogue ---------------------------- */
+
+/* Dense convolution as an implicit GEMM on the 5th-generation tensor cores
+ * (tcgen05.mma kind::i8, int32 accumulation in tensor memory):
+ * M = N*Ho*Wo output pixels, N = Cout, K = KH*KW*Cin.
+ *   act_codes  packed NHWC unsigned codes of `shape`, quantiser act_q.
+ *              act_q->lo must be 0 when conv->pad > 0 (padding is code 0).
+ *   w_packed   from dsq_pack_weights with the same geometry and bits
+ *   y_f32      nullable: fp32 NHWC output [N][Ho][Wo][Cout]
+ *   y_codes    nullable: packed NHWC codes of the output (needs
+ *              ep->requant.bits == act_q->bits)
+ *   acc_out    nullable: raw int32 accumulators [N][Ho][Wo][Cout]
+ *              (2*acc + S_a when w_offset = 0.5)
+ * KH = KW in {1, 3}, stride in {1, 2}; bits in {2, 4} (3-bit convolution is
+ * not implemented: DSQ_ERR_UNSUPPORTED). */
+int dsq_conv2d(const void *act_codes, const dsq_nhwc_t *shape,
+               const dsq_quant_t *act_q, const void *w_packed,
+               const dsq_conv_t *conv, const dsq_epilogue_t *ep,
+               float *y_f32, void *y_codes, int32_t *acc_out,
+               void *workspace, size_t ws_bytes, void *stream);
+
+/* Depthwise 3x3 convolution on CUDA cores (not a dense contraction):
+ * acc[n][ho][wo][c] = sum over the 3x3 taps of q_a * c_w, then the same
+ * epilogue with per-channel S_a.  Same arguments as dsq_conv2d;
+ * conv->groups = Cin = Cout = shape->C, KH = KW = 3, pad = 1, bits in {2,4}.
+ * HBM-bound: bits/8 bytes in and out per element. */
+int dsq_dwconv2d(const void *act_codes, const dsq_nhwc_t *shape,
+                 const dsq_quant_t *act_q, const void *w_packed,
+                 const dsq_conv_t *conv, const dsq_epilogue_t *ep,
+                 float *y_f32, void *y_codes, int32_t *acc_out, void *stream);
+
+/* Plain low-bit GEMM on the tensor cores: C[m][n] = sum_k A[m][k] * B[n][k].
+ *   A_codes   packed rows [M][K] of SIGNED codes
+ *   B_codes   packed rows [N][K] of UNSIGNED codes
+ *   C_i32     nullable: int32 [M][N]
+ *   row_scale nullable unless D_f32 is given: fp32 [M]
+ *   D_f32     nullable: D[m][n] = (float)C[m][n] * row_scale[m]
+ * bits in {2, 3, 4}. */
+int dsq_gemm(const void *A_codes, const void *B_codes, int64_t M, int64_t N,
+             int64_t K, int bits, int32_t *C_i32, const float *row_scale,
+             float *D_f32, void *workspace, size_t ws_bytes, void *stream);
+
+/* 2x2 stride-2 max-pool on packed unsigned codes (exact on codes because the
+ * quantiser is monotone).  H and W must be even. */
+int dsq_maxpool2x2(const void *codes_in, const dsq_nhwc_t *shape, int bits,
+                   void *codes_out, size_t bytes, void *stream);
+
+/* ---- format helpers (tests, tooling) ----------------------------------- */
+
+/* int8 codes [rows][k] (dense) -> packed rows.  Values are truncated to
+ * their low `bits` bits. */
+int dsq_pack_codes(const int8_t *codes, int64_t rows, int64_t k, int bits,
+                   void *packed_out, size_t bytes, void *stream);
+
+/* packed rows -> int8 codes [rows][k] (dense), sign-extended if is_signed. */
+int dsq_unpack(const void *packed, int64_t rows, int64_t k, int bits,
+               int is_signed, int8_t *codes_out, void *stream);
+
+/* ---- measurement ------------------------------------------------------- */
+
+/* Tensor-core rate probe: every SM issues `iters` back-to-back
+ * tcgen05.mma kind::i8 128x256x32 instructions on operands resident in
+ * shared memory.  Synchronises; writes the elapsed milliseconds (CUDA
+ * events) to *ms_out (host) and the number of multiply-accumulates performed
+ * to *macs_out (host).  Gives the denominator "measured INT8 peak". */
+int dsq_probe_i8_mma_rate(int iters, float *ms_out, double *macs_out,
+                          void *workspace, size_t ws_bytes, void *stream);
+
+/* ---- misc --------------------------------------------------------------- */
+const char *dsq_status_string(int status);
+int dsq_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DSQ_H_ */

@@ -1,0 +1,882 @@
+// Low-bit implicit GEMM on the 5th-generation tensor cores (sm_100a).
+//
+//   acc[m][n] = sum_k A[m][k] * B[n][k]       (Algorithm 1 step 5 on codes)
+//
+// A rows are output pixels (or GEMM rows) gathered from packed NHWC codes, B
+// rows are output channels (packed weights, or the GEMM's B).  Both operands
+// live in HBM as packed b-bit codes; the tensor core wants 8-bit integers, so
+// each 128-code K step is expanded on the way through the SM:
+//
+//   B: TMA (cp.async.bulk.tensor.2d) packed tile -> shared ring ->
+//      unpack warps -> int8 tile in the K-major 128B-swizzled layout
+//   A: unpack warps gather 16-byte packed chunks straight from global memory
+//      (implicit im2col, zero fill outside the image) -> same int8 layout
+//   one thread issues tcgen05.mma.kind::i8 (128 x BN x 32 per instruction),
+//      accumulating int32 in tensor memory (two accumulator buffers)
+//   epilogue warps read tensor memory (tcgen05.ld), apply the dequantise /
+//      requantise epilogue and write codes / fp32 / int32.
+//
+// Signed codes are expanded into the TOP b bits of the byte (value * 2^(8-b)):
+// this costs no sign-extension arithmetic, and the exact factor is shifted out
+// of the int32 accumulator in the epilogue.  With the paper's symmetric weight
+// grid (w^ = Delta_w (c + 1/2)) the bit below is set as well, which makes the
+// byte 2^(7-b) (2c + 1) and the accumulator 2^(7-b) (2 acc + S_a).
+//
+// The order of the codes inside a 128-code K step is permuted by the unpack
+// (even / odd nibbles land in different 16-byte chunks); A and B use the same
+// permutation, and a sum over k does not depend on the order.
+//
+// Every wait on an mbarrier is bounded; a wait that runs out records
+// DSQ_ERR_TIMEOUT in the workspace, all roles leave their loops, tensor memory
+// is released and the kernel returns.
+#include <cuda.h>
+
+#include "dsq_epilogue.cuh"
+#include "dsq_ptx.cuh"
+
+using namespace dsq_ptx;
+
+namespace {
+
+constexpr int BM = 128;               // tile rows = MMA M
+constexpr int BK_BYTES = 128;         // int8 bytes per row per K step (128 codes)
+constexpr int S_U = 3;                // stages of unpacked (int8) tiles
+constexpr int S_P = 4;                // stages of packed B tiles
+constexpr int A_TILE_BYTES = BM * BK_BYTES;   // 16 KB
+
+constexpr int WARP_TMA = 0, WARP_MMA = 1, WARP_A0 = 2, WARP_B0 = 6, WARP_E0 = 10;
+constexpr int NUM_WARPS = 14;
+constexpr int NUM_THREADS = NUM_WARPS * 32;
+constexpr uint32_t WAIT_LIMIT = 1u << 24;     // try_wait rounds before giving up
+
+enum { MODE_CONV = 0, MODE_GEMM = 1 };
+
+struct TcParams {
+    // problem
+    int M, Ncols, ksteps, BN, m_tiles, n_tiles;
+    // A gather geometry (a GEMM is a 1x1 convolution over an M x 1 image)
+    const uint8_t *act;
+    int H, W, Ho, Wo, stride, pad, KW, taps, P;
+    // epilogue
+    int mode, shift, out_pitch;
+    DsqEpi e;
+    int32_t *C_i32;
+    const float *row_scale;
+    float *D_f32;
+    uint32_t orv;                     // OR-ed into every signed byte
+    int *ws;
+};
+
+// ---------------------------------------------------------------------------
+// bounded wait
+// ---------------------------------------------------------------------------
+struct Ctl {
+    volatile int *abort_flag;   // shared memory
+    int *ws;
+};
+
+__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, const Ctl &c,
+                                         int tag)
+{
+    for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 1023u) == 1023u && *c.abort_flag) return false;
+    }
+    if (atomicCAS(c.ws + DSQ_WS_STATUS, 0, (int)DSQ_ERR_TIMEOUT) == 0)
+        c.ws[DSQ_WS_DETAIL] = tag;
+    *c.abort_flag = 1;
+    return false;
+}
+
+// ---------------------------------------------------------------------------
+// packed -> int8 expansion of one 16-byte chunk
+// ---------------------------------------------------------------------------
+template <int BITS, bool SIGNED>
+struct Unpack;
+
+template <bool SIGNED>
+struct Unpack<4, SIGNED> {          // 32 codes -> 2 chunks
+    static constexpr int OUT = 2;
+    __device__ static __forceinline__ uint32_t e(uint32_t w, int c, uint32_t orv)
+    {
+        if (!SIGNED) return (c == 0 ? w : (w >> 4)) & 0x0F0F0F0Fu;
+        return ((c == 0 ? (w << 4) : w) & 0xF0F0F0F0u) | orv;
+    }
+};
+template <bool SIGNED>
+struct Unpack<2, SIGNED> {          // 64 codes -> 4 chunks
+    static constexpr int OUT = 4;
+    __device__ static __forceinline__ uint32_t e(uint32_t w, int c, uint32_t orv)
+    {
+        if (!SIGNED) return (w >> (2 * c)) & 0x03030303u;
+        return ((c == 3 ? w : (w << (6 - 2 * c))) & 0xC0C0C0C0u) | orv;
+    }
+};
+
+// Expand chunk `v` (logical packed chunk j of the row) into row `row` of an
+// int8 tile in the 128B-swizzled K-major layout: logical 16-byte chunk q of
+// the row sits at physical chunk q ^ (row & 7).
+template <int BITS, bool SIGNED>
+__device__ __forceinline__ void expand_chunk(uint8_t *tile, int row, int j, uint4 v,
+                                             uint32_t orv)
+{
+    using U = Unpack<BITS, SIGNED>;
+    uint8_t *rowp = tile + row * BK_BYTES;
+#pragma unroll
+    for (int c = 0; c < U::OUT; ++c) {
+        const uint4 o = make_uint4(U::e(v.x, c, orv), U::e(v.y, c, orv),
+                                   U::e(v.z, c, orv), U::e(v.w, c, orv));
+        const int q = j * U::OUT + c;
+        *reinterpret_cast<uint4 *>(rowp + ((q ^ (row & 7)) << 4)) = o;
+    }
+}
+
+// 3-bit: a row step is 48 packed bytes (12 words, 128 codes).  Four codes
+// (12 bits) at a time are spread to one 32-bit word of bytes.
+template <bool SIGNED>
+__device__ __forceinline__ void expand_row3(uint8_t *tile, int row, const uint32_t (&w)[12],
+                                            uint32_t orv)
+{
+    uint8_t *rowp = tile + row * BK_BYTES;
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {          // output chunk q: codes 16q .. 16q+15
+        uint32_t o[4];
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+            const int bit = (16 * q + 4 * t) * 3;
+            const int wi = bit >> 5, sh = bit & 31;
+            const uint32_t hi = wi + 1 < 12 ? w[wi + 1] : 0u;
+            const uint32_t x = __funnelshift_r(w[wi], hi, sh);
+            uint32_t b = (x & 7u) | ((x & 0x38u) << 5) | ((x & 0x1C0u) << 10) |
+                         ((x & 0xE00u) << 15);
+            if (SIGNED) b = (b << 5) | orv;
+            o[t] = b;
+        }
+        *reinterpret_cast<uint4 *>(rowp + ((q ^ (row & 7)) << 4)) =
+            make_uint4(o[0], o[1], o[2], o[3]);
+    }
+}
+
+// ---------------------------------------------------------------------------
+// A gather: position of a thread in the flattened (tile, k-step) sequence
+// ---------------------------------------------------------------------------
+template <int BITS>
+struct AGather {
+    static constexpr int CH = BITS;                    // 16-byte chunks per row step
+    static constexpr int ITEMS = (BITS == 3) ? 1 : CH; // rows per thread
+    static constexpr int LOADS = (BITS == 3) ? 3 : 1;  // chunks per item
+    static constexpr int ROW_STRIDE = (BITS == 3) ? 0 : BM / CH;
+
+    int tile, ks, off, kh, kw, tap;
+    int row0, j;
+    // per item
+    int64_t base[ITEMS];      // pixel index of (n, 0, 0)
+    int hb[ITEMS], wb[ITEMS];
+    bool rv[ITEMS];
+
+    __device__ __forceinline__ void set_tile(const TcParams &p, int t, int tid)
+    {
+        tile = t;
+        ks = 0;
+        if (BITS == 3) { row0 = tid; j = 0; }
+        else { row0 = tid / CH; j = tid % CH; }
+        off = 16 * j;
+        tap = kh = kw = 0;
+        normalise(p);
+        const int m_tile = t / p.n_tiles;
+#pragma unroll
+        for (int i = 0; i < ITEMS; ++i) {
+            const int m = m_tile * BM + row0 + i * ROW_STRIDE;
+            rv[i] = m < p.M;
+            const int mm = rv[i] ? m : 0;
+            const int wo = mm % p.Wo;
+            const int ho = (mm / p.Wo) % p.Ho;
+            const int n = mm / (p.Wo * p.Ho);
+            base[i] = (int64_t)n * p.H * p.W;
+            hb[i] = ho * p.stride - p.pad;
+            wb[i] = wo * p.stride - p.pad;
+        }
+    }
+    __device__ __forceinline__ void normalise(const TcParams &p)
+    {
+        while (off >= p.P) {
+            off -= p.P;
+            ++tap;
+            if (++kw == p.KW) { kw = 0; ++kh; }
+        }
+    }
+    __device__ __forceinline__ bool valid(const TcParams &p) const
+    {
+        return tile < p.m_tiles * p.n_tiles;
+    }
+    __device__ __forceinline__ void advance(const TcParams &p, int tid)
+    {
+        if (++ks == p.ksteps) {
+            set_tile(p, tile + gridDim.x, tid);
+        } else {
+            off += 16 * CH;
+            normalise(p);
+        }
+    }
+    // Issue this step's global loads.  For 3-bit the three chunks of a row
+    // step may sit in different filter taps only when P < 48, which a GEMM
+    // (taps = 1) never has; 3-bit is GEMM-only.
+    __device__ __forceinline__ void load(const TcParams &p, uint4 (&r)[ITEMS * LOADS]) const
+    {
+#pragma unroll
+        for (int i = 0; i < ITEMS; ++i) {
+            const int hi = hb[i] + kh, wi = wb[i] + kw;
+            const bool ok = rv[i] && tap < p.taps && hi >= 0 && hi < p.H && wi >= 0 &&
+                            wi < p.W;
+            const uint8_t *src =
+                p.act + (base[i] + (int64_t)hi * p.W + wi) * p.P + off;
+#pragma unroll
+            for (int l = 0; l < LOADS; ++l) {
+                r[i * LOADS + l] = make_uint4(0u, 0u, 0u, 0u);
+                if (ok && off + 16 * l < p.P)
+                    r[i * LOADS + l] = __ldg(reinterpret_cast<const uint4 *>(src) + l);
+            }
+        }
+    }
+};
+
+// ---------------------------------------------------------------------------
+// the kernel
+// ---------------------------------------------------------------------------
+struct SmemLayout {
+    uint32_t a_tiles, b_tiles, b_packed, bars, tmem_slot, abort_flag, total;
+};
+
+__host__ __device__ inline SmemLayout smem_layout(int BN, int bits)
+{
+    SmemLayout L;
+    uint32_t o = 0;
+    L.a_tiles = o;  o += S_U * A_TILE_BYTES;
+    L.b_tiles = o;  o += S_U * BN * BK_BYTES;
+    L.b_packed = o; o += S_P * BN * 16 * bits;
+    o = (o + 127u) & ~127u;
+    L.bars = o;     o += 8 * (2 * S_U + 2 * S_P + 4);
+    L.tmem_slot = o; o += 8;
+    L.abort_flag = o; o += 8;
+    L.total = o;
+    return L;
+}
+
+template <int BITS, bool A_SIGNED>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
+{
+    constexpr bool B_SIGNED = !A_SIGNED;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>(
+        (reinterpret_cast<uintptr_t>(smem_raw) + 1023u) & ~(uintptr_t)1023u);
+    const SmemLayout L = smem_layout(p.BN, BITS);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int BN = p.BN;
+    const int total_tiles = p.m_tiles * p.n_tiles;
+    const uint32_t b_tile_bytes = BN * BK_BYTES;
+    const uint32_t b_packed_bytes = BN * 16 * BITS;
+
+    const uint32_t bars = smem_u32(smem + L.bars);
+    auto bar_u_full = [&](int s) { return bars + 8u * s; };
+    auto bar_u_empty = [&](int s) { return bars + 8u * (S_U + s); };
+    auto bar_p_full = [&](int s) { return bars + 8u * (2 * S_U + s); };
+    auto bar_p_empty = [&](int s) { return bars + 8u * (2 * S_U + S_P + s); };
+    auto bar_acc_full = [&](int s) { return bars + 8u * (2 * S_U + 2 * S_P + s); };
+    auto bar_acc_empty = [&](int s) { return bars + 8u * (2 * S_U + 2 * S_P + 2 + s); };
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + L.tmem_slot);
+    Ctl ctl{reinterpret_cast<volatile int *>(smem + L.abort_flag), p.ws};
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < S_U; ++s) {
+            mbar_init(bar_u_full(s), 8);     // 4 A-unpack warps + 4 B-unpack warps
+            mbar_init(bar_u_empty(s), 1);    // tcgen05.commit
+        }
+        for (int s = 0; s < S_P; ++s) {
+            mbar_init(bar_p_full(s), 1);     // TMA producer (+ transaction bytes)
+            mbar_init(bar_p_empty(s), 4);    // 4 B-unpack warps
+        }
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(bar_acc_full(s), 1);   // tcgen05.commit
+            mbar_init(bar_acc_empty(s), 4);  // 4 epilogue warps
+        }
+        *ctl.abort_flag = 0;
+        mbar_init_fence();
+    }
+    if (warp == WARP_MMA) {
+        tmem_alloc(smem_u32((const void *)tmem_slot), 512);
+        tmem_relinquish();
+    }
+    if (warp == WARP_TMA && lane == 0) tma_prefetch_desc(&tmap_b);
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == WARP_TMA) {
+        // ---------------- B producer: TMA packed tiles --------------------
+        if (lane == 0) {
+            uint32_t g = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+                const int n_tile = tile % p.n_tiles;
+                for (int ks = 0; ks < p.ksteps; ++ks, ++g) {
+                    const int s = g % S_P;
+                    const uint32_t ph = (g / S_P) & 1u;
+                    if (!(ok = wait_bar(bar_p_empty(s), ph ^ 1u, ctl, 1))) break;
+                    mbar_arrive_expect_tx(bar_p_full(s), b_packed_bytes);
+                    tma_load_2d(smem_u32(smem + L.b_packed + s * b_packed_bytes), &tmap_b,
+                                ks * 16 * BITS, n_tile * BN, bar_p_full(s));
+                }
+            }
+            // let outstanding copies land before the CTA can exit
+            const uint32_t issued = g;
+            for (uint32_t k = (issued > (uint32_t)S_P ? issued - S_P : 0); k < issued; ++k)
+                wait_bar(bar_p_full(k % S_P), (k / S_P) & 1u, ctl, 2);
+        }
+    } else if (warp == WARP_MMA) {
+        // ---------------- MMA issuer ---------------------------------------
+        if (lane == 0) {
+            const uint32_t idesc = idesc_i8(BN, A_SIGNED, B_SIGNED);
+            uint32_t g = 0, it = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++it) {
+                const int as = it & 1;
+                const uint32_t aph = (it >> 1) & 1u;
+                if (!(ok = wait_bar(bar_acc_empty(as), aph ^ 1u, ctl, 3))) break;
+                tc_fence_after_sync();
+                const uint32_t d_tmem = tmem_base + as * 256;
+                for (int ks = 0; ks < p.ksteps; ++ks, ++g) {
+                    const int s = g % S_U;
+                    const uint32_t ph = (g / S_U) & 1u;
+                    if (!(ok = wait_bar(bar_u_full(s), ph, ctl, 4))) break;
+                    tc_fence_after_sync();
+                    const uint64_t ad =
+                        smem_desc_sw128(smem_u32(smem + L.a_tiles + s * A_TILE_BYTES));
+                    const uint64_t bd =
+                        smem_desc_sw128(smem_u32(smem + L.b_tiles + s * b_tile_bytes));
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk)   // 32 bytes of K per instruction
+                        mma_i8(d_tmem, ad + 2 * kk, bd + 2 * kk, idesc,
+                               (ks | kk) != 0 ? 1u : 0u);
+                    mma_commit(bar_u_empty(s));
+                }
+                if (ok) mma_commit(bar_acc_full(as));
+            }
+        }
+    } else if (warp < WARP_B0) {
+        // ---------------- A: gather from global + expand --------------------
+        const int tid = threadIdx.x - WARP_A0 * 32;
+        using G = AGather<BITS>;
+        G st;
+        st.set_tile(p, blockIdx.x, tid);
+        uint4 cur[G::ITEMS * G::LOADS], nxt[G::ITEMS * G::LOADS];
+        if (st.valid(p)) st.load(p, cur);
+        uint32_t g = 0;
+        while (st.valid(p)) {
+            G nx = st;
+            nx.advance(p, tid);
+            if (nx.valid(p)) nx.load(p, nxt);
+            const int s = g % S_U;
+            const uint32_t ph = (g / S_U) & 1u;
+            if (!wait_bar(bar_u_empty(s), ph ^ 1u, ctl, 5)) break;
+            uint8_t *tile = smem + L.a_tiles + s * A_TILE_BYTES;
+            if (BITS == 3) {
+                uint32_t w[12];
+#pragma unroll
+                for (int l = 0; l < 3; ++l) {
+                    w[4 * l] = cur[l].x; w[4 * l + 1] = cur[l].y;
+                    w[4 * l + 2] = cur[l].z; w[4 * l + 3] = cur[l].w;
+                }
+                expand_row3<A_SIGNED>(tile, st.row0, w, p.orv);
+            } else {
+#pragma unroll
+                for (int i = 0; i < G::ITEMS; ++i)
+                    expand_chunk<BITS == 3 ? 4 : BITS, A_SIGNED>(
+                        tile, st.row0 + i * G::ROW_STRIDE, st.j, cur[i], p.orv);
+            }
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_u_full(s));
+#pragma unroll
+            for (int i = 0; i < G::ITEMS * G::LOADS; ++i) cur[i] = nxt[i];
+            st = nx;
+            ++g;
+        }
+    } else if (warp < WARP_E0) {
+        // ---------------- B: expand packed shared tiles ---------------------
+        const int tid = threadIdx.x - WARP_B0 * 32;
+        uint32_t g = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+            for (int ks = 0; ks < p.ksteps; ++ks, ++g) {
+                const int sp = g % S_P, su = g % S_U;
+                const uint32_t php = (g / S_P) & 1u, phu = (g / S_U) & 1u;
+                if (!(ok = wait_bar(bar_p_full(sp), php, ctl, 6))) break;
+                if (!(ok = wait_bar(bar_u_empty(su), phu ^ 1u, ctl, 7))) break;
+                const uint8_t *src = smem + L.b_packed + sp * b_packed_bytes;
+                uint8_t *dst = smem + L.b_tiles + su * b_tile_bytes;
+                if (BITS == 3) {
+                    for (int row = tid; row < BN; row += 128) {
+                        uint32_t w[12];
+                        const uint4 *r4 = reinterpret_cast<const uint4 *>(src + row * 48);
+#pragma unroll
+                        for (int l = 0; l < 3; ++l) {
+                            const uint4 v = r4[l];
+                            w[4 * l] = v.x; w[4 * l + 1] = v.y;
+                            w[4 * l + 2] = v.z; w[4 * l + 3] = v.w;
+                        }
+                        expand_row3<B_SIGNED>(dst, row, w, p.orv);
+                    }
+                } else {
+                    constexpr int CH = (BITS == 3) ? 4 : BITS;
+                    for (int c = tid; c < BN * CH; c += 128) {
+                        const uint4 v = reinterpret_cast<const uint4 *>(src)[c];
+                        expand_chunk<BITS == 3 ? 4 : BITS, B_SIGNED>(dst, c / CH, c % CH, v,
+                                                                     p.orv);
+                    }
+                }
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) {
+                    mbar_arrive(bar_u_full(su));
+                    mbar_arrive(bar_p_empty(sp));
+                }
+            }
+        }
+    } else {
+        // ---------------- epilogue -------------------------------------------
+        const int quarter = warp & 3;                 // TMEM lanes 32q .. 32q+31
+        const int row_in_tile = quarter * 32 + lane;
+        uint32_t it = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++it) {
+            const int as = it & 1;
+            const uint32_t aph = (it >> 1) & 1u;
+            const int m_tile = tile / p.n_tiles, n_tile = tile % p.n_tiles;
+            const int64_t m = (int64_t)m_tile * BM + row_in_tile;
+            const bool row_ok = m < p.M;
+            if (!(ok = wait_bar(bar_acc_full(as), aph, ctl, 8))) break;
+            tc_fence_after_sync();
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + as * 256;
+            float rs = 0.f;
+            if (p.mode == MODE_GEMM && p.row_scale && row_ok) rs = __ldg(p.row_scale + m);
+            for (int c0 = 0; c0 < BN; c0 += 32) {
+                uint32_t r[32];
+                __syncwarp();
+                tmem_ld_32x32(taddr + c0, r);
+                tmem_ld_wait();
+                const int n0 = n_tile * BN + c0;
+                if (!row_ok) continue;
+                if (p.mode == MODE_GEMM) {
+                    if (n0 >= p.Ncols) continue;
+                    const bool full = n0 + 32 <= p.Ncols && (p.Ncols & 3) == 0;
+                    if (p.C_i32) {
+                        int32_t *dst = p.C_i32 + m * p.Ncols + n0;
+                        if (full) {
+#pragma unroll
+                            for (int v = 0; v < 8; ++v)
+                                reinterpret_cast<int4 *>(dst)[v] = make_int4(
+                                    (int)r[4 * v] >> p.shift, (int)r[4 * v + 1] >> p.shift,
+                                    (int)r[4 * v + 2] >> p.shift, (int)r[4 * v + 3] >> p.shift);
+                        } else {
+#pragma unroll
+                            for (int c = 0; c < 32; ++c)
+                                if (n0 + c < p.Ncols) dst[c] = (int)r[c] >> p.shift;
+                        }
+                    }
+                    if (p.D_f32) {
+                        float *dst = p.D_f32 + m * p.Ncols + n0;
+                        if (full) {
+#pragma unroll
+                            for (int v = 0; v < 8; ++v)
+                                reinterpret_cast<float4 *>(dst)[v] = make_float4(
+                                    __fmul_rn((float)((int)r[4 * v] >> p.shift), rs),
+                                    __fmul_rn((float)((int)r[4 * v + 1] >> p.shift), rs),
+                                    __fmul_rn((float)((int)r[4 * v + 2] >> p.shift), rs),
+                                    __fmul_rn((float)((int)r[4 * v + 3] >> p.shift), rs));
+                        } else {
+#pragma unroll
+                            for (int c = 0; c < 32; ++c)
+                                if (n0 + c < p.Ncols)
+                                    dst[c] = __fmul_rn((float)((int)r[c] >> p.shift), rs);
+                        }
+                    }
+                } else {
+                    const DsqEpi &e = p.e;
+                    constexpr uint32_t MASK = (1u << BITS) - 1u;
+                    constexpr int CW = 32 * BITS / 32;       // code words per 32 columns
+                    const int byte0 = n0 * BITS / 8;
+                    uint32_t resw[CW];
+#pragma unroll
+                    for (int w = 0; w < CW; ++w) resw[w] = 0u;
+                    if (e.residual && byte0 < p.out_pitch) {
+                        const uint32_t *rp = reinterpret_cast<const uint32_t *>(
+                            e.residual + m * p.out_pitch + byte0);
+#pragma unroll
+                        for (int w = 0; w < CW; ++w) resw[w] = __ldg(rp + w);
+                    }
+                    uint32_t cw[CW];
+#pragma unroll
+                    for (int w = 0; w < CW; ++w) cw[w] = 0u;
+                    const bool full = n0 + 32 <= p.Ncols && (p.Ncols & 3) == 0;
+                    float yv[32];
+#pragma unroll
+                    for (int c = 0; c < 32; ++c) {
+                        const int n = n0 + c;
+                        const int v = (int)r[c] >> p.shift;
+                        r[c] = (uint32_t)v;
+                        float y = 0.f;
+                        if (n < p.Ncols) {
+                            float sc = __ldg(e.scale + n);
+                            if (e.half_offset) sc = __fmul_rn(sc, 0.5f);
+                            y = dsq_epi_y(v, sc, __ldg(e.bias + n));
+                            if (e.residual) {
+                                const uint32_t qr =
+                                    (resw[(c * BITS) >> 5] >> ((c * BITS) & 31)) & MASK;
+                                y = dsq_epi_residual(y, qr, e.res_delta, e.res_lo);
+                            }
+                            if (e.has_requant)
+                                cw[(c * BITS) >> 5] |= dsq_code(y, e.rq) << ((c * BITS) & 31);
+                        }
+                        yv[c] = y;
+                    }
+                    if (e.y_codes && byte0 < p.out_pitch) {
+                        uint32_t *dst = reinterpret_cast<uint32_t *>(
+                            e.y_codes + m * p.out_pitch + byte0);
+                        if (CW == 4)
+                            *reinterpret_cast<uint4 *>(dst) =
+                                make_uint4(cw[0], cw[1], cw[2], cw[CW - 1]);
+                        else
+                            *reinterpret_cast<uint2 *>(dst) = make_uint2(cw[0], cw[CW - 1]);
+                    }
+                    if (n0 < p.Ncols) {
+                        if (e.y_f32) {
+                            float *dst = e.y_f32 + m * p.Ncols + n0;
+                            if (full) {
+#pragma unroll
+                                for (int v = 0; v < 8; ++v)
+                                    reinterpret_cast<float4 *>(dst)[v] = make_float4(
+                                        yv[4 * v], yv[4 * v + 1], yv[4 * v + 2], yv[4 * v + 3]);
+                            } else {
+#pragma unroll
+                                for (int c = 0; c < 32; ++c)
+                                    if (n0 + c < p.Ncols) dst[c] = yv[c];
+                            }
+                        }
+                        if (e.acc_out) {
+                            int32_t *dst = e.acc_out + m * p.Ncols + n0;
+                            if (full) {
+#pragma unroll
+                                for (int v = 0; v < 8; ++v)
+                                    reinterpret_cast<int4 *>(dst)[v] =
+                                        make_int4((int)r[4 * v], (int)r[4 * v + 1],
+                                                  (int)r[4 * v + 2], (int)r[4 * v + 3]);
+                            } else {
+#pragma unroll
+                                for (int c = 0; c < 32; ++c)
+                                    if (n0 + c < p.Ncols) dst[c] = (int)r[c];
+                            }
+                        }
+                    }
+                }
+            }
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_acc_empty(as));
+        }
+    }
+
+    // ---------------- teardown ---------------------------------------------
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == WARP_MMA) {
+        __syncwarp();
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, 512);
+    }
+}
+
+// ---------------------------------------------------------------------------
+// tensor-core rate probe: MMAs only, operands resident in shared memory
+// ---------------------------------------------------------------------------
+__global__ void __launch_bounds__(128, 1) mma_rate_kernel(int iters, int *ws)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>(
+        (reinterpret_cast<uintptr_t>(smem_raw) + 1023u) & ~(uintptr_t)1023u);
+    __shared__ uint64_t bar_storage[2];
+    __shared__ uint32_t tmem_slot;
+    __shared__ int abort_flag;
+    const int warp = threadIdx.x >> 5;
+    // A: 128 rows x 128 B, B: 256 rows x 128 B, filled with varied bytes
+    for (int i = threadIdx.x; i < (128 + 256) * 128 / 4; i += blockDim.x)
+        reinterpret_cast<uint32_t *>(smem)[i] = 0x9E3779B9u * (uint32_t)(i + 1);
+    const uint32_t bar = smem_u32(&bar_storage[0]);
+    if (threadIdx.x == 0) {
+        mbar_init(bar, 1);
+        mbar_init(bar + 8, 1);
+        abort_flag = 0;
+        mbar_init_fence();
+    }
+    if (warp == 0) {
+        tmem_alloc(smem_u32(&tmem_slot), 256);
+        tmem_relinquish();
+    }
+    fence_proxy_async_smem();
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = tmem_slot;
+    if (threadIdx.x == 0) {
+        Ctl ctl{&abort_flag, ws};
+        const uint32_t idesc = idesc_i8(256, true, false);
+        const uint64_t ad = smem_desc_sw128(smem_u32(smem));
+        const uint64_t bd = smem_desc_sw128(smem_u32(smem + 128 * 128));
+        // batches of 64 instructions, two in flight: wait for batch b-1 only
+        // after batch b has been issued, so the pipe never drains
+        const int batches = (iters + 63) / 64;
+        bool ok = true;
+        for (int b = 0; ok && b < batches; ++b) {
+            const int n = min(64, iters - 64 * b);
+            for (int k = 0; k < n; ++k)
+                mma_i8(tmem, ad + 2 * (k & 3), bd + 2 * (k & 3), idesc, 1u);
+            mma_commit(bar + 8 * (b & 1));
+            if (b > 0)
+                ok = wait_bar(bar + 8 * ((b - 1) & 1), ((b - 1) >> 1) & 1u, ctl, 9);
+        }
+        if (ok && batches > 0)
+            wait_bar(bar + 8 * ((batches - 1) & 1), ((batches - 1) >> 1) & 1u, ctl, 9);
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 0) {
+        __syncwarp();
+        tc_fence_after_sync();
+        tmem_dealloc(tmem, 256);
+    }
+}
+
+// ---------------------------------------------------------------------------
+// host side
+// ---------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *,
+                                  const cuuint64_t *, const cuuint64_t *, const cuuint32_t *,
+                                  const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void *sym = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) ==
+                cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(sym);
+    }
+    return fn;
+}
+
+// 2-D byte map over packed rows: inner dimension = row bytes, outer = rows.
+int make_rows_tmap(CUtensorMap *map, const void *base, uint64_t row_bytes, uint64_t rows,
+                   uint64_t pitch, uint32_t box_bytes, uint32_t box_rows)
+{
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return DSQ_ERR_CUDA;
+    cuuint64_t dims[2] = {row_bytes, rows};
+    cuuint64_t strides[1] = {pitch};
+    cuuint32_t box[2] = {box_bytes, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(base), dims,
+                    strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                    CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? DSQ_OK : DSQ_ERR_CUDA;
+}
+
+int pick_bn(int m_tiles, int ncols, int bits)
+{
+    const int cands[4] = {256, 128, 64, 32};
+    int best = 0;
+    double best_cost = 1e30;
+    for (int i = 0; i < 4; ++i) {
+        const int bn = cands[i];
+        if (bits == 2 && bn < 64) continue;
+        const int n_tiles = (ncols + bn - 1) / bn;
+        const int64_t tiles = (int64_t)m_tiles * n_tiles;
+        const int64_t waves = (tiles + 147) / 148;
+        const double cost = (double)waves * (128.0 + 1.5 * bn);
+        if (cost < best_cost) { best_cost = cost; best = bn; }
+    }
+    return best;
+}
+
+template <int BITS, bool A_SIGNED>
+int launch_tc(const CUtensorMap &tmap, const TcParams &p, cudaStream_t s)
+{
+    const SmemLayout L = smem_layout(p.BN, BITS);
+    const int smem_bytes = (int)L.total + 1024;
+    static int configured = 0;
+    if (configured < smem_bytes) {
+        if (cudaFuncSetAttribute(dsq_tc_kernel<BITS, A_SIGNED>,
+                                 cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 227 * 1024) != cudaSuccess)
+            return DSQ_ERR_CUDA;
+        configured = 227 * 1024;
+    }
+    int grid = p.m_tiles * p.n_tiles;
+    if (grid > 148) grid = 148;
+    dsq_tc_kernel<BITS, A_SIGNED><<<grid, NUM_THREADS, smem_bytes, s>>>(tmap, p);
+    return dsq_launch_status();
+}
+
+int dispatch_tc(int bits, bool a_signed, const CUtensorMap &tmap, const TcParams &p,
+                cudaStream_t s)
+{
+    if (bits == 4) return a_signed ? launch_tc<4, true>(tmap, p, s) : launch_tc<4, false>(tmap, p, s);
+    if (bits == 2) return a_signed ? launch_tc<2, true>(tmap, p, s) : launch_tc<2, false>(tmap, p, s);
+    if (bits == 3 && a_signed) return launch_tc<3, true>(tmap, p, s);
+    return DSQ_ERR_UNSUPPORTED;
+}
+
+}  // namespace
+
+extern "C" {
+
+int dsq_gemm(const void *A_codes, const void *B_codes, int64_t M, int64_t N, int64_t K,
+             int bits, int32_t *C_i32, const float *row_scale, float *D_f32, void *workspace,
+             size_t ws_bytes, void *stream)
+{
+    if (!A_codes || !B_codes || !workspace) return DSQ_ERR_NULL;
+    if (!C_i32 && !D_f32) return DSQ_ERR_NULL;
+    if (D_f32 && !row_scale) return DSQ_ERR_NULL;
+    if (bits < 2 || bits > 4) return DSQ_ERR_BITS;
+    if (M <= 0 || N <= 0 || K <= 0 || M > (1 << 24) || N > (1 << 24) || K > (1 << 24))
+        return DSQ_ERR_SHAPE;
+    if ((double)K * 128.0 * (double)((1 << bits) - 1) > 2147483647.0) return DSQ_ERR_OVERFLOW;
+    if (!dsq_aligned16(A_codes) || !dsq_aligned16(B_codes) || !dsq_aligned16(workspace) ||
+        (C_i32 && !dsq_aligned16(C_i32)) || (D_f32 && !dsq_aligned16(D_f32)))
+        return DSQ_ERR_ALIGN;
+    if (ws_bytes < DSQ_WS_BYTES) return DSQ_ERR_SIZE;
+
+    const size_t pitch = dsq_row_pitch(K, bits);
+    TcParams p = {};
+    p.M = (int)M;
+    p.Ncols = (int)N;
+    p.ksteps = (int)((pitch + 16 * bits - 1) / (16 * bits));
+    p.m_tiles = (int)((M + BM - 1) / BM);
+    p.BN = pick_bn(p.m_tiles, (int)N, bits);
+    if (bits == 2 && p.BN < 64) p.BN = 64;
+    p.n_tiles = (int)((N + p.BN - 1) / p.BN);
+    p.act = (const uint8_t *)A_codes;
+    p.H = 1; p.W = (int)M; p.Ho = 1; p.Wo = (int)M;
+    p.stride = 1; p.pad = 0; p.KW = 1; p.taps = 1; p.P = (int)pitch;
+    p.mode = MODE_GEMM;
+    p.shift = 8 - bits;
+    p.orv = 0;
+    p.C_i32 = C_i32;
+    p.row_scale = row_scale;
+    p.D_f32 = D_f32;
+    p.ws = (int *)workspace;
+    CUtensorMap tmap;
+    int st = make_rows_tmap(&tmap, B_codes, pitch, (uint64_t)N, pitch, 16 * bits, p.BN);
+    if (st) return st;
+    return dispatch_tc(bits, true, tmap, p, (cudaStream_t)stream);
+}
+
+int dsq_conv2d(const void *act_codes, const dsq_nhwc_t *shape, const dsq_quant_t *act_q,
+               const void *w_packed, const dsq_conv_t *conv, const dsq_epilogue_t *ep,
+               float *y_f32, void *y_codes, int32_t *acc_out, void *workspace,
+               size_t ws_bytes, void *stream)
+{
+    if (!act_codes || !shape || !act_q || !w_packed || !conv || !ep || !workspace)
+        return DSQ_ERR_NULL;
+    int st = dsq_check_quant(act_q);
+    if (st) return st;
+    const int bits = act_q->bits;
+    if (bits == 3) return DSQ_ERR_UNSUPPORTED;
+    if (shape->N <= 0 || shape->H <= 0 || shape->W <= 0 || shape->C <= 0 || conv->Cout <= 0)
+        return DSQ_ERR_SHAPE;
+    if (conv->groups != 1 || conv->Cin != shape->C) return DSQ_ERR_SHAPE;
+    if (conv->KH != conv->KW || (conv->KH != 1 && conv->KH != 3) ||
+        (conv->stride != 1 && conv->stride != 2) || conv->pad < 0 || conv->pad > conv->KH / 2)
+        return DSQ_ERR_UNSUPPORTED;
+    if (conv->pad > 0 && act_q->lo != 0.0f) return DSQ_ERR_UNSUPPORTED;
+    const int Ho = (shape->H + 2 * conv->pad - conv->KH) / conv->stride + 1;
+    const int Wo = (shape->W + 2 * conv->pad - conv->KW) / conv->stride + 1;
+    if (Ho <= 0 || Wo <= 0) return DSQ_ERR_SHAPE;
+    const int64_t M = (int64_t)shape->N * Ho * Wo;
+    if (M > (1 << 30)) return DSQ_ERR_SHAPE;
+    const int taps = conv->KH * conv->KW;
+    if ((double)taps * conv->Cin * 128.0 * (double)((1 << bits) - 1) > 2147483647.0)
+        return DSQ_ERR_OVERFLOW;
+    if (!dsq_aligned16(act_codes) || !dsq_aligned16(w_packed) || !dsq_aligned16(workspace))
+        return DSQ_ERR_ALIGN;
+    if (ws_bytes < DSQ_WS_BYTES) return DSQ_ERR_SIZE;
+    DsqEpi e;
+    st = dsq_make_epi(ep, bits, y_f32, y_codes, acc_out, &e);
+    if (st) return st;
+
+    const size_t P = dsq_row_pitch(conv->Cin, bits);
+    const size_t row_bytes = (size_t)taps * P;
+    TcParams p = {};
+    p.M = (int)M;
+    p.Ncols = conv->Cout;
+    p.ksteps = (int)((row_bytes + 16 * bits - 1) / (16 * bits));
+    p.m_tiles = (int)((M + BM - 1) / BM);
+    p.BN = pick_bn(p.m_tiles, conv->Cout, bits);
+    p.n_tiles = (conv->Cout + p.BN - 1) / p.BN;
+    p.act = (const uint8_t *)act_codes;
+    p.H = shape->H; p.W = shape->W; p.Ho = Ho; p.Wo = Wo;
+    p.stride = conv->stride; p.pad = conv->pad; p.KW = conv->KW; p.taps = taps; p.P = (int)P;
+    p.mode = MODE_CONV;
+    p.e = e;
+    p.out_pitch = (int)dsq_row_pitch(conv->Cout, bits);
+    if (e.half_offset) {
+        p.shift = 7 - bits;
+        p.orv = 0x01010101u << (7 - bits);
+    } else {
+        p.shift = 8 - bits;
+        p.orv = 0;
+    }
+    p.ws = (int *)workspace;
+    CUtensorMap tmap;
+    st = make_rows_tmap(&tmap, w_packed, row_bytes, (uint64_t)conv->Cout, row_bytes, 16 * bits,
+                        p.BN);
+    if (st) return st;
+    return dispatch_tc(bits, false, tmap, p, (cudaStream_t)stream);
+}
+
+int dsq_probe_i8_mma_rate(int iters, float *ms_out, double *macs_out, void *workspace,
+                          size_t ws_bytes, void *stream)
+{
+    if (!ms_out || !macs_out || !workspace) return DSQ_ERR_NULL;
+    if (iters <= 0 || iters > (1 << 24)) return DSQ_ERR_SHAPE;
+    if (ws_bytes < DSQ_WS_BYTES) return DSQ_ERR_SIZE;
+    cudaStream_t s = (cudaStream_t)stream;
+    const int smem_bytes = (128 + 256) * 128 + 1024;
+    DSQ_CUDA_TRY(cudaFuncSetAttribute(mma_rate_kernel,
+                                      cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes));
+    int dev = 0, sms = 0;
+    DSQ_CUDA_TRY(cudaGetDevice(&dev));
+    DSQ_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    cudaEvent_t e0, e1;
+    DSQ_CUDA_TRY(cudaEventCreate(&e0));
+    DSQ_CUDA_TRY(cudaEventCreate(&e1));
+    mma_rate_kernel<<<sms, 128, smem_bytes, s>>>(iters < 64 ? iters : 64, (int *)workspace);
+    DSQ_CUDA_TRY(cudaEventRecord(e0, s));
+    mma_rate_kernel<<<sms, 128, smem_bytes, s>>>(iters, (int *)workspace);
+    DSQ_CUDA_TRY(cudaEventRecord(e1, s));
+    DSQ_CUDA_TRY(cudaEventSynchronize(e1));
+    DSQ_CUDA_TRY(cudaEventElapsedTime(ms_out, e0, e1));
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    *macs_out = (double)sms * (double)iters * 128.0 * 256.0 * 32.0;
+    return dsq_launch_status();
+}
+
+}  // extern "C"

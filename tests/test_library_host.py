@@ -1,0 +1,120 @@
+"""Host-side checks of the C-ABI library that need no GPU: it loads, exports
+every symbol include/dsq.h declares, its size queries agree with the format
+definition, and argument validation returns the documented status codes
+before anything is launched."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+import paper_1908_05033_b200 as dsq
+from paper_1908_05033_b200 import binding as B
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "dsq.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(dsq_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported_and_bound():
+    names = declared_functions()
+    assert "dsq_conv2d" in names and "dsq_gemm" in names and \
+        "dsq_quantize_act" in names and "dsq_pack_weights" in names and \
+        "dsq_dwconv2d" in names
+    for n in names:
+        assert hasattr(dsq.lib, n), n
+    assert set(names) == set(B.EXPORTED_SYMBOLS)
+
+
+def test_size_queries():
+    assert dsq.dsq_row_pitch(64, 4) == 32
+    assert dsq.dsq_row_pitch(144, 4) == 80
+    assert dsq.dsq_row_pitch(64, 2) == 16
+    assert dsq.dsq_row_pitch(4096, 3) == 1536
+    assert dsq.dsq_row_pitch(0, 4) == 0
+    assert dsq.dsq_packed_bytes(10, 64, 4) == 320
+    conv = B.dsq_conv_t(64, 3, 3, 64, 1, 1, 1)
+    assert dsq.dsq_weight_bytes(conv, 4) == 64 * 9 * 32      # config 1: 18432
+    dw = B.dsq_conv_t(96, 3, 3, 96, 1, 1, 96)
+    assert dsq.dsq_weight_bytes(dw, 4) == 9 * 48
+    assert dsq.dsq_workspace_bytes() >= 16
+    assert dsq.dsq_version() >= 100
+    assert "aligned" in dsq.dsq_status_string(-2)
+
+
+def test_validation_status_codes_without_a_gpu():
+    lib = dsq.lib
+    fake = C.c_void_p(0x1000)          # aligned, never dereferenced
+    odd = C.c_void_p(0x1004)
+    shape = B.dsq_nhwc_t(1, 8, 8, 64)
+    q4 = B.dsq_quant_t(4, 0.0, 2.0)
+    # NULL
+    assert lib.dsq_quantize_act(None, C.byref(shape), C.byref(q4), fake, 1 << 20, None) == -1
+    # bits
+    q9 = B.dsq_quant_t(9, 0.0, 2.0)
+    assert lib.dsq_quantize_act(fake, C.byref(shape), C.byref(q9), fake, 1 << 20, None) == -3
+    # range: hi <= lo, NaN
+    for lo, hi in [(1.0, 1.0), (2.0, 1.0), (float("nan"), 1.0), (0.0, float("inf"))]:
+        qb = B.dsq_quant_t(4, lo, hi)
+        assert lib.dsq_quantize_act(fake, C.byref(shape), C.byref(qb), fake, 1 << 20, None) == -6
+    # shape
+    bad = B.dsq_nhwc_t(1, 0, 8, 64)
+    assert lib.dsq_quantize_act(fake, C.byref(bad), C.byref(q4), fake, 1 << 20, None) == -4
+    # alignment
+    assert lib.dsq_quantize_act(odd, C.byref(shape), C.byref(q4), fake, 1 << 20, None) == -2
+    # size
+    assert lib.dsq_quantize_act(fake, C.byref(shape), C.byref(q4), fake, 100, None) == -5
+
+    # gemm
+    assert lib.dsq_gemm(fake, fake, 128, 128, 128, 4, None, None, None, fake, 256, None) == -1
+    assert lib.dsq_gemm(fake, fake, 128, 128, 128, 5, fake, None, None, fake, 256, None) == -3
+    assert lib.dsq_gemm(fake, fake, 0, 128, 128, 4, fake, None, None, fake, 256, None) == -4
+    assert lib.dsq_gemm(fake, fake, 128, 128, 128, 4, fake, None, None, fake, 8, None) == -5
+    assert lib.dsq_gemm(fake, fake, 128, 128, 128, 4, fake, None, fake, fake, 256, None) == -1
+    # K so large that 2^7 * (2^b - 1) * K overflows int32
+    assert lib.dsq_gemm(fake, fake, 128, 128, 1 << 21, 4, fake, None, None, fake, 256, None) == -7
+
+    # conv: unsupported geometry, lo != 0 with padding, 3-bit, bad w_offset
+    scale = C.c_void_p(0x2000)
+    ep = B.dsq_epilogue_t()
+    ep.scale, ep.bias = 0x2000, 0x3000
+    conv = B.dsq_conv_t(64, 3, 3, 64, 1, 1, 1)
+
+    def call(conv=conv, q=q4, ep=ep, shape=shape):
+        return lib.dsq_conv2d(fake, C.byref(shape), C.byref(q), fake, C.byref(conv),
+                              C.byref(ep), fake, None, None, fake, 256, None)
+    assert call(conv=B.dsq_conv_t(64, 5, 5, 64, 1, 2, 1)) == -8
+    assert call(conv=B.dsq_conv_t(64, 3, 3, 64, 3, 1, 1)) == -8
+    assert call(conv=B.dsq_conv_t(64, 3, 3, 32, 1, 1, 1)) == -4
+    assert call(q=B.dsq_quant_t(4, -1.0, 2.0)) == -8
+    assert call(q=B.dsq_quant_t(3, 0.0, 2.0)) == -8
+    ep2 = B.dsq_epilogue_t()
+    ep2.scale, ep2.bias, ep2.w_offset = 0x2000, 0x3000, 0.25
+    assert call(ep=ep2) == -8
+    ep3 = B.dsq_epilogue_t()
+    assert call(ep=ep3) == -1            # scale / bias missing
+    # code output requested but no requantiser given
+    assert lib.dsq_conv2d(fake, C.byref(shape), C.byref(q4), fake, C.byref(conv),
+                          C.byref(ep), None, fake, None, fake, 256, None) == -3
+
+    # depthwise wants groups = C
+    assert lib.dsq_dwconv2d(fake, C.byref(shape), C.byref(q4), fake, C.byref(conv),
+                            C.byref(ep), fake, None, None, None) == -4
+    # pool: odd extent
+    assert lib.dsq_maxpool2x2(fake, C.byref(B.dsq_nhwc_t(1, 7, 8, 64)), 4, fake, 1 << 20, None) == -4
+
+
+def test_import_fails_loudly_without_the_library(tmp_path, monkeypatch):
+    # the binding refuses to import when the shared object is absent
+    import importlib.util
+    src = open(B.__file__).read()
+    mod = tmp_path / "binding_copy.py"
+    mod.write_text(src)
+    spec = importlib.util.spec_from_file_location("binding_copy", mod)
+    m = importlib.util.module_from_spec(spec)
+    with pytest.raises(ImportError):
+        spec.loader.exec_module(m)
