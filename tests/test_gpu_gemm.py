@@ -1,0 +1,88 @@
+"""GPU parity, low-bit GEMM on the tensor cores: int32 results bit-exact
+against the oracle, fp32 dequantised results bit-exact too (one multiply)."""
+import numpy as np
+import pytest
+import torch
+
+pytestmark = pytest.mark.gpu
+
+from oracle import native
+import dsq_inputs
+from gpu_util import T, N
+
+
+@pytest.fixture(scope="module")
+def dsq():
+    import paper_1908_05033_b200 as d
+    return d
+
+
+def run(dsq, A, B, rs, bits):
+    M, K = A.shape
+    Nn = B.shape[0]
+    ws = dsq.new_workspace()
+    Ap, Bp = dsq.dsq_pack_codes(T(A), bits), dsq.dsq_pack_codes(T(B), bits)
+    Cg, Dg = dsq.dsq_gemm(Ap, Bp, M, Nn, K, bits, ws, row_scale=T(rs))
+    assert dsq.dsq_workspace_status(ws) == 0
+    return N(Cg), N(Dg)
+
+
+SIZES = [(1, 1, 1), (128, 32, 128), (128, 256, 128), (130, 70, 200),
+         (300, 257, 1000), (129, 513, 129), (64, 48, 4096), (515, 130, 771)]
+
+
+@pytest.mark.parametrize("bits", [2, 3, 4])
+@pytest.mark.parametrize("size", SIZES)
+def test_gemm_small_and_ragged(dsq, bits, size):
+    M, Nn, K = size
+    A, B, rs = dsq_inputs.gemm_case(M, Nn, K, bits)
+    C = native.gemm(A, B)
+    Cg, Dg = run(dsq, A, B, rs, bits)
+    assert np.array_equal(C, Cg)
+    assert np.array_equal(native.gemm_dequant(C, rs), Dg)
+
+
+@pytest.mark.parametrize("bits", [2, 3, 4])
+def test_gemm_extreme_codes(dsq, bits):
+    # every product at its most negative: K * (-2^(b-1)) * (2^b - 1)
+    half = 1 << (bits - 1)
+    M, Nn, K = 128, 64, 8192
+    A = np.full((M, K), -half, np.int8)
+    B = np.full((Nn, K), 2 * half - 1, np.int8)
+    rs = np.ones(M, np.float32)
+    Cg, Dg = run(dsq, A, B, rs, bits)
+    assert np.all(Cg == K * -half * (2 * half - 1))
+    A[:] = half - 1
+    Cg, _ = run(dsq, A, B, rs, bits)
+    assert np.all(Cg == K * (half - 1) * (2 * half - 1))
+    Cg, _ = run(dsq, np.zeros_like(A), B, rs, bits)
+    assert not Cg.any()
+
+
+@pytest.mark.parametrize("bits", [2, 3, 4])
+def test_gemm_1024_full(dsq, bits):
+    A, B, rs = dsq_inputs.gemm_case(1024, 1024, 1024, bits)
+    C = native.gemm(A, B)
+    Cg, Dg = run(dsq, A, B, rs, bits)
+    assert np.array_equal(C, Cg)
+    assert np.array_equal(native.gemm_dequant(C, rs), Dg)
+
+
+@pytest.mark.parametrize("bits,size", [(4, 4096), (2, 4096), (3, 4096), (4, 8192)])
+def test_gemm_full_size_sampled(dsq, bits, size):
+    """Full-size launch as the benchmark times it; 64 sampled rows x 64
+    sampled columns (4096 complete dot products) against the oracle, plus the
+    whole first tile row."""
+    A, B, rs = dsq_inputs.gemm_case(size, size, size, bits)
+    Cg, Dg = run(dsq, A, B, rs, bits)
+    rng = np.random.default_rng(size + bits)
+    rows = np.sort(rng.choice(size, 64, replace=False))
+    cols = np.sort(rng.choice(size, 64, replace=False))
+    C = native.gemm(A[rows], B[cols])
+    assert np.array_equal(C, Cg[np.ix_(rows, cols)])
+    assert np.array_equal(native.gemm_dequant(C, rs[rows]), Dg[np.ix_(rows, cols)])
+    C = native.gemm(A[size - 3:], B)                      # last rows, all columns
+    assert np.array_equal(C, Cg[size - 3:])
+    # determinism: a second run gives identical bits
+    Cg2, _ = run(dsq, A, B, rs, bits)
+    assert np.array_equal(Cg, Cg2)
