@@ -228,6 +228,12 @@ int dsq_unpack(const void *packed, int64_t rows, int64_t k, int bits,
 int dsq_probe_i8_mma_rate(int iters, float *ms_out, double *macs_out,
                           void *workspace, size_t ws_bytes, void *stream);
 
+/* Tuning hook for the tensor-core kernels: force the tile width along N
+ * (output channels) to 32, 64, 128, 192 or 256 for all later dsq_conv2d /
+ * dsq_gemm calls of this process; 0 restores the automatic choice.  Results
+ * do not depend on it. */
+int dsq_set_tile_n(int bn);
+
 /* ---- misc --------------------------------------------------------------- */
 const char *dsq_status_string(int status);
 int dsq_version(void);

@@ -72,6 +72,7 @@ _SIGNATURES = {
     "dsq_unpack": (_int, [_vp, _i64, _i64, _int, _int, _vp, _vp]),
     "dsq_probe_i8_mma_rate": (_int, [_int, C.POINTER(C.c_float),
                                      C.POINTER(C.c_double), _vp, _sz, _vp]),
+    "dsq_set_tile_n": (_int, [_int]),
     "dsq_status_string": (C.c_char_p, [_int]),
     "dsq_version": (_int, []),
 }
@@ -312,6 +313,10 @@ def dsq_gemm(A, B, M, N, K, bits, ws, row_scale=None, want_i32=True,
     _check(lib.dsq_gemm(_p(A), _p(B), M, N, K, bits, _p(Cm), _p(row_scale),
                         _p(D), _p(ws), ws.numel(), _stream()), "dsq_gemm")
     return Cm, D
+
+
+def dsq_set_tile_n(bn):
+    _check(lib.dsq_set_tile_n(bn), "dsq_set_tile_n")
 
 
 # ---- measurement ------------------------------------------------------------------

@@ -9,10 +9,14 @@
 //
 //   B: TMA (cp.async.bulk.tensor.2d) packed tile -> shared ring ->
 //      unpack warps -> int8 tile in the K-major 128B-swizzled layout
-//   A: unpack warps gather 16-byte packed chunks straight from global memory
-//      (implicit im2col, zero fill outside the image) -> same int8 layout
-//   one thread issues tcgen05.mma.kind::i8 (128 x BN x 32 per instruction),
-//      accumulating int32 in tensor memory (two accumulator buffers)
+//   A: one thread per tile row gathers the row's packed 16-byte chunks
+//      straight from global memory (implicit im2col, zero fill outside the
+//      image), expands them in registers and stores them to TENSOR MEMORY
+//      (tcgen05.st): the A operand never touches shared memory, whose
+//      bandwidth is what bounds this kernel
+//   one thread issues tcgen05.mma.kind::i8 (128 x BN x 32 per instruction,
+//      A from tensor memory, B from shared memory), accumulating int32 in
+//      tensor memory (two accumulator buffers when BN <= 192)
 //   epilogue warps read tensor memory (tcgen05.ld), apply the dequantise /
 //      requantise epilogue and write codes / fp32 / int32.
 //
@@ -40,12 +44,15 @@ namespace {
 
 constexpr int BM = 128;               // tile rows = MMA M
 constexpr int BK_BYTES = 128;         // int8 bytes per row per K step (128 codes)
-constexpr int S_U = 3;                // stages of unpacked (int8) tiles
+constexpr int S_U = 4;                // stages of expanded operands (A in TMEM, B in smem)
 constexpr int S_P = 4;                // stages of packed B tiles
-constexpr int A_TILE_BYTES = BM * BK_BYTES;   // 16 KB
+constexpr int TMEM_COLS = 512;
+constexpr int A_COL0 = TMEM_COLS - S_U * 32;  // A stages live in the top columns
 
-constexpr int WARP_TMA = 0, WARP_MMA = 1, WARP_A0 = 2, WARP_B0 = 6, WARP_E0 = 10;
-constexpr int NUM_WARPS = 14;
+constexpr int WARP_TMA = 0, WARP_MMA = 1, WARP_B0 = 6, WARP_E0 = 14;   // A warps: 2..5
+constexpr int NUM_A_WARPS = 4, NUM_B_WARPS = 8, NUM_E_WARPS = 4;
+constexpr int NUM_B_THREADS = NUM_B_WARPS * 32;
+constexpr int NUM_WARPS = 18;
 constexpr int NUM_THREADS = NUM_WARPS * 32;
 constexpr uint32_t WAIT_LIMIT = 1u << 24;     // try_wait rounds before giving up
 
@@ -53,7 +60,7 @@ enum { MODE_CONV = 0, MODE_GEMM = 1 };
 
 struct TcParams {
     // problem
-    int M, Ncols, ksteps, BN, m_tiles, n_tiles;
+    int M, Ncols, ksteps, BN, m_tiles, n_tiles, n_acc;
     // A gather geometry (a GEMM is a 1x1 convolution over an M x 1 image)
     const uint8_t *act;
     int H, W, Ho, Wo, stride, pad, KW, taps, P;
@@ -89,169 +96,93 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, const Ct
 }
 
 // ---------------------------------------------------------------------------
-// packed -> int8 expansion of one 16-byte chunk
+// packed -> int8 expansion.  One 128-code K step of a row is CH packed
+// 16-byte chunks and 32 words (128 bytes) of int8.  Word order (the same for
+// both operands): 4-bit chunk j gives words 8j..8j+3 from the even nibbles of
+// its four words and 8j+4..8j+7 from the odd nibbles; 2-bit chunk j gives
+// words 16j+4c..16j+4c+3 from bit pair c of every byte; 3-bit rows keep the
+// natural order.
 // ---------------------------------------------------------------------------
 template <int BITS, bool SIGNED>
-struct Unpack;
-
-template <bool SIGNED>
-struct Unpack<4, SIGNED> {          // 32 codes -> 2 chunks
-    static constexpr int OUT = 2;
-    __device__ static __forceinline__ uint32_t e(uint32_t w, int c, uint32_t orv)
-    {
+__device__ __forceinline__ uint32_t expand_word(uint32_t w, int c, uint32_t orv)
+{
+    if (BITS == 4) {
         if (!SIGNED) return (c == 0 ? w : (w >> 4)) & 0x0F0F0F0Fu;
         return ((c == 0 ? (w << 4) : w) & 0xF0F0F0F0u) | orv;
-    }
-};
-template <bool SIGNED>
-struct Unpack<2, SIGNED> {          // 64 codes -> 4 chunks
-    static constexpr int OUT = 4;
-    __device__ static __forceinline__ uint32_t e(uint32_t w, int c, uint32_t orv)
-    {
+    } else {
         if (!SIGNED) return (w >> (2 * c)) & 0x03030303u;
         return ((c == 3 ? w : (w << (6 - 2 * c))) & 0xC0C0C0C0u) | orv;
     }
-};
-
-// Expand chunk `v` (logical packed chunk j of the row) into row `row` of an
-// int8 tile in the 128B-swizzled K-major layout: logical 16-byte chunk q of
-// the row sits at physical chunk q ^ (row & 7).
-template <int BITS, bool SIGNED>
-__device__ __forceinline__ void expand_chunk(uint8_t *tile, int row, int j, uint4 v,
-                                             uint32_t orv)
-{
-    using U = Unpack<BITS, SIGNED>;
-    uint8_t *rowp = tile + row * BK_BYTES;
-#pragma unroll
-    for (int c = 0; c < U::OUT; ++c) {
-        const uint4 o = make_uint4(U::e(v.x, c, orv), U::e(v.y, c, orv),
-                                   U::e(v.z, c, orv), U::e(v.w, c, orv));
-        const int q = j * U::OUT + c;
-        *reinterpret_cast<uint4 *>(rowp + ((q ^ (row & 7)) << 4)) = o;
-    }
 }
 
-// 3-bit: a row step is 48 packed bytes (12 words, 128 codes).  Four codes
-// (12 bits) at a time are spread to one 32-bit word of bytes.
+// words 4q..4q+3 of a 3-bit row step held in w[12]
 template <bool SIGNED>
-__device__ __forceinline__ void expand_row3(uint8_t *tile, int row, const uint32_t (&w)[12],
-                                            uint32_t orv)
+__device__ __forceinline__ uint4 expand3_chunk(const uint32_t (&w)[12], int q, uint32_t orv)
 {
-    uint8_t *rowp = tile + row * BK_BYTES;
+    uint32_t o[4];
 #pragma unroll
-    for (int q = 0; q < 8; ++q) {          // output chunk q: codes 16q .. 16q+15
-        uint32_t o[4];
-#pragma unroll
-        for (int t = 0; t < 4; ++t) {
-            const int bit = (16 * q + 4 * t) * 3;
-            const int wi = bit >> 5, sh = bit & 31;
-            const uint32_t hi = wi + 1 < 12 ? w[wi + 1] : 0u;
-            const uint32_t x = __funnelshift_r(w[wi], hi, sh);
-            uint32_t b = (x & 7u) | ((x & 0x38u) << 5) | ((x & 0x1C0u) << 10) |
-                         ((x & 0xE00u) << 15);
-            if (SIGNED) b = (b << 5) | orv;
-            o[t] = b;
-        }
-        *reinterpret_cast<uint4 *>(rowp + ((q ^ (row & 7)) << 4)) =
-            make_uint4(o[0], o[1], o[2], o[3]);
+    for (int t = 0; t < 4; ++t) {
+        const int bit = (16 * q + 4 * t) * 3;
+        const int wi = bit >> 5, sh = bit & 31;
+        const uint32_t hi = wi + 1 < 12 ? w[wi + 1] : 0u;
+        const uint32_t x = __funnelshift_r(w[wi], hi, sh);
+        uint32_t b = (x & 7u) | ((x & 0x38u) << 5) | ((x & 0x1C0u) << 10) |
+                     ((x & 0xE00u) << 15);
+        if (SIGNED) b = (b << 5) | orv;
+        o[t] = b;
     }
+    return make_uint4(o[0], o[1], o[2], o[3]);
 }
 
-// ---------------------------------------------------------------------------
-// A gather: position of a thread in the flattened (tile, k-step) sequence
-// ---------------------------------------------------------------------------
 template <int BITS>
-struct AGather {
-    static constexpr int CH = BITS;                    // 16-byte chunks per row step
-    static constexpr int ITEMS = (BITS == 3) ? 1 : CH; // rows per thread
-    static constexpr int LOADS = (BITS == 3) ? 3 : 1;  // chunks per item
-    static constexpr int ROW_STRIDE = (BITS == 3) ? 0 : BM / CH;
-
-    int tile, ks, off, kh, kw, tap;
-    int row0, j;
-    // per item
-    int64_t base[ITEMS];      // pixel index of (n, 0, 0)
-    int hb[ITEMS], wb[ITEMS];
-    bool rv[ITEMS];
-
-    __device__ __forceinline__ void set_tile(const TcParams &p, int t, int tid)
-    {
-        tile = t;
-        ks = 0;
-        if (BITS == 3) { row0 = tid; j = 0; }
-        else { row0 = tid / CH; j = tid % CH; }
-        off = 16 * j;
-        tap = kh = kw = 0;
-        normalise(p);
-        const int m_tile = t / p.n_tiles;
-#pragma unroll
-        for (int i = 0; i < ITEMS; ++i) {
-            const int m = m_tile * BM + row0 + i * ROW_STRIDE;
-            rv[i] = m < p.M;
-            const int mm = rv[i] ? m : 0;
-            const int wo = mm % p.Wo;
-            const int ho = (mm / p.Wo) % p.Ho;
-            const int n = mm / (p.Wo * p.Ho);
-            base[i] = (int64_t)n * p.H * p.W;
-            hb[i] = ho * p.stride - p.pad;
-            wb[i] = wo * p.stride - p.pad;
-        }
-    }
-    __device__ __forceinline__ void normalise(const TcParams &p)
-    {
-        while (off >= p.P) {
-            off -= p.P;
-            ++tap;
-            if (++kw == p.KW) { kw = 0; ++kh; }
-        }
-    }
-    __device__ __forceinline__ bool valid(const TcParams &p) const
-    {
-        return tile < p.m_tiles * p.n_tiles;
-    }
-    __device__ __forceinline__ void advance(const TcParams &p, int tid)
-    {
-        if (++ks == p.ksteps) {
-            set_tile(p, tile + gridDim.x, tid);
-        } else {
-            off += 16 * CH;
-            normalise(p);
-        }
-    }
-    // Issue this step's global loads.  For 3-bit the three chunks of a row
-    // step may sit in different filter taps only when P < 48, which a GEMM
-    // (taps = 1) never has; 3-bit is GEMM-only.
-    __device__ __forceinline__ void load(const TcParams &p, uint4 (&r)[ITEMS * LOADS]) const
-    {
-#pragma unroll
-        for (int i = 0; i < ITEMS; ++i) {
-            const int hi = hb[i] + kh, wi = wb[i] + kw;
-            const bool ok = rv[i] && tap < p.taps && hi >= 0 && hi < p.H && wi >= 0 &&
-                            wi < p.W;
-            const uint8_t *src =
-                p.act + (base[i] + (int64_t)hi * p.W + wi) * p.P + off;
-#pragma unroll
-            for (int l = 0; l < LOADS; ++l) {
-                r[i * LOADS + l] = make_uint4(0u, 0u, 0u, 0u);
-                if (ok && off + 16 * l < p.P)
-                    r[i * LOADS + l] = __ldg(reinterpret_cast<const uint4 *>(src) + l);
-            }
-        }
-    }
+struct Chunks {
+    static constexpr int CH = BITS;              // packed 16-byte chunks per row step
+    static constexpr int OUT = (BITS == 4) ? 2 : 4;   // int8 chunks per packed chunk (2/4-bit)
 };
+
+// whole row step in registers: v[CH] -> o[32]
+template <int BITS, bool SIGNED>
+__device__ __forceinline__ void expand_row_regs(const uint4 (&v)[Chunks<BITS>::CH],
+                                                uint32_t orv, uint32_t (&o)[32])
+{
+    if (BITS == 3) {
+        uint32_t w[12];
+#pragma unroll
+        for (int l = 0; l < 3; ++l) {
+            w[4 * l] = v[l].x; w[4 * l + 1] = v[l].y;
+            w[4 * l + 2] = v[l].z; w[4 * l + 3] = v[l].w;
+        }
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const uint4 c = expand3_chunk<SIGNED>(w, q, orv);
+            o[4 * q] = c.x; o[4 * q + 1] = c.y; o[4 * q + 2] = c.z; o[4 * q + 3] = c.w;
+        }
+    } else {
+        constexpr int OUT = Chunks<BITS>::OUT;
+#pragma unroll
+        for (int j = 0; j < Chunks<BITS>::CH; ++j)
+#pragma unroll
+            for (int c = 0; c < OUT; ++c) {
+                const int b = (j * OUT + c) * 4;
+                o[b] = expand_word<BITS, SIGNED>(v[j].x, c, orv);
+                o[b + 1] = expand_word<BITS, SIGNED>(v[j].y, c, orv);
+                o[b + 2] = expand_word<BITS, SIGNED>(v[j].z, c, orv);
+                o[b + 3] = expand_word<BITS, SIGNED>(v[j].w, c, orv);
+            }
+    }
+}
 
 // ---------------------------------------------------------------------------
 // the kernel
 // ---------------------------------------------------------------------------
 struct SmemLayout {
-    uint32_t a_tiles, b_tiles, b_packed, bars, tmem_slot, abort_flag, total;
+    uint32_t b_tiles, b_packed, bars, tmem_slot, abort_flag, total;
 };
 
 __host__ __device__ inline SmemLayout smem_layout(int BN, int bits)
 {
     SmemLayout L;
     uint32_t o = 0;
-    L.a_tiles = o;  o += S_U * A_TILE_BYTES;
     L.b_tiles = o;  o += S_U * BN * BK_BYTES;
     L.b_packed = o; o += S_P * BN * 16 * bits;
     o = (o + 127u) & ~127u;
@@ -267,6 +198,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1)
 dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
 {
     constexpr bool B_SIGNED = !A_SIGNED;
+    constexpr int CH = Chunks<BITS>::CH;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>(
         (reinterpret_cast<uintptr_t>(smem_raw) + 1023u) & ~(uintptr_t)1023u);
@@ -289,22 +221,22 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S_U; ++s) {
-            mbar_init(bar_u_full(s), 8);     // 4 A-unpack warps + 4 B-unpack warps
+            mbar_init(bar_u_full(s), NUM_A_WARPS + NUM_B_WARPS);
             mbar_init(bar_u_empty(s), 1);    // tcgen05.commit
         }
         for (int s = 0; s < S_P; ++s) {
             mbar_init(bar_p_full(s), 1);     // TMA producer (+ transaction bytes)
-            mbar_init(bar_p_empty(s), 4);    // 4 B-unpack warps
+            mbar_init(bar_p_empty(s), NUM_B_WARPS);
         }
         for (int s = 0; s < 2; ++s) {
             mbar_init(bar_acc_full(s), 1);   // tcgen05.commit
-            mbar_init(bar_acc_empty(s), 4);  // 4 epilogue warps
+            mbar_init(bar_acc_empty(s), NUM_E_WARPS);
         }
         *ctl.abort_flag = 0;
         mbar_init_fence();
     }
     if (warp == WARP_MMA) {
-        tmem_alloc(smem_u32((const void *)tmem_slot), 512);
+        tmem_alloc(smem_u32((const void *)tmem_slot), TMEM_COLS);
         tmem_relinquish();
     }
     if (warp == WARP_TMA && lane == 0) tma_prefetch_desc(&tmap_b);
@@ -341,71 +273,109 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
             uint32_t g = 0, it = 0;
             bool ok = true;
             for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++it) {
-                const int as = it & 1;
-                const uint32_t aph = (it >> 1) & 1u;
+                const int as = p.n_acc == 2 ? (it & 1) : 0;
+                const uint32_t aph = (p.n_acc == 2 ? (it >> 1) : it) & 1u;
                 if (!(ok = wait_bar(bar_acc_empty(as), aph ^ 1u, ctl, 3))) break;
                 tc_fence_after_sync();
-                const uint32_t d_tmem = tmem_base + as * 256;
+                const uint32_t d_tmem = tmem_base + as * BN;
                 for (int ks = 0; ks < p.ksteps; ++ks, ++g) {
                     const int s = g % S_U;
                     const uint32_t ph = (g / S_U) & 1u;
                     if (!(ok = wait_bar(bar_u_full(s), ph, ctl, 4))) break;
                     tc_fence_after_sync();
-                    const uint64_t ad =
-                        smem_desc_sw128(smem_u32(smem + L.a_tiles + s * A_TILE_BYTES));
+                    const uint32_t a_tmem = tmem_base + A_COL0 + s * 32;
                     const uint64_t bd =
                         smem_desc_sw128(smem_u32(smem + L.b_tiles + s * b_tile_bytes));
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk)   // 32 bytes of K per instruction
-                        mma_i8(d_tmem, ad + 2 * kk, bd + 2 * kk, idesc,
-                               (ks | kk) != 0 ? 1u : 0u);
+                        mma_i8_ts(d_tmem, a_tmem + 8 * kk, bd + 2 * kk, idesc,
+                                  (ks | kk) != 0 ? 1u : 0u);
                     mma_commit(bar_u_empty(s));
                 }
                 if (ok) mma_commit(bar_acc_full(as));
             }
         }
     } else if (warp < WARP_B0) {
-        // ---------------- A: gather from global + expand --------------------
-        const int tid = threadIdx.x - WARP_A0 * 32;
-        using G = AGather<BITS>;
-        G st;
-        st.set_tile(p, blockIdx.x, tid);
-        uint4 cur[G::ITEMS * G::LOADS], nxt[G::ITEMS * G::LOADS];
-        if (st.valid(p)) st.load(p, cur);
-        uint32_t g = 0;
-        while (st.valid(p)) {
-            G nx = st;
-            nx.advance(p, tid);
-            if (nx.valid(p)) nx.load(p, nxt);
-            const int s = g % S_U;
-            const uint32_t ph = (g / S_U) & 1u;
-            if (!wait_bar(bar_u_empty(s), ph ^ 1u, ctl, 5)) break;
-            uint8_t *tile = smem + L.a_tiles + s * A_TILE_BYTES;
-            if (BITS == 3) {
-                uint32_t w[12];
+        // ---------------- A: one thread per tile row; global -> regs -> TMEM ----
+        const int quarter = warp & 3;
+        const int row = quarter * 32 + lane;
+        // loader position (runs one K step ahead of the consumer position)
+        int ld_tile = blockIdx.x, ld_ks = 0;
+        int tap = 0, kh = 0, kw = 0, off = 0;
+        int64_t base = 0;
+        int hb = 0, wb = 0;
+        bool row_ok = false;
+        auto set_tile = [&](int t) {
+            tap = kh = kw = off = 0;
+            if (t >= total_tiles) return;
+            const int m = (t / p.n_tiles) * BM + row;
+            row_ok = m < p.M;
+            const int mm = row_ok ? m : 0;
+            const int wo = mm % p.Wo;
+            const int ho = (mm / p.Wo) % p.Ho;
+            const int n = mm / (p.Wo * p.Ho);
+            base = (int64_t)n * p.H * p.W;
+            hb = ho * p.stride - p.pad;
+            wb = wo * p.stride - p.pad;
+        };
+        auto load_step = [&](uint4 (&v)[CH]) {
 #pragma unroll
-                for (int l = 0; l < 3; ++l) {
-                    w[4 * l] = cur[l].x; w[4 * l + 1] = cur[l].y;
-                    w[4 * l + 2] = cur[l].z; w[4 * l + 3] = cur[l].w;
+            for (int j = 0; j < CH; ++j) {
+                const int hi = hb + kh, wi = wb + kw;
+                const bool ok = row_ok && tap < p.taps && hi >= 0 && hi < p.H && wi >= 0 &&
+                                wi < p.W;
+                v[j] = make_uint4(0u, 0u, 0u, 0u);
+                if (ok)
+                    v[j] = __ldg(reinterpret_cast<const uint4 *>(
+                        p.act + (base + (int64_t)hi * p.W + wi) * p.P + off));
+                off += 16;
+                if (off == p.P) {
+                    off = 0;
+                    ++tap;
+                    if (++kw == p.KW) { kw = 0; ++kh; }
                 }
-                expand_row3<A_SIGNED>(tile, st.row0, w, p.orv);
-            } else {
-#pragma unroll
-                for (int i = 0; i < G::ITEMS; ++i)
-                    expand_chunk<BITS == 3 ? 4 : BITS, A_SIGNED>(
-                        tile, st.row0 + i * G::ROW_STRIDE, st.j, cur[i], p.orv);
             }
-            fence_proxy_async_smem();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar_u_full(s));
+            if (++ld_ks == p.ksteps) {
+                ld_ks = 0;
+                ld_tile += gridDim.x;
+                set_tile(ld_tile);
+            }
+        };
+        set_tile(ld_tile);
+        uint4 cur[CH], nxt[CH];
+        if (ld_tile < total_tiles) load_step(cur);
+        uint32_t g = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+            for (int ks = 0; ks < p.ksteps; ++ks, ++g) {
+                if (ld_tile < total_tiles) load_step(nxt);
+                const int s = g % S_U;
+                const uint32_t ph = (g / S_U) & 1u;
+                uint32_t o[32];
+                expand_row_regs<BITS, A_SIGNED>(cur, p.orv, o);
+                if (!(ok = wait_bar(bar_u_empty(s), ph ^ 1u, ctl, 5))) break;
+                tc_fence_after_sync();
+                __syncwarp();
+                tmem_st_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + A_COL0 + s * 32, o);
+                tmem_st_wait();
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_u_full(s));
 #pragma unroll
-            for (int i = 0; i < G::ITEMS * G::LOADS; ++i) cur[i] = nxt[i];
-            st = nx;
-            ++g;
+                for (int j = 0; j < CH; ++j) cur[j] = nxt[j];
+            }
         }
     } else if (warp < WARP_E0) {
         // ---------------- B: expand packed shared tiles ---------------------
         const int tid = threadIdx.x - WARP_B0 * 32;
+        // chunk c = tid + NUM_B_THREADS*i -> row = c / CH, j = c % CH; the
+        // swizzle term (row & 7) does not depend on i
+        constexpr int ROWS_PER_IT = (BITS == 3) ? NUM_B_THREADS : NUM_B_THREADS / CH;
+        constexpr int MAX_IT = (BITS == 3) ? 1 : (256 * CH) / NUM_B_THREADS;
+        const int row0 = (BITS == 3) ? tid : tid / CH;
+        const int j = (BITS == 3) ? 0 : tid % CH;
+        const int sw = row0 & 7;
+        const int n_it = (BN + ROWS_PER_IT - 1) / ROWS_PER_IT;
         uint32_t g = 0;
         bool ok = true;
         for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
@@ -413,27 +383,50 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
                 const int sp = g % S_P, su = g % S_U;
                 const uint32_t php = (g / S_P) & 1u, phu = (g / S_U) & 1u;
                 if (!(ok = wait_bar(bar_p_full(sp), php, ctl, 6))) break;
-                if (!(ok = wait_bar(bar_u_empty(su), phu ^ 1u, ctl, 7))) break;
                 const uint8_t *src = smem + L.b_packed + sp * b_packed_bytes;
                 uint8_t *dst = smem + L.b_tiles + su * b_tile_bytes;
                 if (BITS == 3) {
-                    for (int row = tid; row < BN; row += 128) {
-                        uint32_t w[12];
-                        const uint4 *r4 = reinterpret_cast<const uint4 *>(src + row * 48);
+                    uint32_t w[12];
+                    if (row0 < BN) {
+                        const uint4 *r4 = reinterpret_cast<const uint4 *>(src + row0 * 48);
 #pragma unroll
                         for (int l = 0; l < 3; ++l) {
                             const uint4 v = r4[l];
                             w[4 * l] = v.x; w[4 * l + 1] = v.y;
                             w[4 * l + 2] = v.z; w[4 * l + 3] = v.w;
                         }
-                        expand_row3<B_SIGNED>(dst, row, w, p.orv);
+                    }
+                    if (!(ok = wait_bar(bar_u_empty(su), phu ^ 1u, ctl, 7))) break;
+                    if (row0 < BN) {
+                        uint8_t *rowp = dst + row0 * BK_BYTES;
+#pragma unroll
+                        for (int q = 0; q < 8; ++q)
+                            *reinterpret_cast<uint4 *>(rowp + ((q ^ sw) << 4)) =
+                                expand3_chunk<B_SIGNED>(w, q, p.orv);
                     }
                 } else {
-                    constexpr int CH = (BITS == 3) ? 4 : BITS;
-                    for (int c = tid; c < BN * CH; c += 128) {
-                        const uint4 v = reinterpret_cast<const uint4 *>(src)[c];
-                        expand_chunk<BITS == 3 ? 4 : BITS, B_SIGNED>(dst, c / CH, c % CH, v,
-                                                                     p.orv);
+                    constexpr int OUT = Chunks<BITS>::OUT;
+                    uint4 v[MAX_IT];
+#pragma unroll
+                    for (int i = 0; i < MAX_IT; ++i)
+                        if (i < n_it && row0 + i * ROWS_PER_IT < BN)
+                            v[i] = reinterpret_cast<const uint4 *>(src)[tid + i * NUM_B_THREADS];
+                    if (!(ok = wait_bar(bar_u_empty(su), phu ^ 1u, ctl, 7))) break;
+                    uint8_t *rowp = dst + row0 * BK_BYTES;
+#pragma unroll
+                    for (int i = 0; i < MAX_IT; ++i) {
+                        if (i < n_it && row0 + i * ROWS_PER_IT < BN) {
+#pragma unroll
+                            for (int c = 0; c < OUT; ++c) {
+                                const uint4 o = make_uint4(
+                                    expand_word<BITS, B_SIGNED>(v[i].x, c, p.orv),
+                                    expand_word<BITS, B_SIGNED>(v[i].y, c, p.orv),
+                                    expand_word<BITS, B_SIGNED>(v[i].z, c, p.orv),
+                                    expand_word<BITS, B_SIGNED>(v[i].w, c, p.orv));
+                                *reinterpret_cast<uint4 *>(rowp + i * ROWS_PER_IT * BK_BYTES +
+                                                           (((j * OUT + c) ^ sw) << 4)) = o;
+                            }
+                        }
                     }
                 }
                 fence_proxy_async_smem();
@@ -451,14 +444,14 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
         uint32_t it = 0;
         bool ok = true;
         for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++it) {
-            const int as = it & 1;
-            const uint32_t aph = (it >> 1) & 1u;
+            const int as = p.n_acc == 2 ? (it & 1) : 0;
+            const uint32_t aph = (p.n_acc == 2 ? (it >> 1) : it) & 1u;
             const int m_tile = tile / p.n_tiles, n_tile = tile % p.n_tiles;
             const int64_t m = (int64_t)m_tile * BM + row_in_tile;
             const bool row_ok = m < p.M;
             if (!(ok = wait_bar(bar_acc_full(as), aph, ctl, 8))) break;
             tc_fence_after_sync();
-            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + as * 256;
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + as * BN;
             float rs = 0.f;
             if (p.mode == MODE_GEMM && p.row_scale && row_ok) rs = __ldg(p.row_scale + m);
             for (int c0 = 0; c0 < BN; c0 += 32) {
@@ -468,21 +461,23 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
                 tmem_ld_wait();
                 const int n0 = n_tile * BN + c0;
                 if (!row_ok) continue;
+#pragma unroll
+                for (int c = 0; c < 32; ++c) r[c] = (uint32_t)((int)r[c] >> p.shift);
+                const bool full = n0 + 32 <= p.Ncols && (p.Ncols & 3) == 0;
                 if (p.mode == MODE_GEMM) {
                     if (n0 >= p.Ncols) continue;
-                    const bool full = n0 + 32 <= p.Ncols && (p.Ncols & 3) == 0;
                     if (p.C_i32) {
                         int32_t *dst = p.C_i32 + m * p.Ncols + n0;
                         if (full) {
 #pragma unroll
                             for (int v = 0; v < 8; ++v)
-                                reinterpret_cast<int4 *>(dst)[v] = make_int4(
-                                    (int)r[4 * v] >> p.shift, (int)r[4 * v + 1] >> p.shift,
-                                    (int)r[4 * v + 2] >> p.shift, (int)r[4 * v + 3] >> p.shift);
+                                reinterpret_cast<int4 *>(dst)[v] =
+                                    make_int4((int)r[4 * v], (int)r[4 * v + 1],
+                                              (int)r[4 * v + 2], (int)r[4 * v + 3]);
                         } else {
 #pragma unroll
                             for (int c = 0; c < 32; ++c)
-                                if (n0 + c < p.Ncols) dst[c] = (int)r[c] >> p.shift;
+                                if (n0 + c < p.Ncols) dst[c] = (int)r[c];
                         }
                     }
                     if (p.D_f32) {
@@ -490,22 +485,22 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
                         if (full) {
 #pragma unroll
                             for (int v = 0; v < 8; ++v)
-                                reinterpret_cast<float4 *>(dst)[v] = make_float4(
-                                    __fmul_rn((float)((int)r[4 * v] >> p.shift), rs),
-                                    __fmul_rn((float)((int)r[4 * v + 1] >> p.shift), rs),
-                                    __fmul_rn((float)((int)r[4 * v + 2] >> p.shift), rs),
-                                    __fmul_rn((float)((int)r[4 * v + 3] >> p.shift), rs));
+                                reinterpret_cast<float4 *>(dst)[v] =
+                                    make_float4(__fmul_rn((float)(int)r[4 * v], rs),
+                                                __fmul_rn((float)(int)r[4 * v + 1], rs),
+                                                __fmul_rn((float)(int)r[4 * v + 2], rs),
+                                                __fmul_rn((float)(int)r[4 * v + 3], rs));
                         } else {
 #pragma unroll
                             for (int c = 0; c < 32; ++c)
                                 if (n0 + c < p.Ncols)
-                                    dst[c] = __fmul_rn((float)((int)r[c] >> p.shift), rs);
+                                    dst[c] = __fmul_rn((float)(int)r[c], rs);
                         }
                     }
                 } else {
                     const DsqEpi &e = p.e;
                     constexpr uint32_t MASK = (1u << BITS) - 1u;
-                    constexpr int CW = 32 * BITS / 32;       // code words per 32 columns
+                    constexpr int CW = BITS;                 // code words per 32 columns
                     const int byte0 = n0 * BITS / 8;
                     uint32_t resw[CW];
 #pragma unroll
@@ -519,27 +514,54 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
                     uint32_t cw[CW];
 #pragma unroll
                     for (int w = 0; w < CW; ++w) cw[w] = 0u;
-                    const bool full = n0 + 32 <= p.Ncols && (p.Ncols & 3) == 0;
-                    float yv[32];
+                    if (e.acc_out && n0 < p.Ncols) {
+                        int32_t *dst = e.acc_out + m * p.Ncols + n0;
+                        if (full) {
 #pragma unroll
-                    for (int c = 0; c < 32; ++c) {
-                        const int n = n0 + c;
-                        const int v = (int)r[c] >> p.shift;
-                        r[c] = (uint32_t)v;
-                        float y = 0.f;
-                        if (n < p.Ncols) {
-                            float sc = __ldg(e.scale + n);
-                            if (e.half_offset) sc = __fmul_rn(sc, 0.5f);
-                            y = dsq_epi_y(v, sc, __ldg(e.bias + n));
-                            if (e.residual) {
-                                const uint32_t qr =
-                                    (resw[(c * BITS) >> 5] >> ((c * BITS) & 31)) & MASK;
-                                y = dsq_epi_residual(y, qr, e.res_delta, e.res_lo);
-                            }
-                            if (e.has_requant)
-                                cw[(c * BITS) >> 5] |= dsq_code(y, e.rq) << ((c * BITS) & 31);
+                            for (int v = 0; v < 8; ++v)
+                                reinterpret_cast<int4 *>(dst)[v] =
+                                    make_int4((int)r[4 * v], (int)r[4 * v + 1],
+                                              (int)r[4 * v + 2], (int)r[4 * v + 3]);
+                        } else {
+#pragma unroll
+                            for (int c = 0; c < 32; ++c)
+                                if (n0 + c < p.Ncols) dst[c] = (int)r[c];
                         }
-                        yv[c] = y;
+                    }
+#pragma unroll
+                    for (int v = 0; v < 8; ++v) {
+                        float y4[4];
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            const int c = 4 * v + u;
+                            const int n = n0 + c;
+                            float y = 0.f;
+                            if (n < p.Ncols) {
+                                float sc = __ldg(e.scale + n);
+                                if (e.half_offset) sc = __fmul_rn(sc, 0.5f);
+                                y = dsq_epi_y((int)r[c], sc, __ldg(e.bias + n));
+                                if (e.residual) {
+                                    const uint32_t qr =
+                                        (resw[(c * BITS) >> 5] >> ((c * BITS) & 31)) & MASK;
+                                    y = dsq_epi_residual(y, qr, e.res_delta, e.res_lo);
+                                }
+                                if (e.has_requant)
+                                    cw[(c * BITS) >> 5] |= dsq_code(y, e.rq)
+                                                           << ((c * BITS) & 31);
+                            }
+                            y4[u] = y;
+                        }
+                        if (e.y_f32 && n0 + 4 * v < p.Ncols) {
+                            float *dst = e.y_f32 + m * p.Ncols + n0 + 4 * v;
+                            if (full) {
+                                *reinterpret_cast<float4 *>(dst) =
+                                    make_float4(y4[0], y4[1], y4[2], y4[3]);
+                            } else {
+#pragma unroll
+                                for (int u = 0; u < 4; ++u)
+                                    if (n0 + 4 * v + u < p.Ncols) dst[u] = y4[u];
+                            }
+                        }
                     }
                     if (e.y_codes && byte0 < p.out_pitch) {
                         uint32_t *dst = reinterpret_cast<uint32_t *>(
@@ -549,35 +571,6 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
                                 make_uint4(cw[0], cw[1], cw[2], cw[CW - 1]);
                         else
                             *reinterpret_cast<uint2 *>(dst) = make_uint2(cw[0], cw[CW - 1]);
-                    }
-                    if (n0 < p.Ncols) {
-                        if (e.y_f32) {
-                            float *dst = e.y_f32 + m * p.Ncols + n0;
-                            if (full) {
-#pragma unroll
-                                for (int v = 0; v < 8; ++v)
-                                    reinterpret_cast<float4 *>(dst)[v] = make_float4(
-                                        yv[4 * v], yv[4 * v + 1], yv[4 * v + 2], yv[4 * v + 3]);
-                            } else {
-#pragma unroll
-                                for (int c = 0; c < 32; ++c)
-                                    if (n0 + c < p.Ncols) dst[c] = yv[c];
-                            }
-                        }
-                        if (e.acc_out) {
-                            int32_t *dst = e.acc_out + m * p.Ncols + n0;
-                            if (full) {
-#pragma unroll
-                                for (int v = 0; v < 8; ++v)
-                                    reinterpret_cast<int4 *>(dst)[v] =
-                                        make_int4((int)r[4 * v], (int)r[4 * v + 1],
-                                                  (int)r[4 * v + 2], (int)r[4 * v + 3]);
-                            } else {
-#pragma unroll
-                                for (int c = 0; c < 32; ++c)
-                                    if (n0 + c < p.Ncols) dst[c] = (int)r[c];
-                            }
-                        }
                     }
                 }
             }
@@ -593,7 +586,7 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
     if (warp == WARP_MMA) {
         __syncwarp();
         tc_fence_after_sync();
-        tmem_dealloc(tmem_base, 512);
+        tmem_dealloc(tmem_base, TMEM_COLS);
     }
 }
 
@@ -698,18 +691,21 @@ int make_rows_tmap(CUtensorMap *map, const void *base, uint64_t row_bytes, uint6
     return r == CUDA_SUCCESS ? DSQ_OK : DSQ_ERR_CUDA;
 }
 
+int g_forced_bn = 0;   // dsq_set_tile_n
+
 int pick_bn(int m_tiles, int ncols, int bits)
 {
-    const int cands[4] = {256, 128, 64, 32};
+    if (g_forced_bn) return (bits == 2 && g_forced_bn < 64) ? 64 : g_forced_bn;
+    const int cands[5] = {256, 192, 128, 64, 32};
     int best = 0;
     double best_cost = 1e30;
-    for (int i = 0; i < 4; ++i) {
+    for (int i = 0; i < 5; ++i) {
         const int bn = cands[i];
         if (bits == 2 && bn < 64) continue;
         const int n_tiles = (ncols + bn - 1) / bn;
         const int64_t tiles = (int64_t)m_tiles * n_tiles;
         const int64_t waves = (tiles + 147) / 148;
-        const double cost = (double)waves * (128.0 + 1.5 * bn);
+        const double cost = (double)waves * (64.0 + (bn > 192 ? 1.1 : 1.0) * bn);
         if (cost < best_cost) { best_cost = cost; best = bn; }
     }
     return best;
@@ -730,6 +726,7 @@ int launch_tc(const CUtensorMap &tmap, const TcParams &p, cudaStream_t s)
     }
     int grid = p.m_tiles * p.n_tiles;
     if (grid > 148) grid = 148;
+    if (p.BN * p.n_acc > A_COL0) return DSQ_ERR_UNSUPPORTED;
     dsq_tc_kernel<BITS, A_SIGNED><<<grid, NUM_THREADS, smem_bytes, s>>>(tmap, p);
     return dsq_launch_status();
 }
@@ -746,6 +743,14 @@ int dispatch_tc(int bits, bool a_signed, const CUtensorMap &tmap, const TcParams
 }  // namespace
 
 extern "C" {
+
+int dsq_set_tile_n(int bn)
+{
+    if (bn != 0 && bn != 32 && bn != 64 && bn != 128 && bn != 192 && bn != 256)
+        return DSQ_ERR_SHAPE;
+    g_forced_bn = bn;
+    return DSQ_OK;
+}
 
 int dsq_gemm(const void *A_codes, const void *B_codes, int64_t M, int64_t N, int64_t K,
              int bits, int32_t *C_i32, const float *row_scale, float *D_f32, void *workspace,
@@ -772,6 +777,7 @@ int dsq_gemm(const void *A_codes, const void *B_codes, int64_t M, int64_t N, int
     p.BN = pick_bn(p.m_tiles, (int)N, bits);
     if (bits == 2 && p.BN < 64) p.BN = 64;
     p.n_tiles = (int)((N + p.BN - 1) / p.BN);
+    p.n_acc = 2 * p.BN <= A_COL0 ? 2 : 1;
     p.act = (const uint8_t *)A_codes;
     p.H = 1; p.W = (int)M; p.Ho = 1; p.Wo = (int)M;
     p.stride = 1; p.pad = 0; p.KW = 1; p.taps = 1; p.P = (int)pitch;
@@ -830,6 +836,7 @@ int dsq_conv2d(const void *act_codes, const dsq_nhwc_t *shape, const dsq_quant_t
     p.m_tiles = (int)((M + BM - 1) / BM);
     p.BN = pick_bn(p.m_tiles, conv->Cout, bits);
     p.n_tiles = (conv->Cout + p.BN - 1) / p.BN;
+    p.n_acc = 2 * p.BN <= A_COL0 ? 2 : 1;
     p.act = (const uint8_t *)act_codes;
     p.H = shape->H; p.W = shape->W; p.Ho = Ho; p.Wo = Wo;
     p.stride = conv->stride; p.pad = conv->pad; p.KW = conv->KW; p.taps = taps; p.P = (int)P;
