@@ -45,22 +45,23 @@ namespace {
 constexpr int BM = 128;               // tile rows = MMA M
 constexpr int BK_BYTES = 128;         // int8 bytes per row per K step (128 codes)
 constexpr int S_U = 4;                // stages of expanded operands (A in TMEM, B in smem)
-constexpr int S_P = 4;                // stages of packed B tiles
+constexpr int A_D = 5;                // A row steps in flight per thread (cp.async groups)
+constexpr int A_RING = A_D + 1;       // packed A ring slots
 constexpr int TMEM_COLS = 512;
 constexpr int A_COL0 = TMEM_COLS - S_U * 32;  // A stages live in the top columns
 
-constexpr int WARP_TMA = 0, WARP_MMA = 1, WARP_B0 = 6, WARP_E0 = 14;   // A warps: 2..5
-constexpr int NUM_A_WARPS = 4, NUM_B_WARPS = 8, NUM_E_WARPS = 4;
+constexpr int WARP_TMA = 0, WARP_MMA = 1, WARP_A0 = 2, WARP_B0 = 10, WARP_E0 = 18;
+constexpr int NUM_A_WARPS = 8, NUM_B_WARPS = 8, NUM_E_WARPS = 4;
 constexpr int NUM_B_THREADS = NUM_B_WARPS * 32;
-constexpr int NUM_WARPS = 18;
+constexpr int NUM_WARPS = 22;
 constexpr int NUM_THREADS = NUM_WARPS * 32;
-constexpr uint32_t WAIT_LIMIT = 1u << 24;     // try_wait rounds before giving up
+constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;   // a wait gives up after 2 s
 
 enum { MODE_CONV = 0, MODE_GEMM = 1 };
 
 struct TcParams {
     // problem
-    int M, Ncols, ksteps, BN, m_tiles, n_tiles, n_acc;
+    int M, Ncols, ksteps, BN, m_tiles, n_tiles, n_acc, s_p;
     // A gather geometry (a GEMM is a 1x1 convolution over an M x 1 image)
     const uint8_t *act;
     int H, W, Ho, Wo, stride, pad, KW, taps, P;
@@ -85,9 +86,14 @@ struct Ctl {
 __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, const Ctl &c,
                                          int tag)
 {
-    for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = global_timer_ns();
+    for (uint32_t it = 1;; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
-        if ((it & 1023u) == 1023u && *c.abort_flag) return false;
+        if ((it & 63u) == 0u) {
+            if (*c.abort_flag) return false;
+            if (global_timer_ns() - t0 > WAIT_LIMIT_NS) break;
+        }
     }
     if (atomicCAS(c.ws + DSQ_WS_STATUS, 0, (int)DSQ_ERR_TIMEOUT) == 0)
         c.ws[DSQ_WS_DETAIL] = tag;
@@ -172,21 +178,66 @@ __device__ __forceinline__ void expand_row_regs(const uint4 (&v)[Chunks<BITS>::C
     }
 }
 
+// half a row step in registers (what one A thread handles): 16 int8 words.
+// 4-bit: 2 packed chunks; 2-bit: 1 chunk; 3-bit: the 6 packed words
+// w[first..first+5] out of the 8 words held in v[0..1].
+template <int BITS, bool SIGNED>
+__device__ __forceinline__ void expand_half_regs(const uint4 (&v)[2], int half, uint32_t orv,
+                                                 uint32_t (&o)[16])
+{
+    if (BITS == 3) {
+        // half 0 loaded bytes 0..31 of the 48-byte step and owns words 0..5;
+        // half 1 loaded bytes 16..47 and owns words 6..11 = its words 2..7
+        const uint32_t l[8] = {v[0].x, v[0].y, v[0].z, v[0].w, v[1].x, v[1].y, v[1].z, v[1].w};
+        uint32_t w[7];
+#pragma unroll
+        for (int i = 0; i < 6; ++i) w[i] = half ? l[i + 2] : l[i];
+        w[6] = 0u;
+#pragma unroll
+        for (int t = 0; t < 16; ++t) {
+            const int bit = 12 * t;
+            const int wi = bit >> 5, sh = bit & 31;
+            const uint32_t x = __funnelshift_r(w[wi], w[wi + 1], sh);
+            uint32_t b = (x & 7u) | ((x & 0x38u) << 5) | ((x & 0x1C0u) << 10) |
+                         ((x & 0xE00u) << 15);
+            if (SIGNED) b = (b << 5) | orv;
+            o[t] = b;
+        }
+    } else {
+        constexpr int OUT = Chunks<BITS>::OUT;
+        constexpr int NCH = (BITS == 4) ? 2 : 1;
+#pragma unroll
+        for (int j = 0; j < NCH; ++j)
+#pragma unroll
+            for (int c = 0; c < OUT; ++c) {
+                const int b = (j * OUT + c) * 4;
+                o[b] = expand_word<BITS, SIGNED>(v[j].x, c, orv);
+                o[b + 1] = expand_word<BITS, SIGNED>(v[j].y, c, orv);
+                o[b + 2] = expand_word<BITS, SIGNED>(v[j].z, c, orv);
+                o[b + 3] = expand_word<BITS, SIGNED>(v[j].w, c, orv);
+            }
+    }
+}
+
 // ---------------------------------------------------------------------------
 // the kernel
 // ---------------------------------------------------------------------------
 struct SmemLayout {
-    uint32_t b_tiles, b_packed, bars, tmem_slot, abort_flag, total;
+    uint32_t b_tiles, b_packed, a_ring, epi, bars, tmem_slot, abort_flag, total;
 };
 
-__host__ __device__ inline SmemLayout smem_layout(int BN, int bits)
+constexpr int MAX_S_P = 4;
+
+__host__ __device__ inline SmemLayout smem_layout(int BN, int bits, int s_p)
 {
     SmemLayout L;
     uint32_t o = 0;
     L.b_tiles = o;  o += S_U * BN * BK_BYTES;
-    L.b_packed = o; o += S_P * BN * 16 * bits;
+    L.b_packed = o; o += s_p * BN * 16 * bits;
+    L.a_ring = o;   o += A_RING * BM * (bits == 3 ? 64 : 16 * bits);
+    L.epi = o;      o += NUM_E_WARPS * 64 * 4;       // per-warp scale / bias staging
     o = (o + 127u) & ~127u;
-    L.bars = o;     o += 8 * (2 * S_U + 2 * S_P + 4);
+    L.bars = o;     o += 8 * (2 * S_U + 2 * MAX_S_P + 4);
     L.tmem_slot = o; o += 8;
     L.abort_flag = o; o += 8;
     L.total = o;
@@ -202,7 +253,8 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>(
         (reinterpret_cast<uintptr_t>(smem_raw) + 1023u) & ~(uintptr_t)1023u);
-    const SmemLayout L = smem_layout(p.BN, BITS);
+    const SmemLayout L = smem_layout(p.BN, BITS, p.s_p);
+    const int S_P = p.s_p;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int BN = p.BN;
     const int total_tiles = p.m_tiles * p.n_tiles;
@@ -213,9 +265,9 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
     auto bar_u_full = [&](int s) { return bars + 8u * s; };
     auto bar_u_empty = [&](int s) { return bars + 8u * (S_U + s); };
     auto bar_p_full = [&](int s) { return bars + 8u * (2 * S_U + s); };
-    auto bar_p_empty = [&](int s) { return bars + 8u * (2 * S_U + S_P + s); };
-    auto bar_acc_full = [&](int s) { return bars + 8u * (2 * S_U + 2 * S_P + s); };
-    auto bar_acc_empty = [&](int s) { return bars + 8u * (2 * S_U + 2 * S_P + 2 + s); };
+    auto bar_p_empty = [&](int s) { return bars + 8u * (2 * S_U + MAX_S_P + s); };
+    auto bar_acc_full = [&](int s) { return bars + 8u * (2 * S_U + 2 * MAX_S_P + s); };
+    auto bar_acc_empty = [&](int s) { return bars + 8u * (2 * S_U + 2 * MAX_S_P + 2 + s); };
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + L.tmem_slot);
     Ctl ctl{reinterpret_cast<volatile int *>(smem + L.abort_flag), p.ws};
 
@@ -248,17 +300,17 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
     if (warp == WARP_TMA) {
         // ---------------- B producer: TMA packed tiles --------------------
         if (lane == 0) {
-            uint32_t g = 0;
+            uint32_t g = 0, ph = 0;
+            int s = 0;
             bool ok = true;
             for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
                 const int n_tile = tile % p.n_tiles;
                 for (int ks = 0; ks < p.ksteps; ++ks, ++g) {
-                    const int s = g % S_P;
-                    const uint32_t ph = (g / S_P) & 1u;
                     if (!(ok = wait_bar(bar_p_empty(s), ph ^ 1u, ctl, 1))) break;
                     mbar_arrive_expect_tx(bar_p_full(s), b_packed_bytes);
                     tma_load_2d(smem_u32(smem + L.b_packed + s * b_packed_bytes), &tmap_b,
                                 ks * 16 * BITS, n_tile * BN, bar_p_full(s));
+                    if (++s == S_P) { s = 0; ph ^= 1u; }
                 }
             }
             // let outstanding copies land before the CTA can exit
@@ -296,75 +348,125 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
             }
         }
     } else if (warp < WARP_B0) {
-        // ---------------- A: one thread per tile row; global -> regs -> TMEM ----
-        const int quarter = warp & 3;
+        // ---------------- A: two threads per tile row ------------------------
+        // Each thread owns half of its row's 128-code step (16 int8 words):
+        // global --cp.async--> private 16-byte cells of a shared ring (A_D steps
+        // in flight, thread-local completion) -> registers -> expand ->
+        // tensor memory (tcgen05.st).  The store of step g is completed (and
+        // the stage published) only after step g+1 has been expanded, so the
+        // store latency overlaps the next step's arithmetic.
+        const int aw = warp - WARP_A0;
+        const int quarter = warp & 3;              // TMEM lane quarter of this warp
+        const int half = aw >> 2;                  // which 16 columns of the step
         const int row = quarter * 32 + lane;
-        // loader position (runs one K step ahead of the consumer position)
-        int ld_tile = blockIdx.x, ld_ks = 0;
-        int tap = 0, kh = 0, kw = 0, off = 0;
-        int64_t base = 0;
-        int hb = 0, wb = 0;
-        bool row_ok = false;
+        constexpr int NLD = (BITS == 2) ? 1 : 2;   // 16-byte loads per thread per step
+        constexpr int PLANES = 2 * NLD;            // ring slot = PLANES x 128 rows x 16 B
+        constexpr int SLOT_BYTES = PLANES * BM * 16;
+        const uint32_t cell0 = smem_u32(smem + L.a_ring) + ((half * NLD) * BM + row) * 16;
+        // issue position (runs A_D steps ahead of the consume position)
+        int ld_tile = blockIdx.x, ld_ks = 0, ld_slot = 0;
+        int tap = 0, kw = 0, off = 0;
+        uint32_t tap_mask = 0;                     // bit t: filter tap t is inside the image
+        const uint8_t *src = p.act;
+        const int64_t row_jump = (int64_t)(p.W - p.KW) * p.P;
+        auto advance16 = [&]() {
+            off += 16;
+            src += 16;
+            if (off == p.P) {
+                off = 0;
+                ++tap;
+                if (++kw == p.KW) { kw = 0; src += row_jump; }
+            }
+        };
         auto set_tile = [&](int t) {
-            tap = kh = kw = off = 0;
+            tap = kw = off = 0;
+            tap_mask = 0;
             if (t >= total_tiles) return;
             const int m = (t / p.n_tiles) * BM + row;
-            row_ok = m < p.M;
-            const int mm = row_ok ? m : 0;
-            const int wo = mm % p.Wo;
-            const int ho = (mm / p.Wo) % p.Ho;
-            const int n = mm / (p.Wo * p.Ho);
-            base = (int64_t)n * p.H * p.W;
-            hb = ho * p.stride - p.pad;
-            wb = wo * p.stride - p.pad;
+            if (m < p.M) {
+                const int wo = m % p.Wo;
+                const int ho = (m / p.Wo) % p.Ho;
+                const int n = m / (p.Wo * p.Ho);
+                const int hb = ho * p.stride - p.pad, wb = wo * p.stride - p.pad;
+                for (int tt = 0; tt < p.taps; ++tt) {
+                    const int hi = hb + tt / p.KW, wi = wb + tt % p.KW;
+                    if (hi >= 0 && hi < p.H && wi >= 0 && wi < p.W) tap_mask |= 1u << tt;
+                }
+                src = p.act + (((int64_t)n * p.H + hb) * p.W + wb) * p.P;
+            }
+            if (BITS == 3) {
+                src += 16 * half;                  // bytes 0..31 or 16..47 of each step
+                off = 16 * half;
+            } else {
+                for (int i = 0; i < half * NLD; ++i) advance16();
+            }
         };
-        auto load_step = [&](uint4 (&v)[CH]) {
+        auto issue_step = [&]() {
+            if (ld_tile < total_tiles) {
+                const uint32_t dst = cell0 + ld_slot * SLOT_BYTES;
 #pragma unroll
-            for (int j = 0; j < CH; ++j) {
-                const int hi = hb + kh, wi = wb + kw;
-                const bool ok = row_ok && tap < p.taps && hi >= 0 && hi < p.H && wi >= 0 &&
-                                wi < p.W;
-                v[j] = make_uint4(0u, 0u, 0u, 0u);
-                if (ok)
-                    v[j] = __ldg(reinterpret_cast<const uint4 *>(
-                        p.act + (base + (int64_t)hi * p.W + wi) * p.P + off));
-                off += 16;
-                if (off == p.P) {
-                    off = 0;
-                    ++tap;
-                    if (++kw == p.KW) { kw = 0; ++kh; }
+                for (int j = 0; j < NLD; ++j) {
+                    bool ok;
+                    if (BITS == 3) ok = (tap_mask & 1u) && off + 16 * j < p.P;
+                    else ok = (tap_mask >> tap) & 1u;
+                    cp_async_16(dst + j * (BM * 16), ok ? src + (BITS == 3 ? 16 * j : 0) : p.act,
+                                ok ? 16u : 0u);
+                    if (BITS != 3) advance16();
+                }
+                if (BITS == 3) {
+                    src += 48;
+                    off += 48;
+                } else {
+#pragma unroll
+                    for (int j = 0; j < NLD; ++j) advance16();   // the other half's chunks
+                }
+                if (++ld_slot == A_RING) ld_slot = 0;
+                if (++ld_ks == p.ksteps) {
+                    ld_ks = 0;
+                    ld_tile += gridDim.x;
+                    set_tile(ld_tile);
                 }
             }
-            if (++ld_ks == p.ksteps) {
-                ld_ks = 0;
-                ld_tile += gridDim.x;
-                set_tile(ld_tile);
-            }
+            cp_async_commit();            // one group per step, empty at the tail
         };
         set_tile(ld_tile);
-        uint4 cur[CH], nxt[CH];
-        if (ld_tile < total_tiles) load_step(cur);
+#pragma unroll
+        for (int d = 0; d < A_D; ++d) issue_step();
         uint32_t g = 0;
+        int rd_slot = 0, pend_s = -1;
         bool ok = true;
+        auto publish = [&]() {
+            tmem_st_wait();
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_u_full(pend_s));
+            pend_s = -1;
+        };
         for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
             for (int ks = 0; ks < p.ksteps; ++ks, ++g) {
-                if (ld_tile < total_tiles) load_step(nxt);
+                issue_step();
+                cp_async_wait<A_D>();     // the group of this step has landed
+                uint4 cur[2];
+                cur[1] = make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+                for (int j = 0; j < NLD; ++j)
+                    cur[j] = lds_128(cell0 + rd_slot * SLOT_BYTES + j * (BM * 16));
+                if (++rd_slot == A_RING) rd_slot = 0;
+                uint32_t o[16];
+                expand_half_regs<BITS, A_SIGNED>(cur, half, p.orv, o);
+                if (pend_s >= 0) publish();
                 const int s = g % S_U;
                 const uint32_t ph = (g / S_U) & 1u;
-                uint32_t o[32];
-                expand_row_regs<BITS, A_SIGNED>(cur, p.orv, o);
                 if (!(ok = wait_bar(bar_u_empty(s), ph ^ 1u, ctl, 5))) break;
                 tc_fence_after_sync();
                 __syncwarp();
-                tmem_st_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + A_COL0 + s * 32, o);
-                tmem_st_wait();
-                tc_fence_before_sync();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar_u_full(s));
-#pragma unroll
-                for (int j = 0; j < CH; ++j) cur[j] = nxt[j];
+                tmem_st_32x16(tmem_base + ((uint32_t)(quarter * 32) << 16) + A_COL0 + s * 32 +
+                                  16 * half, o);
+                pend_s = s;
             }
         }
+        if (ok && pend_s >= 0) publish();
+        cp_async_wait<0>();
     } else if (warp < WARP_E0) {
         // ---------------- B: expand packed shared tiles ---------------------
         const int tid = threadIdx.x - WARP_B0 * 32;
@@ -376,12 +478,14 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
         const int j = (BITS == 3) ? 0 : tid % CH;
         const int sw = row0 & 7;
         const int n_it = (BN + ROWS_PER_IT - 1) / ROWS_PER_IT;
-        uint32_t g = 0;
+        uint32_t g = 0, php = 0;
+        int sp = -1;
         bool ok = true;
         for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
             for (int ks = 0; ks < p.ksteps; ++ks, ++g) {
-                const int sp = g % S_P, su = g % S_U;
-                const uint32_t php = (g / S_P) & 1u, phu = (g / S_U) & 1u;
+                if (++sp == S_P) { sp = 0; php ^= 1u; }
+                const int su = g % S_U;
+                const uint32_t phu = (g / S_U) & 1u;
                 if (!(ok = wait_bar(bar_p_full(sp), php, ctl, 6))) break;
                 const uint8_t *src = smem + L.b_packed + sp * b_packed_bytes;
                 uint8_t *dst = smem + L.b_tiles + su * b_tile_bytes;
@@ -454,10 +558,32 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + as * BN;
             float rs = 0.f;
             if (p.mode == MODE_GEMM && p.row_scale && row_ok) rs = __ldg(p.row_scale + m);
+            // per-warp staging of the chunk's 32 scale / bias values: lane i fetches
+            // column i (prefetched one chunk ahead), the warp reads them back as
+            // broadcast 128-bit shared loads
+            float *epi_scale = reinterpret_cast<float *>(smem + L.epi) + (warp - WARP_E0) * 64;
+            float *epi_bias = epi_scale + 32;
+            float sc_nx = 0.f, bi_nx = 0.f;
+            auto fetch_cols = [&](int c0) {
+                const int n = n_tile * BN + c0 + lane;
+                sc_nx = 0.f; bi_nx = 0.f;
+                if (p.mode == MODE_CONV && c0 < BN && n < p.Ncols) {
+                    sc_nx = __ldg(p.e.scale + n);
+                    if (p.e.half_offset) sc_nx = __fmul_rn(sc_nx, 0.5f);
+                    bi_nx = __ldg(p.e.bias + n);
+                }
+            };
+            fetch_cols(0);
             for (int c0 = 0; c0 < BN; c0 += 32) {
                 uint32_t r[32];
                 __syncwarp();
                 tmem_ld_32x32(taddr + c0, r);
+                if (p.mode == MODE_CONV) {
+                    epi_scale[lane] = sc_nx;
+                    epi_bias[lane] = bi_nx;
+                    fetch_cols(c0 + 32);
+                    __syncwarp();
+                }
                 tmem_ld_wait();
                 const int n0 = n_tile * BN + c0;
                 if (!row_ok) continue;
@@ -531,15 +657,17 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
 #pragma unroll
                     for (int v = 0; v < 8; ++v) {
                         float y4[4];
+                        const float4 sc4 = *reinterpret_cast<const float4 *>(epi_scale + 4 * v);
+                        const float4 bi4 = *reinterpret_cast<const float4 *>(epi_bias + 4 * v);
+                        const float scs[4] = {sc4.x, sc4.y, sc4.z, sc4.w};
+                        const float bis[4] = {bi4.x, bi4.y, bi4.z, bi4.w};
 #pragma unroll
                         for (int u = 0; u < 4; ++u) {
                             const int c = 4 * v + u;
                             const int n = n0 + c;
                             float y = 0.f;
                             if (n < p.Ncols) {
-                                float sc = __ldg(e.scale + n);
-                                if (e.half_offset) sc = __fmul_rn(sc, 0.5f);
-                                y = dsq_epi_y((int)r[c], sc, __ldg(e.bias + n));
+                                y = dsq_epi_y((int)r[c], scs[u], bis[u]);
                                 if (e.residual) {
                                     const uint32_t qr =
                                         (resw[(c * BITS) >> 5] >> ((c * BITS) & 31)) & MASK;
@@ -714,7 +842,7 @@ int pick_bn(int m_tiles, int ncols, int bits)
 template <int BITS, bool A_SIGNED>
 int launch_tc(const CUtensorMap &tmap, const TcParams &p, cudaStream_t s)
 {
-    const SmemLayout L = smem_layout(p.BN, BITS);
+    const SmemLayout L = smem_layout(p.BN, BITS, p.s_p);
     const int smem_bytes = (int)L.total + 1024;
     static int configured = 0;
     if (configured < smem_bytes) {
@@ -778,6 +906,7 @@ int dsq_gemm(const void *A_codes, const void *B_codes, int64_t M, int64_t N, int
     if (bits == 2 && p.BN < 64) p.BN = 64;
     p.n_tiles = (int)((N + p.BN - 1) / p.BN);
     p.n_acc = 2 * p.BN <= A_COL0 ? 2 : 1;
+    p.s_p = p.BN > 192 ? 3 : 4;
     p.act = (const uint8_t *)A_codes;
     p.H = 1; p.W = (int)M; p.Ho = 1; p.Wo = (int)M;
     p.stride = 1; p.pad = 0; p.KW = 1; p.taps = 1; p.P = (int)pitch;
@@ -837,6 +966,7 @@ int dsq_conv2d(const void *act_codes, const dsq_nhwc_t *shape, const dsq_quant_t
     p.BN = pick_bn(p.m_tiles, conv->Cout, bits);
     p.n_tiles = (conv->Cout + p.BN - 1) / p.BN;
     p.n_acc = 2 * p.BN <= A_COL0 ? 2 : 1;
+    p.s_p = p.BN > 192 ? 3 : 4;
     p.act = (const uint8_t *)act_codes;
     p.H = shape->H; p.W = shape->W; p.Ho = Ho; p.Wo = Wo;
     p.stride = conv->stride; p.pad = conv->pad; p.KW = conv->KW; p.taps = taps; p.P = (int)P;
