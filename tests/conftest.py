@@ -8,8 +8,22 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 
+def _build_if_stale():
+    """The shared libraries are build products (not in the history): compile
+    them when missing or older than their sources (nvcc cross-compiles without
+    a GPU)."""
+    import importlib.util
+    for name, rel in (("dsq_lib_build", "paper_1908_05033_b200/build.py"),
+                      ("dsq_oracle_build", "oracle/build.py")):
+        spec = importlib.util.spec_from_file_location(name, os.path.join(ROOT, rel))
+        mod = importlib.util.module_from_spec(spec)
+        spec.loader.exec_module(mod)
+        mod.build()
+
+
 def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (B200)")
+    _build_if_stale()
 
 
 def _have_gpu():
