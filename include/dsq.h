@@ -202,6 +202,38 @@ int dsq_gemm(const void *A_codes, const void *B_codes, int64_t M, int64_t N,
              int64_t K, int bits, int32_t *C_i32, const float *row_scale,
              float *D_f32, void *workspace, size_t ws_bytes, void *stream);
 
+/* dsq_gemm for callers that cannot allocate device memory.  (The paper has
+ * no counterpart: this is a deployment convenience of the library.)
+ *
+ * dsq_gemm needs a small device workspace from its caller.  Some callers have
+ * no way to provide one: code running inside a host framework whose memory
+ * pool they may not touch, plug-ins loaded after the application has handed
+ * all device memory to its own allocator, or real-time loops in which
+ * cudaMalloc (which synchronises the device) is forbidden.  This variant
+ * takes the same operands and outputs but no workspace: it uses a 256-byte
+ * array that is part of the library image on every GPU that loads it (held
+ * until the process exits).  It calls no allocator of any kind.
+ *
+ *  - Limits: M, N, K <= 65536 each; larger problems return DSQ_ERR_SIZE
+ *    (use dsq_gemm with your own workspace).  The scratch itself does not
+ *    grow with the problem.
+ *  - The first call on a device looks up the array's device address.  Make
+ *    that first call with the device current and before starting any stream
+ *    capture on it.
+ *  - The array is shared by every call on the device and keeps the last
+ *    call's contents; each call clears it on `stream` before launching.  Two
+ *    calls that can overlap on the GPU (different streams, no dependency
+ *    between them) race on it: order them, or use dsq_gemm.
+ *  - wait_and_check != 0: the call synchronises `stream` and returns the
+ *    device-side status (DSQ_OK or DSQ_ERR_TIMEOUT), like
+ *    dsq_workspace_status.  With 0 it returns after enqueueing, and a later
+ *    call with wait_and_check reports only its own launch.
+ * Results are identical to dsq_gemm's. */
+int dsq_gemm_static_ws(const void *A_codes, const void *B_codes, int64_t M,
+                       int64_t N, int64_t K, int bits, int32_t *C_i32,
+                       const float *row_scale, float *D_f32,
+                       int wait_and_check, void *stream);
+
 /* 2x2 stride-2 max-pool on packed unsigned codes (exact on codes because the
  * quantiser is monotone).  H and W must be even. */
 int dsq_maxpool2x2(const void *codes_in, const dsq_nhwc_t *shape, int bits,

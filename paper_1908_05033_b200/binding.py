@@ -66,6 +66,8 @@ _SIGNATURES = {
                             _vp, _vp, _vp, _vp]),
     "dsq_gemm": (_int, [_vp, _vp, _i64, _i64, _i64, _int, _vp, _vp, _vp, _vp,
                         _sz, _vp]),
+    "dsq_gemm_static_ws": (_int, [_vp, _vp, _i64, _i64, _i64, _int, _vp, _vp, _vp,
+                                  _int, _vp]),
     "dsq_maxpool2x2": (_int, [_vp, C.POINTER(dsq_nhwc_t), _int, _vp, _sz,
                               _vp]),
     "dsq_pack_codes": (_int, [_vp, _i64, _i64, _int, _vp, _sz, _vp]),
@@ -317,6 +319,20 @@ def dsq_gemm(A, B, M, N, K, bits, ws, row_scale=None, want_i32=True,
 
 def dsq_set_tile_n(bn):
     _check(lib.dsq_set_tile_n(bn), "dsq_set_tile_n")
+
+
+def dsq_gemm_static_ws(A, B, M, N, K, bits, out_i32=None, row_scale=None,
+                       out_f32=None, wait_and_check=True):
+    """dsq_gemm without a caller workspace (the library's own 256-byte static
+    array is the scratch).  The caller passes the outputs; nothing is
+    allocated here.  Returns the status of the call."""
+    _need(A, torch.uint8, "A")
+    _need(B, torch.uint8, "B")
+    st = lib.dsq_gemm_static_ws(_p(A), _p(B), M, N, K, bits, _p(out_i32),
+                                _p(row_scale), _p(out_f32),
+                                int(wait_and_check), _stream())
+    _check(st, "dsq_gemm_static_ws")
+    return st
 
 
 # ---- measurement ------------------------------------------------------------------

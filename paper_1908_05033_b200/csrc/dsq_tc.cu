@@ -40,6 +40,13 @@
 
 using namespace dsq_ptx;
 
+// Scratch of dsq_gemm_static_ws: the workspace (status word, failure detail)
+// that dsq_gemm normally receives from its caller, held by the library
+// itself.  One copy lives on every GPU that loads the library, until exit.
+#define DSQ_STATIC_WS_BYTES 256
+#define DSQ_STATIC_WS_MAX_DIM 65536
+static __device__ __align__(256) unsigned char g_static_ws[DSQ_STATIC_WS_BYTES];
+
 namespace {
 
 constexpr int BM = 128;               // tile rows = MMA M
@@ -1014,6 +1021,38 @@ int dsq_probe_i8_mma_rate(int iters, float *ms_out, double *macs_out, void *work
     cudaEventDestroy(e1);
     *macs_out = (double)sms * (double)iters * 128.0 * 256.0 * 32.0;
     return dsq_launch_status();
+}
+
+int dsq_gemm_static_ws(const void *A_codes, const void *B_codes, int64_t M, int64_t N,
+                       int64_t K, int bits, int32_t *C_i32, const float *row_scale,
+                       float *D_f32, int wait_and_check, void *stream)
+{
+    static_assert(DSQ_STATIC_WS_BYTES >= DSQ_WS_BYTES, "static workspace too small");
+    if (M > DSQ_STATIC_WS_MAX_DIM || N > DSQ_STATIC_WS_MAX_DIM || K > DSQ_STATIC_WS_MAX_DIM)
+        return DSQ_ERR_SIZE;
+    // In host code `g_static_ws` is only a handle for the symbol, not a device
+    // address.  The address on the current device is looked up once per device
+    // (no allocation happens: the array is part of the loaded module).
+    static void *dev_ptr[64] = {};
+    int dev = -1;
+    DSQ_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return DSQ_ERR_UNSUPPORTED;
+    if (!dev_ptr[dev]) {
+        void *ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_static_ws) != cudaSuccess || !ptr) return DSQ_ERR_CUDA;
+        dev_ptr[dev] = ptr;
+    }
+    void *ws = dev_ptr[dev];
+    cudaStream_t s = (cudaStream_t)stream;
+    // the array keeps what the previous call left: the status words start at 0
+    DSQ_CUDA_TRY(cudaMemsetAsync(ws, 0, DSQ_STATIC_WS_BYTES, s));
+    const int st = dsq_gemm(A_codes, B_codes, M, N, K, bits, C_i32, row_scale, D_f32, ws,
+                            DSQ_STATIC_WS_BYTES, stream);
+    if (st != DSQ_OK || !wait_and_check) return st;
+    int host[2] = {0, 0};
+    DSQ_CUDA_TRY(cudaMemcpyAsync(host, ws, sizeof(host), cudaMemcpyDeviceToHost, s));
+    DSQ_CUDA_TRY(cudaStreamSynchronize(s));
+    return host[DSQ_WS_STATUS];
 }
 
 }  // extern "C"
