@@ -65,6 +65,9 @@ constexpr int NUM_THREADS = NUM_WARPS * 32;
 constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;   // a wait gives up after 2 s
 
 enum { MODE_CONV = 0, MODE_GEMM = 1 };
+// epilogue variants (template parameter): GEMM; convolution writing codes
+// only, without / with a residual operand; convolution with any outputs
+enum { EPI_GEMM = 0, EPI_CODES = 1, EPI_CODES_RES = 2, EPI_GENERAL = 3 };
 
 struct TcParams {
     // problem
@@ -73,7 +76,7 @@ struct TcParams {
     const uint8_t *act;
     int H, W, Ho, Wo, stride, pad, KW, taps, P;
     // epilogue
-    int mode, shift, out_pitch;
+    int mode, shift, out_pitch, small_acc;
     DsqEpi e;
     int32_t *C_i32;
     const float *row_scale;
@@ -90,8 +93,9 @@ struct Ctl {
     int *ws;
 };
 
-__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, const Ctl &c,
-                                         int tag)
+// Not inlined on purpose: the kernel has a dozen wait sites and its code must
+// stay small enough for the instruction caches.
+__device__ __noinline__ bool wait_bar(uint32_t bar, uint32_t parity, const Ctl &c, int tag)
 {
     if (mbar_try_wait(bar, parity)) return true;
     const uint64_t t0 = global_timer_ns();
@@ -251,7 +255,7 @@ __host__ __device__ inline SmemLayout smem_layout(int BN, int bits, int s_p)
     return L;
 }
 
-template <int BITS, bool A_SIGNED>
+template <int BITS, bool A_SIGNED, int EPI>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
 {
@@ -310,8 +314,10 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
             uint32_t g = 0, ph = 0;
             int s = 0;
             bool ok = true;
+#pragma unroll 1
             for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
                 const int n_tile = tile % p.n_tiles;
+#pragma unroll 1
                 for (int ks = 0; ks < p.ksteps; ++ks, ++g) {
                     if (!(ok = wait_bar(bar_p_empty(s), ph ^ 1u, ctl, 1))) break;
                     mbar_arrive_expect_tx(bar_p_full(s), b_packed_bytes);
@@ -331,12 +337,14 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
             const uint32_t idesc = idesc_i8(BN, A_SIGNED, B_SIGNED);
             uint32_t g = 0, it = 0;
             bool ok = true;
+#pragma unroll 1
             for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++it) {
                 const int as = p.n_acc == 2 ? (it & 1) : 0;
                 const uint32_t aph = (p.n_acc == 2 ? (it >> 1) : it) & 1u;
                 if (!(ok = wait_bar(bar_acc_empty(as), aph ^ 1u, ctl, 3))) break;
                 tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + as * BN;
+#pragma unroll 1
                 for (int ks = 0; ks < p.ksteps; ++ks, ++g) {
                     const int s = g % S_U;
                     const uint32_t ph = (g / S_U) & 1u;
@@ -371,7 +379,8 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
         constexpr int SLOT_BYTES = PLANES * BM * 16;
         const uint32_t cell0 = smem_u32(smem + L.a_ring) + ((half * NLD) * BM + row) * 16;
         // issue position (runs A_D steps ahead of the consume position)
-        int ld_tile = blockIdx.x, ld_ks = 0, ld_slot = 0;
+        // (starts one tile back with ld_ks at its end: the first issue advances)
+        int ld_tile = (int)blockIdx.x - (int)gridDim.x, ld_ks = p.ksteps, ld_slot = 0;
         int tap = 0, kw = 0, off = 0;
         uint32_t tap_mask = 0;                     // bit t: filter tap t is inside the image
         const uint8_t *src = p.act;
@@ -395,9 +404,10 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
                 const int ho = (m / p.Wo) % p.Ho;
                 const int n = m / (p.Wo * p.Ho);
                 const int hb = ho * p.stride - p.pad, wb = wo * p.stride - p.pad;
-                for (int tt = 0; tt < p.taps; ++tt) {
-                    const int hi = hb + tt / p.KW, wi = wb + tt % p.KW;
+                for (int tt = 0, th = 0, tw = 0; tt < p.taps; ++tt) {
+                    const int hi = hb + th, wi = wb + tw;
                     if (hi >= 0 && hi < p.H && wi >= 0 && wi < p.W) tap_mask |= 1u << tt;
+                    if (++tw == p.KW) { tw = 0; ++th; }
                 }
                 src = p.act + (((int64_t)n * p.H + hb) * p.W + wb) * p.P;
             }
@@ -409,6 +419,11 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
             }
         };
         auto issue_step = [&]() {
+            if (ld_ks == p.ksteps) {
+                ld_ks = 0;
+                ld_tile += gridDim.x;
+                set_tile(ld_tile);
+            }
             if (ld_tile < total_tiles) {
                 const uint32_t dst = cell0 + ld_slot * SLOT_BYTES;
 #pragma unroll
@@ -428,18 +443,13 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
                     for (int j = 0; j < NLD; ++j) advance16();   // the other half's chunks
                 }
                 if (++ld_slot == A_RING) ld_slot = 0;
-                if (++ld_ks == p.ksteps) {
-                    ld_ks = 0;
-                    ld_tile += gridDim.x;
-                    set_tile(ld_tile);
-                }
+                ++ld_ks;
             }
             cp_async_commit();            // one group per step, empty at the tail
         };
-        set_tile(ld_tile);
-#pragma unroll
-        for (int d = 0; d < A_D; ++d) issue_step();
-        uint32_t g = 0;
+        int my_tiles = 0;
+        for (int t = blockIdx.x; t < total_tiles; t += gridDim.x) ++my_tiles;
+        const uint32_t n_steps = (uint32_t)my_tiles * p.ksteps;
         int rd_slot = 0, pend_s = -1;
         bool ok = true;
         auto publish = [&]() {
@@ -449,28 +459,31 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
             if (lane == 0) mbar_arrive(bar_u_full(pend_s));
             pend_s = -1;
         };
-        for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
-            for (int ks = 0; ks < p.ksteps; ++ks, ++g) {
-                issue_step();
-                cp_async_wait<A_D>();     // the group of this step has landed
-                uint4 cur[2];
-                cur[1] = make_uint4(0u, 0u, 0u, 0u);
+        // one loop, one issue site: iteration i issues step i and consumes step
+        // i - A_D (the first A_D iterations only fill the ring)
+#pragma unroll 1
+        for (uint32_t i = 0; ok && i < n_steps + A_D; ++i) {
+            issue_step();
+            if (i < (uint32_t)A_D) continue;
+            const uint32_t g = i - A_D;
+            cp_async_wait<A_D>();         // the group of step g has landed
+            uint4 cur[2];
+            cur[1] = make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
-                for (int j = 0; j < NLD; ++j)
-                    cur[j] = lds_128(cell0 + rd_slot * SLOT_BYTES + j * (BM * 16));
-                if (++rd_slot == A_RING) rd_slot = 0;
-                uint32_t o[16];
-                expand_half_regs<BITS, A_SIGNED>(cur, half, p.orv, o);
-                if (pend_s >= 0) publish();
-                const int s = g % S_U;
-                const uint32_t ph = (g / S_U) & 1u;
-                if (!(ok = wait_bar(bar_u_empty(s), ph ^ 1u, ctl, 5))) break;
-                tc_fence_after_sync();
-                __syncwarp();
-                tmem_st_32x16(tmem_base + ((uint32_t)(quarter * 32) << 16) + A_COL0 + s * 32 +
-                                  16 * half, o);
-                pend_s = s;
-            }
+            for (int j = 0; j < NLD; ++j)
+                cur[j] = lds_128(cell0 + rd_slot * SLOT_BYTES + j * (BM * 16));
+            if (++rd_slot == A_RING) rd_slot = 0;
+            uint32_t o[16];
+            expand_half_regs<BITS, A_SIGNED>(cur, half, p.orv, o);
+            if (pend_s >= 0) publish();
+            const int s = g % S_U;
+            const uint32_t ph = (g / S_U) & 1u;
+            if (!(ok = wait_bar(bar_u_empty(s), ph ^ 1u, ctl, 5))) break;
+            tc_fence_after_sync();
+            __syncwarp();
+            tmem_st_32x16(tmem_base + ((uint32_t)(quarter * 32) << 16) + A_COL0 + s * 32 +
+                              16 * half, o);
+            pend_s = s;
         }
         if (ok && pend_s >= 0) publish();
         cp_async_wait<0>();
@@ -488,7 +501,9 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
         uint32_t g = 0, php = 0;
         int sp = -1;
         bool ok = true;
+#pragma unroll 1
         for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+#pragma unroll 1
             for (int ks = 0; ks < p.ksteps; ++ks, ++g) {
                 if (++sp == S_P) { sp = 0; php ^= 1u; }
                 const int su = g % S_U;
@@ -554,6 +569,7 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
         const int row_in_tile = quarter * 32 + lane;
         uint32_t it = 0;
         bool ok = true;
+#pragma unroll 1
         for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++it) {
             const int as = p.n_acc == 2 ? (it & 1) : 0;
             const uint32_t aph = (p.n_acc == 2 ? (it >> 1) : it) & 1u;
@@ -564,7 +580,7 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
             tc_fence_after_sync();
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + as * BN;
             float rs = 0.f;
-            if (p.mode == MODE_GEMM && p.row_scale && row_ok) rs = __ldg(p.row_scale + m);
+            if (EPI == EPI_GEMM && p.row_scale && row_ok) rs = __ldg(p.row_scale + m);
             // per-warp staging of the chunk's 32 scale / bias values: lane i fetches
             // column i (prefetched one chunk ahead), the warp reads them back as
             // broadcast 128-bit shared loads
@@ -574,18 +590,19 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
             auto fetch_cols = [&](int c0) {
                 const int n = n_tile * BN + c0 + lane;
                 sc_nx = 0.f; bi_nx = 0.f;
-                if (p.mode == MODE_CONV && c0 < BN && n < p.Ncols) {
+                if (EPI != EPI_GEMM && c0 < BN && n < p.Ncols) {
                     sc_nx = __ldg(p.e.scale + n);
                     if (p.e.half_offset) sc_nx = __fmul_rn(sc_nx, 0.5f);
                     bi_nx = __ldg(p.e.bias + n);
                 }
             };
             fetch_cols(0);
+#pragma unroll 1
             for (int c0 = 0; c0 < BN; c0 += 32) {
                 uint32_t r[32];
                 __syncwarp();
                 tmem_ld_32x32(taddr + c0, r);
-                if (p.mode == MODE_CONV) {
+                if (EPI != EPI_GEMM) {
                     epi_scale[lane] = sc_nx;
                     epi_bias[lane] = bi_nx;
                     fetch_cols(c0 + 32);
@@ -597,7 +614,7 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
 #pragma unroll
                 for (int c = 0; c < 32; ++c) r[c] = (uint32_t)((int)r[c] >> p.shift);
                 const bool full = n0 + 32 <= p.Ncols && (p.Ncols & 3) == 0;
-                if (p.mode == MODE_GEMM) {
+                if (EPI == EPI_GEMM) {
                     if (n0 >= p.Ncols) continue;
                     if (p.C_i32) {
                         int32_t *dst = p.C_i32 + m * p.Ncols + n0;
@@ -630,6 +647,72 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
                                     dst[c] = __fmul_rn((float)(int)r[c], rs);
                         }
                     }
+                } else if (EPI == EPI_CODES || EPI == EPI_CODES_RES) {
+                    // codes-only convolution epilogue (the form the stacks use):
+                    // four columns at a time, their scale / bias vectors fetched
+                    // one group ahead; exact int->float and floor are taken with
+                    // the 2^23 bias trick so the conversion unit stays idle
+                    const DsqEpi &e = p.e;
+                    constexpr uint32_t MASK = (1u << BITS) - 1u;
+                    constexpr int CW = BITS;                 // code words per 32 columns
+                    const int byte0 = n0 * BITS / 8;
+                    if (byte0 >= p.out_pitch) continue;
+                    uint32_t resw[CW];
+#pragma unroll
+                    for (int w = 0; w < CW; ++w) resw[w] = 0u;
+                    if (EPI == EPI_CODES_RES) {
+                        const uint32_t *rp = reinterpret_cast<const uint32_t *>(
+                            e.residual + m * p.out_pitch + byte0);
+#pragma unroll
+                        for (int w = 0; w < CW; ++w) resw[w] = __ldg(rp + w);
+                    }
+                    uint32_t cw[CW];
+#pragma unroll
+                    for (int w = 0; w < CW; ++w) cw[w] = 0u;
+                    const float4 *sc4 = reinterpret_cast<const float4 *>(epi_scale);
+                    const float4 *bi4 = reinterpret_cast<const float4 *>(epi_bias);
+                    float4 s_nx = sc4[0], b_nx = bi4[0];
+#pragma unroll
+                    for (int v = 0; v < 8; ++v) {
+                        const float4 s_cur = s_nx, b_cur = b_nx;
+                        if (v < 7) { s_nx = sc4[v + 1]; b_nx = bi4[v + 1]; }
+                        const float scs[4] = {s_cur.x, s_cur.y, s_cur.z, s_cur.w};
+                        const float bis[4] = {b_cur.x, b_cur.y, b_cur.z, b_cur.w};
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            const int c = 4 * v + u;
+                            const float vf = p.small_acc
+                                ? __fsub_rn(__int_as_float(0x4B400000 + (int)r[c]), 12582912.0f)
+                                : (float)(int)r[c];
+                            float y = __fmaf_rn(vf, scs[u], bis[u]);
+                            if (EPI == EPI_CODES_RES) {
+                                const uint32_t qr =
+                                    (resw[(c * BITS) >> 5] >> ((c * BITS) & 31)) & MASK;
+                                const float qf =
+                                    __fsub_rn(__int_as_float(0x4B000000 | qr), 8388608.0f);
+                                y = __fadd_rn(y, __fmaf_rn(qf, e.res_delta, e.res_lo));
+                            }
+                            const float xc = fminf(fmaxf(y, e.rq.lo), e.rq.hi);
+                            const float rr = __fmaf_rn(__fsub_rn(xc, e.rq.lo), e.rq.inv, 0.5f);
+                            const uint32_t q =
+                                min((uint32_t)__float_as_int(__fadd_rd(rr, 8388608.0f)) - 0x4B000000u,
+                                    (uint32_t)e.rq.qmax);
+                            cw[(c * BITS) >> 5] |= q << ((c * BITS) & 31);
+                        }
+                    }
+                    // columns past Cout are padding lanes of the packed row: zero
+                    const int nvalid_bits = min(32, max(0, p.Ncols - n0)) * BITS;
+#pragma unroll
+                    for (int w = 0; w < CW; ++w) {
+                        const int nb = nvalid_bits - 32 * w;
+                        cw[w] &= nb >= 32 ? 0xFFFFFFFFu : nb <= 0 ? 0u : ((1u << nb) - 1u);
+                    }
+                    uint32_t *dst =
+                        reinterpret_cast<uint32_t *>(e.y_codes + m * p.out_pitch + byte0);
+                    if (CW == 4)
+                        *reinterpret_cast<uint4 *>(dst) = make_uint4(cw[0], cw[1], cw[2], cw[CW - 1]);
+                    else
+                        *reinterpret_cast<uint2 *>(dst) = make_uint2(cw[0], cw[CW - 1]);
                 } else {
                     const DsqEpi &e = p.e;
                     constexpr uint32_t MASK = (1u << BITS) - 1u;
@@ -846,32 +929,46 @@ int pick_bn(int m_tiles, int ncols, int bits)
     return best;
 }
 
-template <int BITS, bool A_SIGNED>
+template <int BITS, bool A_SIGNED, int EPI>
 int launch_tc(const CUtensorMap &tmap, const TcParams &p, cudaStream_t s)
 {
     const SmemLayout L = smem_layout(p.BN, BITS, p.s_p);
     const int smem_bytes = (int)L.total + 1024;
-    static int configured = 0;
-    if (configured < smem_bytes) {
-        if (cudaFuncSetAttribute(dsq_tc_kernel<BITS, A_SIGNED>,
+    static bool configured = false;
+    if (!configured) {
+        if (cudaFuncSetAttribute(dsq_tc_kernel<BITS, A_SIGNED, EPI>,
                                  cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  227 * 1024) != cudaSuccess)
             return DSQ_ERR_CUDA;
-        configured = 227 * 1024;
+        configured = true;
     }
     int grid = p.m_tiles * p.n_tiles;
     if (grid > 148) grid = 148;
     if (p.BN * p.n_acc > A_COL0) return DSQ_ERR_UNSUPPORTED;
-    dsq_tc_kernel<BITS, A_SIGNED><<<grid, NUM_THREADS, smem_bytes, s>>>(tmap, p);
+    dsq_tc_kernel<BITS, A_SIGNED, EPI><<<grid, NUM_THREADS, smem_bytes, s>>>(tmap, p);
     return dsq_launch_status();
 }
 
-int dispatch_tc(int bits, bool a_signed, const CUtensorMap &tmap, const TcParams &p,
-                cudaStream_t s)
+template <int BITS>
+int launch_conv(int epi, const CUtensorMap &tmap, const TcParams &p, cudaStream_t s)
 {
-    if (bits == 4) return a_signed ? launch_tc<4, true>(tmap, p, s) : launch_tc<4, false>(tmap, p, s);
-    if (bits == 2) return a_signed ? launch_tc<2, true>(tmap, p, s) : launch_tc<2, false>(tmap, p, s);
-    if (bits == 3 && a_signed) return launch_tc<3, true>(tmap, p, s);
+    switch (epi) {
+    case EPI_CODES: return launch_tc<BITS, false, EPI_CODES>(tmap, p, s);
+    case EPI_CODES_RES: return launch_tc<BITS, false, EPI_CODES_RES>(tmap, p, s);
+    default: return launch_tc<BITS, false, EPI_GENERAL>(tmap, p, s);
+    }
+}
+
+int dispatch_tc(int bits, int epi, const CUtensorMap &tmap, const TcParams &p, cudaStream_t s)
+{
+    if (epi == EPI_GEMM) {
+        if (bits == 4) return launch_tc<4, true, EPI_GEMM>(tmap, p, s);
+        if (bits == 3) return launch_tc<3, true, EPI_GEMM>(tmap, p, s);
+        if (bits == 2) return launch_tc<2, true, EPI_GEMM>(tmap, p, s);
+        return DSQ_ERR_UNSUPPORTED;
+    }
+    if (bits == 4) return launch_conv<4>(epi, tmap, p, s);
+    if (bits == 2) return launch_conv<2>(epi, tmap, p, s);
     return DSQ_ERR_UNSUPPORTED;
 }
 
@@ -927,7 +1024,7 @@ int dsq_gemm(const void *A_codes, const void *B_codes, int64_t M, int64_t N, int
     CUtensorMap tmap;
     int st = make_rows_tmap(&tmap, B_codes, pitch, (uint64_t)N, pitch, 16 * bits, p.BN);
     if (st) return st;
-    return dispatch_tc(bits, true, tmap, p, (cudaStream_t)stream);
+    return dispatch_tc(bits, EPI_GEMM, tmap, p, (cudaStream_t)stream);
 }
 
 int dsq_conv2d(const void *act_codes, const dsq_nhwc_t *shape, const dsq_quant_t *act_q,
@@ -992,7 +1089,13 @@ int dsq_conv2d(const void *act_codes, const dsq_nhwc_t *shape, const dsq_quant_t
     st = make_rows_tmap(&tmap, w_packed, row_bytes, (uint64_t)conv->Cout, row_bytes, 16 * bits,
                         p.BN);
     if (st) return st;
-    return dispatch_tc(bits, false, tmap, p, (cudaStream_t)stream);
+    // largest |2*acc + S_a| below 2^22: the epilogue may convert integers to
+    // float through the 1.5 * 2^23 bias trick, which is exact there
+    p.small_acc = (double)taps * conv->Cin * (double)((1 << bits) - 1) *
+                          (2.0 * (double)(1 << (bits - 1)) + 1.0) < 4194304.0;
+    const int epi = (y_f32 || acc_out || !y_codes) ? EPI_GENERAL
+                    : (e.residual ? EPI_CODES_RES : EPI_CODES);
+    return dispatch_tc(bits, epi, tmap, p, (cudaStream_t)stream);
 }
 
 int dsq_probe_i8_mma_rate(int iters, float *ms_out, double *macs_out, void *workspace,
