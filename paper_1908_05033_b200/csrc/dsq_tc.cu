@@ -72,6 +72,9 @@ enum { EPI_GEMM = 0, EPI_CODES = 1, EPI_CODES_RES = 2, EPI_GENERAL = 3 };
 struct TcParams {
     // problem
     int M, Ncols, ksteps, BN, m_tiles, n_tiles, n_acc, s_p;
+    // b_res = 1: the whole expanded B tile (all K steps) stays in shared memory
+    // for the life of the CTA (one N tile, few K steps: small weight matrices)
+    int b_res, b_stages;
     // A gather geometry (a GEMM is a 1x1 convolution over an M x 1 image)
     const uint8_t *act;
     int H, W, Ho, Wo, stride, pad, KW, taps, P;
@@ -238,17 +241,18 @@ struct SmemLayout {
 };
 
 constexpr int MAX_S_P = 4;
+constexpr int MAX_B_STAGES = 16;
 
-__host__ __device__ inline SmemLayout smem_layout(int BN, int bits, int s_p)
+__host__ __device__ inline SmemLayout smem_layout(int BN, int bits, int s_p, int b_stages)
 {
     SmemLayout L;
     uint32_t o = 0;
-    L.b_tiles = o;  o += S_U * BN * BK_BYTES;
+    L.b_tiles = o;  o += b_stages * BN * BK_BYTES;
     L.b_packed = o; o += s_p * BN * 16 * bits;
     L.a_ring = o;   o += A_RING * BM * (bits == 3 ? 64 : 16 * bits);
     L.epi = o;      o += NUM_E_WARPS * 64 * 4;       // per-warp scale / bias staging
     o = (o + 127u) & ~127u;
-    L.bars = o;     o += 8 * (2 * S_U + 2 * MAX_S_P + 4);
+    L.bars = o;     o += 8 * (2 * S_U + MAX_B_STAGES + 2 * MAX_S_P + 4);
     L.tmem_slot = o; o += 8;
     L.abort_flag = o; o += 8;
     L.total = o;
@@ -264,29 +268,37 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>(
         (reinterpret_cast<uintptr_t>(smem_raw) + 1023u) & ~(uintptr_t)1023u);
-    const SmemLayout L = smem_layout(p.BN, BITS, p.s_p);
+    const SmemLayout L = smem_layout(p.BN, BITS, p.s_p, p.b_stages);
     const int S_P = p.s_p;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int BN = p.BN;
     const int total_tiles = p.m_tiles * p.n_tiles;
     const uint32_t b_tile_bytes = BN * BK_BYTES;
     const uint32_t b_packed_bytes = BN * 16 * BITS;
+    int my_tiles_all = 0;
+    for (int t = blockIdx.x; t < total_tiles; t += gridDim.x) ++my_tiles_all;
+    // B is produced for every step of every tile, or once (resident mode)
+    const uint32_t n_b_steps =
+        my_tiles_all == 0 ? 0u : (p.b_res ? (uint32_t)p.ksteps : (uint32_t)my_tiles_all * p.ksteps);
 
     const uint32_t bars = smem_u32(smem + L.bars);
-    auto bar_u_full = [&](int s) { return bars + 8u * s; };
+    auto bar_a_full = [&](int s) { return bars + 8u * s; };
     auto bar_u_empty = [&](int s) { return bars + 8u * (S_U + s); };
-    auto bar_p_full = [&](int s) { return bars + 8u * (2 * S_U + s); };
-    auto bar_p_empty = [&](int s) { return bars + 8u * (2 * S_U + MAX_S_P + s); };
-    auto bar_acc_full = [&](int s) { return bars + 8u * (2 * S_U + 2 * MAX_S_P + s); };
-    auto bar_acc_empty = [&](int s) { return bars + 8u * (2 * S_U + 2 * MAX_S_P + 2 + s); };
+    auto bar_b_full = [&](int s) { return bars + 8u * (2 * S_U + s); };
+    constexpr int BAR_P = 2 * S_U + MAX_B_STAGES;
+    auto bar_p_full = [&](int s) { return bars + 8u * (BAR_P + s); };
+    auto bar_p_empty = [&](int s) { return bars + 8u * (BAR_P + MAX_S_P + s); };
+    auto bar_acc_full = [&](int s) { return bars + 8u * (BAR_P + 2 * MAX_S_P + s); };
+    auto bar_acc_empty = [&](int s) { return bars + 8u * (BAR_P + 2 * MAX_S_P + 2 + s); };
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + L.tmem_slot);
     Ctl ctl{reinterpret_cast<volatile int *>(smem + L.abort_flag), p.ws};
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S_U; ++s) {
-            mbar_init(bar_u_full(s), NUM_A_WARPS + NUM_B_WARPS);
+            mbar_init(bar_a_full(s), NUM_A_WARPS);
             mbar_init(bar_u_empty(s), 1);    // tcgen05.commit
         }
+        for (int s = 0; s < MAX_B_STAGES; ++s) mbar_init(bar_b_full(s), NUM_B_WARPS);
         for (int s = 0; s < S_P; ++s) {
             mbar_init(bar_p_full(s), 1);     // TMA producer (+ transaction bytes)
             mbar_init(bar_p_empty(s), NUM_B_WARPS);
@@ -312,19 +324,15 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
         // ---------------- B producer: TMA packed tiles --------------------
         if (lane == 0) {
             uint32_t g = 0, ph = 0;
-            int s = 0;
-            bool ok = true;
+            int s = 0, ks = 0, tile = blockIdx.x;
 #pragma unroll 1
-            for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
-                const int n_tile = tile % p.n_tiles;
-#pragma unroll 1
-                for (int ks = 0; ks < p.ksteps; ++ks, ++g) {
-                    if (!(ok = wait_bar(bar_p_empty(s), ph ^ 1u, ctl, 1))) break;
-                    mbar_arrive_expect_tx(bar_p_full(s), b_packed_bytes);
-                    tma_load_2d(smem_u32(smem + L.b_packed + s * b_packed_bytes), &tmap_b,
-                                ks * 16 * BITS, n_tile * BN, bar_p_full(s));
-                    if (++s == S_P) { s = 0; ph ^= 1u; }
-                }
+            for (; g < n_b_steps; ++g) {
+                if (!wait_bar(bar_p_empty(s), ph ^ 1u, ctl, 1)) break;
+                mbar_arrive_expect_tx(bar_p_full(s), b_packed_bytes);
+                tma_load_2d(smem_u32(smem + L.b_packed + s * b_packed_bytes), &tmap_b,
+                            ks * 16 * BITS, (tile % p.n_tiles) * BN, bar_p_full(s));
+                if (++s == S_P) { s = 0; ph ^= 1u; }
+                if (++ks == p.ksteps) { ks = 0; tile += gridDim.x; }
             }
             // let outstanding copies land before the CTA can exit
             const uint32_t issued = g;
@@ -348,11 +356,14 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
                 for (int ks = 0; ks < p.ksteps; ++ks, ++g) {
                     const int s = g % S_U;
                     const uint32_t ph = (g / S_U) & 1u;
-                    if (!(ok = wait_bar(bar_u_full(s), ph, ctl, 4))) break;
+                    const int bs = p.b_res ? ks : s;
+                    if (!p.b_res || it == 0)
+                        if (!(ok = wait_bar(bar_b_full(bs), p.b_res ? 0u : ph, ctl, 10))) break;
+                    if (!(ok = wait_bar(bar_a_full(s), ph, ctl, 4))) break;
                     tc_fence_after_sync();
                     const uint32_t a_tmem = tmem_base + A_COL0 + s * 32;
                     const uint64_t bd =
-                        smem_desc_sw128(smem_u32(smem + L.b_tiles + s * b_tile_bytes));
+                        smem_desc_sw128(smem_u32(smem + L.b_tiles + bs * b_tile_bytes));
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk)   // 32 bytes of K per instruction
                         mma_i8_ts(d_tmem, a_tmem + 8 * kk, bd + 2 * kk, idesc,
@@ -456,7 +467,7 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
             tmem_st_wait();
             tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar_u_full(pend_s));
+            if (lane == 0) mbar_arrive(bar_a_full(pend_s));
             pend_s = -1;
         };
         // one loop, one issue site: iteration i issues step i and consumes step
@@ -498,15 +509,14 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
         const int j = (BITS == 3) ? 0 : tid % CH;
         const int sw = row0 & 7;
         const int n_it = (BN + ROWS_PER_IT - 1) / ROWS_PER_IT;
-        uint32_t g = 0, php = 0;
+        uint32_t php = 0;
         int sp = -1;
         bool ok = true;
+        {
 #pragma unroll 1
-        for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
-#pragma unroll 1
-            for (int ks = 0; ks < p.ksteps; ++ks, ++g) {
+            for (uint32_t g = 0; g < n_b_steps; ++g) {
                 if (++sp == S_P) { sp = 0; php ^= 1u; }
-                const int su = g % S_U;
+                const int su = p.b_res ? (int)g : (int)(g % S_U);
                 const uint32_t phu = (g / S_U) & 1u;
                 if (!(ok = wait_bar(bar_p_full(sp), php, ctl, 6))) break;
                 const uint8_t *src = smem + L.b_packed + sp * b_packed_bytes;
@@ -522,7 +532,7 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
                             w[4 * l + 2] = v.z; w[4 * l + 3] = v.w;
                         }
                     }
-                    if (!(ok = wait_bar(bar_u_empty(su), phu ^ 1u, ctl, 7))) break;
+                    if (!p.b_res && !(ok = wait_bar(bar_u_empty(su), phu ^ 1u, ctl, 7))) break;
                     if (row0 < BN) {
                         uint8_t *rowp = dst + row0 * BK_BYTES;
 #pragma unroll
@@ -537,7 +547,7 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
                     for (int i = 0; i < MAX_IT; ++i)
                         if (i < n_it && row0 + i * ROWS_PER_IT < BN)
                             v[i] = reinterpret_cast<const uint4 *>(src)[tid + i * NUM_B_THREADS];
-                    if (!(ok = wait_bar(bar_u_empty(su), phu ^ 1u, ctl, 7))) break;
+                    if (!p.b_res && !(ok = wait_bar(bar_u_empty(su), phu ^ 1u, ctl, 7))) break;
                     uint8_t *rowp = dst + row0 * BK_BYTES;
 #pragma unroll
                     for (int i = 0; i < MAX_IT; ++i) {
@@ -558,7 +568,7 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
                 fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0) {
-                    mbar_arrive(bar_u_full(su));
+                    mbar_arrive(bar_b_full(su));
                     mbar_arrive(bar_p_empty(sp));
                 }
             }
@@ -909,6 +919,22 @@ int make_rows_tmap(CUtensorMap *map, const void *base, uint64_t row_bytes, uint6
     return r == CUDA_SUCCESS ? DSQ_OK : DSQ_ERR_CUDA;
 }
 
+// Resident B: one N tile and few K steps, so the expanded B tile of every K
+// step fits in shared memory next to the rings; it is then expanded once per
+// CTA instead of once per M tile.
+void choose_b_mode(TcParams *p, int bits)
+{
+    p->b_res = 0;
+    p->b_stages = S_U;
+    if (p->n_tiles == 1 && p->ksteps <= MAX_B_STAGES && p->m_tiles > 148) {
+        const SmemLayout L = smem_layout(p->BN, bits, p->s_p, p->ksteps);
+        if (L.total + 1024 <= 227u * 1024u) {
+            p->b_res = 1;
+            p->b_stages = p->ksteps;
+        }
+    }
+}
+
 int g_forced_bn = 0;   // dsq_set_tile_n
 
 int pick_bn(int m_tiles, int ncols, int bits)
@@ -932,7 +958,7 @@ int pick_bn(int m_tiles, int ncols, int bits)
 template <int BITS, bool A_SIGNED, int EPI>
 int launch_tc(const CUtensorMap &tmap, const TcParams &p, cudaStream_t s)
 {
-    const SmemLayout L = smem_layout(p.BN, BITS, p.s_p);
+    const SmemLayout L = smem_layout(p.BN, BITS, p.s_p, p.b_stages);
     const int smem_bytes = (int)L.total + 1024;
     static bool configured = false;
     if (!configured) {
@@ -1011,6 +1037,7 @@ int dsq_gemm(const void *A_codes, const void *B_codes, int64_t M, int64_t N, int
     p.n_tiles = (int)((N + p.BN - 1) / p.BN);
     p.n_acc = 2 * p.BN <= A_COL0 ? 2 : 1;
     p.s_p = p.BN > 192 ? 3 : 4;
+    choose_b_mode(&p, bits);
     p.act = (const uint8_t *)A_codes;
     p.H = 1; p.W = (int)M; p.Ho = 1; p.Wo = (int)M;
     p.stride = 1; p.pad = 0; p.KW = 1; p.taps = 1; p.P = (int)pitch;
@@ -1071,6 +1098,7 @@ int dsq_conv2d(const void *act_codes, const dsq_nhwc_t *shape, const dsq_quant_t
     p.n_tiles = (conv->Cout + p.BN - 1) / p.BN;
     p.n_acc = 2 * p.BN <= A_COL0 ? 2 : 1;
     p.s_p = p.BN > 192 ? 3 : 4;
+    choose_b_mode(&p, bits);
     p.act = (const uint8_t *)act_codes;
     p.H = shape->H; p.W = shape->W; p.Ho = Ho; p.Wo = Wo;
     p.stride = conv->stride; p.pad = conv->pad; p.KW = conv->KW; p.taps = taps; p.P = (int)P;
