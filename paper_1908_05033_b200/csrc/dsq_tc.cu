@@ -57,10 +57,10 @@ constexpr int A_RING = A_D + 1;       // packed A ring slots
 constexpr int TMEM_COLS = 512;
 constexpr int A_COL0 = TMEM_COLS - S_U * 32;  // A stages live in the top columns
 
-constexpr int WARP_TMA = 0, WARP_MMA = 1, WARP_A0 = 2, WARP_B0 = 10, WARP_E0 = 18;
-constexpr int NUM_A_WARPS = 8, NUM_B_WARPS = 8, NUM_E_WARPS = 4;
+constexpr int WARP_TMA = 0, WARP_MMA = 1, WARP_B0 = 6, WARP_E0 = 14;   // A warps: 2..5
+constexpr int NUM_A_WARPS = 4, NUM_B_WARPS = 8, NUM_E_WARPS = 4;
 constexpr int NUM_B_THREADS = NUM_B_WARPS * 32;
-constexpr int NUM_WARPS = 22;
+constexpr int NUM_WARPS = 18;
 constexpr int NUM_THREADS = NUM_WARPS * 32;
 constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;   // a wait gives up after 2 s
 
@@ -192,47 +192,6 @@ __device__ __forceinline__ void expand_row_regs(const uint4 (&v)[Chunks<BITS>::C
     }
 }
 
-// half a row step in registers (what one A thread handles): 16 int8 words.
-// 4-bit: 2 packed chunks; 2-bit: 1 chunk; 3-bit: the 6 packed words
-// w[first..first+5] out of the 8 words held in v[0..1].
-template <int BITS, bool SIGNED>
-__device__ __forceinline__ void expand_half_regs(const uint4 (&v)[2], int half, uint32_t orv,
-                                                 uint32_t (&o)[16])
-{
-    if (BITS == 3) {
-        // half 0 loaded bytes 0..31 of the 48-byte step and owns words 0..5;
-        // half 1 loaded bytes 16..47 and owns words 6..11 = its words 2..7
-        const uint32_t l[8] = {v[0].x, v[0].y, v[0].z, v[0].w, v[1].x, v[1].y, v[1].z, v[1].w};
-        uint32_t w[7];
-#pragma unroll
-        for (int i = 0; i < 6; ++i) w[i] = half ? l[i + 2] : l[i];
-        w[6] = 0u;
-#pragma unroll
-        for (int t = 0; t < 16; ++t) {
-            const int bit = 12 * t;
-            const int wi = bit >> 5, sh = bit & 31;
-            const uint32_t x = __funnelshift_r(w[wi], w[wi + 1], sh);
-            uint32_t b = (x & 7u) | ((x & 0x38u) << 5) | ((x & 0x1C0u) << 10) |
-                         ((x & 0xE00u) << 15);
-            if (SIGNED) b = (b << 5) | orv;
-            o[t] = b;
-        }
-    } else {
-        constexpr int OUT = Chunks<BITS>::OUT;
-        constexpr int NCH = (BITS == 4) ? 2 : 1;
-#pragma unroll
-        for (int j = 0; j < NCH; ++j)
-#pragma unroll
-            for (int c = 0; c < OUT; ++c) {
-                const int b = (j * OUT + c) * 4;
-                o[b] = expand_word<BITS, SIGNED>(v[j].x, c, orv);
-                o[b + 1] = expand_word<BITS, SIGNED>(v[j].y, c, orv);
-                o[b + 2] = expand_word<BITS, SIGNED>(v[j].z, c, orv);
-                o[b + 3] = expand_word<BITS, SIGNED>(v[j].w, c, orv);
-            }
-    }
-}
-
 // ---------------------------------------------------------------------------
 // the kernel
 // ---------------------------------------------------------------------------
@@ -249,7 +208,7 @@ __host__ __device__ inline SmemLayout smem_layout(int BN, int bits, int s_p, int
     uint32_t o = 0;
     L.b_tiles = o;  o += b_stages * BN * BK_BYTES;
     L.b_packed = o; o += s_p * BN * 16 * bits;
-    L.a_ring = o;   o += A_RING * BM * (bits == 3 ? 64 : 16 * bits);
+    L.a_ring = o;   o += A_RING * BM * 16 * bits;
     L.epi = o;      o += NUM_E_WARPS * 64 * 4;       // per-warp scale / bias staging
     o = (o + 127u) & ~127u;
     L.bars = o;     o += 8 * (2 * S_U + MAX_B_STAGES + 2 * MAX_S_P + 4);
@@ -374,37 +333,23 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
             }
         }
     } else if (warp < WARP_B0) {
-        // ---------------- A: two threads per tile row ------------------------
-        // Each thread owns half of its row's 128-code step (16 int8 words):
+        // ---------------- A: one thread per tile row ------------------------
         // global --cp.async--> private 16-byte cells of a shared ring (A_D steps
-        // in flight, thread-local completion) -> registers -> expand ->
-        // tensor memory (tcgen05.st).  The store of step g is completed (and
-        // the stage published) only after step g+1 has been expanded, so the
-        // store latency overlaps the next step's arithmetic.
-        const int aw = warp - WARP_A0;
+        // in flight, thread-local completion) -> registers -> expand -> tensor
+        // memory (tcgen05.st).  The store of step g is completed (and the stage
+        // published) only after step g+1 has been expanded, so the store latency
+        // overlaps the next step's arithmetic.
         const int quarter = warp & 3;              // TMEM lane quarter of this warp
-        const int half = aw >> 2;                  // which 16 columns of the step
         const int row = quarter * 32 + lane;
-        constexpr int NLD = (BITS == 2) ? 1 : 2;   // 16-byte loads per thread per step
-        constexpr int PLANES = 2 * NLD;            // ring slot = PLANES x 128 rows x 16 B
-        constexpr int SLOT_BYTES = PLANES * BM * 16;
-        const uint32_t cell0 = smem_u32(smem + L.a_ring) + ((half * NLD) * BM + row) * 16;
-        // issue position (runs A_D steps ahead of the consume position)
-        // (starts one tile back with ld_ks at its end: the first issue advances)
+        constexpr int SLOT_BYTES = CH * BM * 16;   // ring slot = CH planes x 128 rows x 16 B
+        const uint32_t cell0 = smem_u32(smem + L.a_ring) + row * 16;
+        // issue position (runs A_D steps ahead of the consume position; starts
+        // one tile back with ld_ks at its end, so that the first issue advances)
         int ld_tile = (int)blockIdx.x - (int)gridDim.x, ld_ks = p.ksteps, ld_slot = 0;
         int tap = 0, kw = 0, off = 0;
         uint32_t tap_mask = 0;                     // bit t: filter tap t is inside the image
         const uint8_t *src = p.act;
         const int64_t row_jump = (int64_t)(p.W - p.KW) * p.P;
-        auto advance16 = [&]() {
-            off += 16;
-            src += 16;
-            if (off == p.P) {
-                off = 0;
-                ++tap;
-                if (++kw == p.KW) { kw = 0; src += row_jump; }
-            }
-        };
         auto set_tile = [&](int t) {
             tap = kw = off = 0;
             tap_mask = 0;
@@ -422,12 +367,6 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
                 }
                 src = p.act + (((int64_t)n * p.H + hb) * p.W + wb) * p.P;
             }
-            if (BITS == 3) {
-                src += 16 * half;                  // bytes 0..31 or 16..47 of each step
-                off = 16 * half;
-            } else {
-                for (int i = 0; i < half * NLD; ++i) advance16();
-            }
         };
         auto issue_step = [&]() {
             if (ld_ks == p.ksteps) {
@@ -438,29 +377,23 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
             if (ld_tile < total_tiles) {
                 const uint32_t dst = cell0 + ld_slot * SLOT_BYTES;
 #pragma unroll
-                for (int j = 0; j < NLD; ++j) {
-                    bool ok;
-                    if (BITS == 3) ok = (tap_mask & 1u) && off + 16 * j < p.P;
-                    else ok = (tap_mask >> tap) & 1u;
-                    cp_async_16(dst + j * (BM * 16), ok ? src + (BITS == 3 ? 16 * j : 0) : p.act,
-                                ok ? 16u : 0u);
-                    if (BITS != 3) advance16();
-                }
-                if (BITS == 3) {
-                    src += 48;
-                    off += 48;
-                } else {
-#pragma unroll
-                    for (int j = 0; j < NLD; ++j) advance16();   // the other half's chunks
+                for (int j = 0; j < CH; ++j) {
+                    const bool ok = (tap_mask >> tap) & 1u;
+                    cp_async_16(dst + j * (BM * 16), ok ? src : p.act, ok ? 16u : 0u);
+                    off += 16;
+                    src += 16;
+                    if (off == p.P) {
+                        off = 0;
+                        ++tap;
+                        if (++kw == p.KW) { kw = 0; src += row_jump; }
+                    }
                 }
                 if (++ld_slot == A_RING) ld_slot = 0;
                 ++ld_ks;
             }
             cp_async_commit();            // one group per step, empty at the tail
         };
-        int my_tiles = 0;
-        for (int t = blockIdx.x; t < total_tiles; t += gridDim.x) ++my_tiles;
-        const uint32_t n_steps = (uint32_t)my_tiles * p.ksteps;
+        const uint32_t n_steps = (uint32_t)my_tiles_all * p.ksteps;
         int rd_slot = 0, pend_s = -1;
         bool ok = true;
         auto publish = [&]() {
@@ -478,22 +411,20 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
             if (i < (uint32_t)A_D) continue;
             const uint32_t g = i - A_D;
             cp_async_wait<A_D>();         // the group of step g has landed
-            uint4 cur[2];
-            cur[1] = make_uint4(0u, 0u, 0u, 0u);
+            uint4 cur[CH];
 #pragma unroll
-            for (int j = 0; j < NLD; ++j)
+            for (int j = 0; j < CH; ++j)
                 cur[j] = lds_128(cell0 + rd_slot * SLOT_BYTES + j * (BM * 16));
             if (++rd_slot == A_RING) rd_slot = 0;
-            uint32_t o[16];
-            expand_half_regs<BITS, A_SIGNED>(cur, half, p.orv, o);
+            uint32_t o[32];
+            expand_row_regs<BITS, A_SIGNED>(cur, p.orv, o);
             if (pend_s >= 0) publish();
             const int s = g % S_U;
             const uint32_t ph = (g / S_U) & 1u;
             if (!(ok = wait_bar(bar_u_empty(s), ph ^ 1u, ctl, 5))) break;
             tc_fence_after_sync();
             __syncwarp();
-            tmem_st_32x16(tmem_base + ((uint32_t)(quarter * 32) << 16) + A_COL0 + s * 32 +
-                              16 * half, o);
+            tmem_st_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + A_COL0 + s * 32, o);
             pend_s = s;
         }
         if (ok && pend_s >= 0) publish();
