@@ -355,13 +355,21 @@ def run_ours(args):
     quant_ms = sum(t for k, _, t in kt if k == "dsq_quantize_act")
     n_conv = sum(1 for k, _, _ in kt if k == "dsq_conv2d")
     int8_peak = 2.0 * peaks["bf16_sustained"]       # int8 : bf16 nominal ratio 2
-    achieved = 2.0 * macs_step / (conv_ms * 1e-3) / 1e12
+    # dominant kernel: the 19 tensor-core convolutions.  Its time inside the
+    # timed region is the graph step time minus the quantise kernel's (CUDA
+    # events cannot sit between the nodes of a replayed graph; the eager
+    # per-launch times are reported in extras).
+    step_ms = ms / args.steps
+    conv_in_step_ms = max(step_ms - quant_ms, 1e-6)
+    achieved = 2.0 * macs_step / (conv_in_step_ms * 1e-3) / 1e12
     roofline = {
         "kernel": "dsq_tc_kernel (dsq_conv2d), 19 launches per step",
         "bound": "tensor", "achieved": achieved, "peak": int8_peak, "unit": "TOP/s",
         "frac": achieved / int8_peak,
-        "peak_source": f"2 x bf16_tflops_sustained of {peaks['source']} peaks",
-        "avg_launch_ms": conv_ms / n_conv,
+        "peak_source": f"2 x bf16_tflops_sustained of {peaks['source']} peaks "
+                       "(int8:bf16 nominal ratio); nominal 4500, own MMA-only probe in extras",
+        "avg_launch_ms": conv_in_step_ms / n_conv,
+        "how": "graph step time minus the quantise kernel's eager event time, over 19 launches",
         "traffic": None,
     }
 
