@@ -48,6 +48,17 @@ __device__ __forceinline__ void transpose8x8_u16(uint32_t (&r)[4], int s)
     }
 }
 
+// Streaming 128-bit load: read-only path, no L1 allocation (every byte is used
+// once), 256-byte L2 prefetch granularity.
+__device__ __forceinline__ float4 ld_stream_f4(const float4 *p)
+{
+    float4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.L2::256B.v4.f32 {%0, %1, %2, %3}, [%4];"
+                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+                 : "l"(p));
+    return v;
+}
+
 template <int BITS>
 __device__ __forceinline__ uint32_t quantize4(const float4 v, const DsqQ &q)
 {
@@ -88,7 +99,7 @@ quantize_flat_kernel(const float4 *__restrict__ x, uint4 *__restrict__ out,
             for (int f = 0; f < NF; ++f) {
                 v[j][f] = make_float4(0.f, 0.f, 0.f, 0.f);
                 if (line < n_lines)
-                    v[j][f] = __ldcs(x + line * F4_PER_LINE + 8 * f + s);
+                    v[j][f] = ld_stream_f4(x + line * F4_PER_LINE + 8 * f + s);
             }
         }
         uint32_t h[8];
@@ -352,7 +363,9 @@ int dsq_quantize_act(const float *x, const dsq_nhwc_t *shape,
     const bool flat = (bits == 4 || bits == 2) && ((size_t)k * bits == pitch * 8);
     if (flat) {
         const int64_t n_lines = rows * (int64_t)(pitch / 16);
-        const int grid = grid_for((n_lines + 31) / 32 * 32, 256);
+        // many more CTAs than SMs: at 8-16 loads per thread the memory system
+        // needs the extra resident warps to stay full
+        const int grid = grid_for((n_lines + 31) / 32 * 32, 256, 148 * 64);
         if (bits == 4)
             quantize_flat_kernel<4><<<grid, 256, 0, s>>>(
                 (const float4 *)x, (uint4 *)codes_out, n_lines, dq);
