@@ -52,15 +52,19 @@ namespace {
 constexpr int BM = 128;               // tile rows = MMA M
 constexpr int BK_BYTES = 128;         // int8 bytes per row per K step (128 codes)
 constexpr int S_U = 4;                // stages of expanded operands (A in TMEM, B in smem)
-constexpr int A_D = 5;                // A row steps in flight per thread (cp.async groups)
+constexpr int A_D = 2;                // own A steps in flight per thread (cp.async groups)
 constexpr int A_RING = A_D + 1;       // packed A ring slots
 constexpr int TMEM_COLS = 512;
 constexpr int A_COL0 = TMEM_COLS - S_U * 32;  // A stages live in the top columns
 
-constexpr int WARP_TMA = 0, WARP_MMA = 1, WARP_B0 = 6, WARP_E0 = 14;   // A warps: 2..5
-constexpr int NUM_A_WARPS = 4, NUM_B_WARPS = 8, NUM_E_WARPS = 4;
+constexpr int WARP_TMA = 0, WARP_MMA = 1, WARP_A0 = 2, WARP_B0 = 10, WARP_E0 = 18;
+// two groups of four A warps take alternate K steps
+constexpr int NUM_A_GROUPS = 2, NUM_A_WARPS = 4 * NUM_A_GROUPS, NUM_B_WARPS = 8, NUM_E_WARPS = 4;
 constexpr int NUM_B_THREADS = NUM_B_WARPS * 32;
-constexpr int NUM_WARPS = 18;
+constexpr int NUM_WARPS = 22;
+static_assert(WARP_A0 + NUM_A_WARPS == WARP_B0 && WARP_B0 + NUM_B_WARPS == WARP_E0 &&
+                  WARP_E0 + NUM_E_WARPS == NUM_WARPS,
+              "warp roles");
 constexpr int NUM_THREADS = NUM_WARPS * 32;
 constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;   // a wait gives up after 2 s
 
@@ -208,7 +212,7 @@ __host__ __device__ inline SmemLayout smem_layout(int BN, int bits, int s_p, int
     uint32_t o = 0;
     L.b_tiles = o;  o += b_stages * BN * BK_BYTES;
     L.b_packed = o; o += s_p * BN * 16 * bits;
-    L.a_ring = o;   o += A_RING * BM * 16 * bits;
+    L.a_ring = o;   o += NUM_A_GROUPS * A_RING * BM * 16 * bits;
     L.epi = o;      o += NUM_E_WARPS * 64 * 4;       // per-warp scale / bias staging
     o = (o + 127u) & ~127u;
     L.bars = o;     o += 8 * (2 * S_U + MAX_B_STAGES + 2 * MAX_S_P + 4);
@@ -254,7 +258,7 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S_U; ++s) {
-            mbar_init(bar_a_full(s), NUM_A_WARPS);
+            mbar_init(bar_a_full(s), 4);     // the four warps of one A group
             mbar_init(bar_u_empty(s), 1);    // tcgen05.commit
         }
         for (int s = 0; s < MAX_B_STAGES; ++s) mbar_init(bar_b_full(s), NUM_B_WARPS);
@@ -333,18 +337,22 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
             }
         }
     } else if (warp < WARP_B0) {
-        // ---------------- A: one thread per tile row ------------------------
-        // global --cp.async--> private 16-byte cells of a shared ring (A_D steps
-        // in flight, thread-local completion) -> registers -> expand -> tensor
-        // memory (tcgen05.st).  The store of step g is completed (and the stage
-        // published) only after step g+1 has been expanded, so the store latency
-        // overlaps the next step's arithmetic.
+        // ---------------- A: one thread per tile row, two groups ---------------
+        // Group k (four warps, one per TMEM lane quarter) handles the K steps with
+        // step index = k (mod 2), so two steps are in flight at once and the
+        // per-step latency chain of one group overlaps the other's.  Per step:
+        // global --cp.async--> private 16-byte cells of a shared ring (A_D own
+        // steps in flight, thread-local completion) -> registers -> expand ->
+        // tensor memory (tcgen05.st).  The store of a step is completed (and the
+        // stage published) only after the group's next step has been expanded.
+        const int group = (warp - WARP_A0) >> 2;
         const int quarter = warp & 3;              // TMEM lane quarter of this warp
         const int row = quarter * 32 + lane;
         constexpr int SLOT_BYTES = CH * BM * 16;   // ring slot = CH planes x 128 rows x 16 B
-        const uint32_t cell0 = smem_u32(smem + L.a_ring) + row * 16;
-        // issue position (runs A_D steps ahead of the consume position; starts
-        // one tile back with ld_ks at its end, so that the first issue advances)
+        const uint32_t cell0 =
+            smem_u32(smem + L.a_ring) + group * (A_RING * SLOT_BYTES) + row * 16;
+        // walk position over the flattened (tile, K step) sequence; starts one
+        // tile back with ld_ks at its end, so that the first step advances
         int ld_tile = (int)blockIdx.x - (int)gridDim.x, ld_ks = p.ksteps, ld_slot = 0;
         int tap = 0, kw = 0, off = 0;
         uint32_t tap_mask = 0;                     // bit t: filter tap t is inside the image
@@ -368,7 +376,8 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
                 src = p.act + (((int64_t)n * p.H + hb) * p.W + wb) * p.P;
             }
         };
-        auto issue_step = [&]() {
+        // one K step of the walk: with `load`, its CH chunks go to the ring
+        auto walk_step = [&](bool load) {
             if (ld_ks == p.ksteps) {
                 ld_ks = 0;
                 ld_tile += gridDim.x;
@@ -378,8 +387,10 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
                 const uint32_t dst = cell0 + ld_slot * SLOT_BYTES;
 #pragma unroll
                 for (int j = 0; j < CH; ++j) {
-                    const bool ok = (tap_mask >> tap) & 1u;
-                    cp_async_16(dst + j * (BM * 16), ok ? src : p.act, ok ? 16u : 0u);
+                    if (load) {
+                        const bool ok = (tap_mask >> tap) & 1u;
+                        cp_async_16(dst + j * (BM * 16), ok ? src : p.act, ok ? 16u : 0u);
+                    }
                     off += 16;
                     src += 16;
                     if (off == p.P) {
@@ -388,12 +399,13 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
                         if (++kw == p.KW) { kw = 0; src += row_jump; }
                     }
                 }
-                if (++ld_slot == A_RING) ld_slot = 0;
                 ++ld_ks;
+                if (load && ++ld_slot == A_RING) ld_slot = 0;
             }
-            cp_async_commit();            // one group per step, empty at the tail
         };
         const uint32_t n_steps = (uint32_t)my_tiles_all * p.ksteps;
+        // own steps: g = group, group + 2, ...
+        const uint32_t n_own = n_steps > (uint32_t)group ? (n_steps - group + 1) / 2 : 0u;
         int rd_slot = 0, pend_s = -1;
         bool ok = true;
         auto publish = [&]() {
@@ -403,21 +415,25 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
             if (lane == 0) mbar_arrive(bar_a_full(pend_s));
             pend_s = -1;
         };
-        // one loop, one issue site: iteration i issues step i and consumes step
-        // i - A_D (the first A_D iterations only fill the ring)
+        if (group == 1) walk_step(false);          // step 0 belongs to group 0
+        // iteration i issues own step i and consumes own step i - A_D
 #pragma unroll 1
-        for (uint32_t i = 0; ok && i < n_steps + A_D; ++i) {
-            issue_step();
+        for (uint32_t i = 0; ok && i < n_own + A_D; ++i) {
+            walk_step(true);                       // own step (no-op past the end)
+            cp_async_commit();                     // one group per own step
+            walk_step(false);                      // the other group's step
             if (i < (uint32_t)A_D) continue;
-            const uint32_t g = i - A_D;
-            cp_async_wait<A_D>();         // the group of step g has landed
-            uint4 cur[CH];
-#pragma unroll
-            for (int j = 0; j < CH; ++j)
-                cur[j] = lds_128(cell0 + rd_slot * SLOT_BYTES + j * (BM * 16));
-            if (++rd_slot == A_RING) rd_slot = 0;
+            const uint32_t g = 2 * (i - A_D) + group;
+            cp_async_wait<A_D>();                  // own step i - A_D has landed
             uint32_t o[32];
-            expand_row_regs<BITS, A_SIGNED>(cur, p.orv, o);
+            {
+                uint4 cur[CH];
+#pragma unroll
+                for (int j = 0; j < CH; ++j)
+                    cur[j] = lds_128(cell0 + rd_slot * SLOT_BYTES + j * (BM * 16));
+                expand_row_regs<BITS, A_SIGNED>(cur, p.orv, o);
+            }
+            if (++rd_slot == A_RING) rd_slot = 0;
             if (pend_s >= 0) publish();
             const int s = g % S_U;
             const uint32_t ph = (g / S_U) & 1u;
