@@ -306,6 +306,8 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
         // ---------------- MMA issuer ---------------------------------------
         if (lane == 0) {
             const uint32_t idesc = idesc_i8(BN, A_SIGNED, B_SIGNED);
+            const uint64_t b_desc0 = smem_desc_sw128(smem_u32(smem + L.b_tiles));
+            const uint32_t b_desc_lo0 = (uint32_t)b_desc0, b_desc_hi = (uint32_t)(b_desc0 >> 32);
             uint32_t g = 0, it = 0;
             bool ok = true;
 #pragma unroll 1
@@ -324,13 +326,10 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
                         if (!(ok = wait_bar(bar_b_full(bs), p.b_res ? 0u : ph, ctl, 10))) break;
                     if (!(ok = wait_bar(bar_a_full(s), ph, ctl, 4))) break;
                     tc_fence_after_sync();
-                    const uint32_t a_tmem = tmem_base + A_COL0 + s * 32;
-                    const uint64_t bd =
-                        smem_desc_sw128(smem_u32(smem + L.b_tiles + bs * b_tile_bytes));
-#pragma unroll
-                    for (int kk = 0; kk < 4; ++kk)   // 32 bytes of K per instruction
-                        mma_i8_ts(d_tmem, a_tmem + 8 * kk, bd + 2 * kk, idesc,
-                                  (ks | kk) != 0 ? 1u : 0u);
+                    // 4 instructions, 32 bytes of K each
+                    mma_i8_ts_x4(d_tmem, tmem_base + A_COL0 + s * 32,
+                                 b_desc_lo0 + bs * (b_tile_bytes >> 4), b_desc_hi, idesc,
+                                 (uint32_t)ks);
                     mma_commit(bar_u_empty(s));
                 }
                 if (ok) mma_commit(bar_acc_full(as));
