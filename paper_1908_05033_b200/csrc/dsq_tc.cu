@@ -342,8 +342,7 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
         // per-step latency chain of one group overlaps the other's.  Per step:
         // global --cp.async--> private 16-byte cells of a shared ring (A_D own
         // steps in flight, thread-local completion) -> registers -> expand ->
-        // tensor memory (tcgen05.st).  The store of a step is completed (and the
-        // stage published) only after the group's next step has been expanded.
+        // tensor memory (tcgen05.st), completed and published at once.
         const int group = (warp - WARP_A0) >> 2;
         const int quarter = warp & 3;              // TMEM lane quarter of this warp
         const int row = quarter * 32 + lane;
@@ -433,7 +432,6 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
                 expand_row_regs<BITS, A_SIGNED>(cur, p.orv, o);
             }
             if (++rd_slot == A_RING) rd_slot = 0;
-            if (pend_s >= 0) publish();
             const int s = g % S_U;
             const uint32_t ph = (g / S_U) & 1u;
             if (!(ok = wait_bar(bar_u_empty(s), ph ^ 1u, ctl, 5))) break;
@@ -441,8 +439,8 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
             __syncwarp();
             tmem_st_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + A_COL0 + s * 32, o);
             pend_s = s;
+            publish();                             // the other group's step overlaps this
         }
-        if (ok && pend_s >= 0) publish();
         cp_async_wait<0>();
     } else if (warp < WARP_E0) {
         // ---------------- B: expand packed shared tiles ---------------------
