@@ -266,6 +266,11 @@ int dsq_probe_i8_mma_rate(int iters, float *ms_out, double *macs_out,
  * do not depend on it. */
 int dsq_set_tile_n(int bn);
 
+/* Second tuning hook: K steps (of 128 codes) per pipeline round of the
+ * tensor-core kernels, 1 or 2; 0 restores the automatic choice (2 whenever
+ * the N tile is at most 128 wide).  Results do not depend on it. */
+int dsq_set_round_k_steps(int ks);
+
 /* ---- misc --------------------------------------------------------------- */
 const char *dsq_status_string(int status);
 int dsq_version(void);

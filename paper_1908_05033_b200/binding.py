@@ -75,6 +75,7 @@ _SIGNATURES = {
     "dsq_probe_i8_mma_rate": (_int, [_int, C.POINTER(C.c_float),
                                      C.POINTER(C.c_double), _vp, _sz, _vp]),
     "dsq_set_tile_n": (_int, [_int]),
+    "dsq_set_round_k_steps": (_int, [_int]),
     "dsq_status_string": (C.c_char_p, [_int]),
     "dsq_version": (_int, []),
 }
@@ -315,6 +316,10 @@ def dsq_gemm(A, B, M, N, K, bits, ws, row_scale=None, want_i32=True,
     _check(lib.dsq_gemm(_p(A), _p(B), M, N, K, bits, _p(Cm), _p(row_scale),
                         _p(D), _p(ws), ws.numel(), _stream()), "dsq_gemm")
     return Cm, D
+
+
+def dsq_set_round_k_steps(ks):
+    _check(lib.dsq_set_round_k_steps(ks), "dsq_set_round_k_steps")
 
 
 def dsq_set_tile_n(bn):

@@ -53,6 +53,7 @@ def main(argv=None):
     ap.add_argument("--no-flush", action="store_true")
     ap.add_argument("--f32-out", action="store_true")
     ap.add_argument("--tile-n", type=int, default=0)
+    ap.add_argument("--round-k", type=int, default=0)
     a = ap.parse_args(argv)
     dev = "cuda"
     ws = B.new_workspace(dev)
@@ -61,6 +62,7 @@ def main(argv=None):
     gen.manual_seed(1908)
     bits = a.bits
     B.dsq_set_tile_n(a.tile_n)
+    B.dsq_set_round_k_steps(a.round_k)
     out = {"case": a.case, "bits": bits, "tile_n": a.tile_n}
     if a.case == "gemm":
         n = a.size

@@ -51,11 +51,17 @@ namespace {
 
 constexpr int BM = 128;               // tile rows = MMA M
 constexpr int BK_BYTES = 128;         // int8 bytes per row per K step (128 codes)
-constexpr int S_U = 4;                // stages of expanded operands (A in TMEM, B in smem)
-constexpr int A_D = 2;                // own A steps in flight per thread (cp.async groups)
-constexpr int A_RING = A_D + 1;       // packed A ring slots
+// A barrier round covers KS K steps of 128 codes (KS = 1 or 2, template
+// parameter): with small N tiles the fixed cost of a round (barrier hand-offs,
+// MMA issue) outweighs its work, so two K steps share one round.
+constexpr int SU_MAX = 4;
+template <int KS> struct Pipe {
+    static constexpr int SU = KS == 1 ? 4 : 3;       // stages of expanded operands
+    static constexpr int A_D = KS == 1 ? 2 : 1;      // own A rounds in flight per thread
+    static constexpr int A_RING = A_D + 1;           // packed A ring slots per group
+    static constexpr int A_COL0 = 512 - SU * 32 * KS;   // A stages: top TMEM columns
+};
 constexpr int TMEM_COLS = 512;
-constexpr int A_COL0 = TMEM_COLS - S_U * 32;  // A stages live in the top columns
 
 constexpr int WARP_TMA = 0, WARP_MMA = 1, WARP_A0 = 2, WARP_B0 = 10, WARP_E0 = 18;
 // two groups of four A warps take alternate K steps
@@ -75,7 +81,7 @@ enum { EPI_GEMM = 0, EPI_CODES = 1, EPI_CODES_RES = 2, EPI_GENERAL = 3 };
 
 struct TcParams {
     // problem
-    int M, Ncols, ksteps, BN, m_tiles, n_tiles, n_acc, s_p;
+    int M, Ncols, ksteps, rounds, BN, m_tiles, n_tiles, n_acc, s_p;
     // b_res = 1: the whole expanded B tile (all K steps) stays in shared memory
     // for the life of the CTA (one N tile, few K steps: small weight matrices)
     int b_res, b_stages;
@@ -206,49 +212,53 @@ struct SmemLayout {
 constexpr int MAX_S_P = 4;
 constexpr int MAX_B_STAGES = 16;
 
-__host__ __device__ inline SmemLayout smem_layout(int BN, int bits, int s_p, int b_stages)
+__host__ __device__ inline SmemLayout smem_layout(int BN, int bits, int s_p, int b_stages, int ks)
 {
     SmemLayout L;
     uint32_t o = 0;
-    L.b_tiles = o;  o += b_stages * BN * BK_BYTES;
-    L.b_packed = o; o += s_p * BN * 16 * bits;
-    L.a_ring = o;   o += NUM_A_GROUPS * A_RING * BM * 16 * bits;
+    L.b_tiles = o;  o += b_stages * ks * BN * BK_BYTES;
+    L.b_packed = o; o += s_p * ks * BN * 16 * bits;
+    L.a_ring = o;   o += NUM_A_GROUPS * (ks == 1 ? 3 : 2) * ks * BM * 16 * bits;
     L.epi = o;      o += NUM_E_WARPS * 64 * 4;       // per-warp scale / bias staging
     o = (o + 127u) & ~127u;
-    L.bars = o;     o += 8 * (2 * S_U + MAX_B_STAGES + 2 * MAX_S_P + 4);
+    L.bars = o;     o += 8 * (2 * SU_MAX + MAX_B_STAGES + 2 * MAX_S_P + 4);
     L.tmem_slot = o; o += 8;
     L.abort_flag = o; o += 8;
     L.total = o;
     return L;
 }
 
-template <int BITS, bool A_SIGNED, int EPI>
+template <int BITS, bool A_SIGNED, int EPI, int KS>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
 {
     constexpr bool B_SIGNED = !A_SIGNED;
     constexpr int CH = Chunks<BITS>::CH;
+    constexpr int S_U = Pipe<KS>::SU, A_D = Pipe<KS>::A_D, A_RING = Pipe<KS>::A_RING;
+    constexpr int A_COL0 = Pipe<KS>::A_COL0;
+    static_assert(KS == 1 || BITS != 3, "3-bit rows use single K steps");
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>(
         (reinterpret_cast<uintptr_t>(smem_raw) + 1023u) & ~(uintptr_t)1023u);
-    const SmemLayout L = smem_layout(p.BN, BITS, p.s_p, p.b_stages);
+    const SmemLayout L = smem_layout(p.BN, BITS, p.s_p, p.b_stages, KS);
     const int S_P = p.s_p;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int BN = p.BN;
     const int total_tiles = p.m_tiles * p.n_tiles;
-    const uint32_t b_tile_bytes = BN * BK_BYTES;
-    const uint32_t b_packed_bytes = BN * 16 * BITS;
+    const uint32_t b_sub_bytes = BN * BK_BYTES;              // one K step of the tile
+    const uint32_t b_tile_bytes = KS * b_sub_bytes;          // one round
+    const uint32_t b_packed_bytes = KS * BN * 16 * BITS;
     int my_tiles_all = 0;
     for (int t = blockIdx.x; t < total_tiles; t += gridDim.x) ++my_tiles_all;
     // B is produced for every step of every tile, or once (resident mode)
     const uint32_t n_b_steps =
-        my_tiles_all == 0 ? 0u : (p.b_res ? (uint32_t)p.ksteps : (uint32_t)my_tiles_all * p.ksteps);
+        my_tiles_all == 0 ? 0u : (p.b_res ? (uint32_t)p.rounds : (uint32_t)my_tiles_all * p.rounds);
 
     const uint32_t bars = smem_u32(smem + L.bars);
     auto bar_a_full = [&](int s) { return bars + 8u * s; };
-    auto bar_u_empty = [&](int s) { return bars + 8u * (S_U + s); };
-    auto bar_b_full = [&](int s) { return bars + 8u * (2 * S_U + s); };
-    constexpr int BAR_P = 2 * S_U + MAX_B_STAGES;
+    auto bar_u_empty = [&](int s) { return bars + 8u * (SU_MAX + s); };
+    auto bar_b_full = [&](int s) { return bars + 8u * (2 * SU_MAX + s); };
+    constexpr int BAR_P = 2 * SU_MAX + MAX_B_STAGES;
     auto bar_p_full = [&](int s) { return bars + 8u * (BAR_P + s); };
     auto bar_p_empty = [&](int s) { return bars + 8u * (BAR_P + MAX_S_P + s); };
     auto bar_acc_full = [&](int s) { return bars + 8u * (BAR_P + 2 * MAX_S_P + s); };
@@ -293,9 +303,9 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
                 if (!wait_bar(bar_p_empty(s), ph ^ 1u, ctl, 1)) break;
                 mbar_arrive_expect_tx(bar_p_full(s), b_packed_bytes);
                 tma_load_2d(smem_u32(smem + L.b_packed + s * b_packed_bytes), &tmap_b,
-                            ks * 16 * BITS, (tile % p.n_tiles) * BN, bar_p_full(s));
+                            ks * (KS * 16 * BITS), (tile % p.n_tiles) * BN, bar_p_full(s));
                 if (++s == S_P) { s = 0; ph ^= 1u; }
-                if (++ks == p.ksteps) { ks = 0; tile += gridDim.x; }
+                if (++ks == p.rounds) { ks = 0; tile += gridDim.x; }
             }
             // let outstanding copies land before the CTA can exit
             const uint32_t issued = g;
@@ -318,7 +328,7 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
                 tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + as * BN;
 #pragma unroll 1
-                for (int ks = 0; ks < p.ksteps; ++ks, ++g) {
+                for (int ks = 0; ks < p.rounds; ++ks, ++g) {
                     const int s = g % S_U;
                     const uint32_t ph = (g / S_U) & 1u;
                     const int bs = p.b_res ? ks : s;
@@ -326,10 +336,12 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
                         if (!(ok = wait_bar(bar_b_full(bs), p.b_res ? 0u : ph, ctl, 10))) break;
                     if (!(ok = wait_bar(bar_a_full(s), ph, ctl, 4))) break;
                     tc_fence_after_sync();
-                    // 4 instructions, 32 bytes of K each
-                    mma_i8_ts_x4(d_tmem, tmem_base + A_COL0 + s * 32,
-                                 b_desc_lo0 + bs * (b_tile_bytes >> 4), b_desc_hi, idesc,
-                                 (uint32_t)ks);
+                    // per K step 4 instructions, 32 bytes of K each
+#pragma unroll
+                    for (int h = 0; h < KS; ++h)
+                        mma_i8_ts_x4(d_tmem, tmem_base + A_COL0 + (s * KS + h) * 32,
+                                     b_desc_lo0 + (bs * KS + h) * (b_sub_bytes >> 4), b_desc_hi,
+                                     idesc, (uint32_t)(ks | h));
                     mma_commit(bar_u_empty(s));
                 }
                 if (ok) mma_commit(bar_acc_full(as));
@@ -346,12 +358,12 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
         const int group = (warp - WARP_A0) >> 2;
         const int quarter = warp & 3;              // TMEM lane quarter of this warp
         const int row = quarter * 32 + lane;
-        constexpr int SLOT_BYTES = CH * BM * 16;   // ring slot = CH planes x 128 rows x 16 B
+        constexpr int SLOT_BYTES = KS * CH * BM * 16;   // ring slot = KS*CH planes x 128 rows x 16 B
         const uint32_t cell0 =
             smem_u32(smem + L.a_ring) + group * (A_RING * SLOT_BYTES) + row * 16;
         // walk position over the flattened (tile, K step) sequence; starts one
         // tile back with ld_ks at its end, so that the first step advances
-        int ld_tile = (int)blockIdx.x - (int)gridDim.x, ld_ks = p.ksteps, ld_slot = 0;
+        int ld_tile = (int)blockIdx.x - (int)gridDim.x, ld_ks = p.rounds, ld_slot = 0;
         int tap = 0, kw = 0, off = 0;
         uint32_t tap_mask = 0;                     // bit t: filter tap t is inside the image
         const uint8_t *src = p.act;
@@ -376,7 +388,7 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
         };
         // one K step of the walk: with `load`, its CH chunks go to the ring
         auto walk_step = [&](bool load) {
-            if (ld_ks == p.ksteps) {
+            if (ld_ks == p.rounds) {
                 ld_ks = 0;
                 ld_tile += gridDim.x;
                 set_tile(ld_tile);
@@ -384,9 +396,9 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
             if (ld_tile < total_tiles) {
                 const uint32_t dst = cell0 + ld_slot * SLOT_BYTES;
 #pragma unroll
-                for (int j = 0; j < CH; ++j) {
+                for (int j = 0; j < KS * CH; ++j) {
                     if (load) {
-                        const bool ok = (tap_mask >> tap) & 1u;
+                        const bool ok = tap < 32 && ((tap_mask >> tap) & 1u);
                         cp_async_16(dst + j * (BM * 16), ok ? src : p.act, ok ? 16u : 0u);
                     }
                     off += 16;
@@ -401,7 +413,7 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
                 if (load && ++ld_slot == A_RING) ld_slot = 0;
             }
         };
-        const uint32_t n_steps = (uint32_t)my_tiles_all * p.ksteps;
+        const uint32_t n_steps = (uint32_t)my_tiles_all * p.rounds;
         // own steps: g = group, group + 2, ...
         const uint32_t n_own = n_steps > (uint32_t)group ? (n_steps - group + 1) / 2 : 0u;
         int rd_slot = 0, pend_s = -1;
@@ -423,21 +435,28 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
             if (i < (uint32_t)A_D) continue;
             const uint32_t g = 2 * (i - A_D) + group;
             cp_async_wait<A_D>();                  // own step i - A_D has landed
-            uint32_t o[32];
-            {
-                uint4 cur[CH];
-#pragma unroll
-                for (int j = 0; j < CH; ++j)
-                    cur[j] = lds_128(cell0 + rd_slot * SLOT_BYTES + j * (BM * 16));
-                expand_row_regs<BITS, A_SIGNED>(cur, p.orv, o);
-            }
-            if (++rd_slot == A_RING) rd_slot = 0;
             const int s = g % S_U;
             const uint32_t ph = (g / S_U) & 1u;
-            if (!(ok = wait_bar(bar_u_empty(s), ph ^ 1u, ctl, 5))) break;
-            tc_fence_after_sync();
-            __syncwarp();
-            tmem_st_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + A_COL0 + s * 32, o);
+#pragma unroll
+            for (int h = 0; h < KS; ++h) {
+                uint32_t o[32];
+                {
+                    uint4 cur[CH];
+#pragma unroll
+                    for (int j = 0; j < CH; ++j)
+                        cur[j] = lds_128(cell0 + rd_slot * SLOT_BYTES + (h * CH + j) * (BM * 16));
+                    expand_row_regs<BITS, A_SIGNED>(cur, p.orv, o);
+                }
+                if (h == 0) {
+                    if (!(ok = wait_bar(bar_u_empty(s), ph ^ 1u, ctl, 5))) break;
+                    tc_fence_after_sync();
+                }
+                __syncwarp();
+                tmem_st_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + A_COL0 +
+                                  (s * KS + h) * 32, o);
+            }
+            if (!ok) break;
+            if (++rd_slot == A_RING) rd_slot = 0;
             pend_s = s;
             publish();                             // the other group's step overlaps this
         }
@@ -445,11 +464,14 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
     } else if (warp < WARP_E0) {
         // ---------------- B: expand packed shared tiles ---------------------
         const int tid = threadIdx.x - WARP_B0 * 32;
-        // chunk c = tid + NUM_B_THREADS*i -> row = c / CH, j = c % CH; the
-        // swizzle term (row & 7) does not depend on i
-        constexpr int ROWS_PER_IT = (BITS == 3) ? NUM_B_THREADS : NUM_B_THREADS / CH;
+        // a packed row of the round holds CHK = KS*CH chunks; chunk c = tid +
+        // NUM_B_THREADS*i -> row = c / CHK, K step h = (c % CHK) / CH, chunk j =
+        // c % CH; the swizzle term (row & 7) does not depend on i
+        constexpr int CHK = KS * CH;
+        constexpr int ROWS_PER_IT = (BITS == 3) ? NUM_B_THREADS : NUM_B_THREADS / CHK;
         constexpr int MAX_IT = (BITS == 3) ? 1 : (256 * CH) / NUM_B_THREADS;
-        const int row0 = (BITS == 3) ? tid : tid / CH;
+        const int row0 = (BITS == 3) ? tid : tid / CHK;
+        const int h = (BITS == 3) ? 0 : (tid % CHK) / CH;
         const int j = (BITS == 3) ? 0 : tid % CH;
         const int sw = row0 & 7;
         const int n_it = (BN + ROWS_PER_IT - 1) / ROWS_PER_IT;
@@ -492,7 +514,7 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
                         if (i < n_it && row0 + i * ROWS_PER_IT < BN)
                             v[i] = reinterpret_cast<const uint4 *>(src)[tid + i * NUM_B_THREADS];
                     if (!p.b_res && !(ok = wait_bar(bar_u_empty(su), phu ^ 1u, ctl, 7))) break;
-                    uint8_t *rowp = dst + row0 * BK_BYTES;
+                    uint8_t *rowp = dst + h * b_sub_bytes + row0 * BK_BYTES;
 #pragma unroll
                     for (int i = 0; i < MAX_IT; ++i) {
                         if (i < n_it && row0 + i * ROWS_PER_IT < BN) {
@@ -866,15 +888,17 @@ int make_rows_tmap(CUtensorMap *map, const void *base, uint64_t row_bytes, uint6
 // Resident B: one N tile and few K steps, so the expanded B tile of every K
 // step fits in shared memory next to the rings; it is then expanded once per
 // CTA instead of once per M tile.
-void choose_b_mode(TcParams *p, int bits)
+void choose_b_mode(TcParams *p, int bits, int ks)
 {
+    p->rounds = (p->ksteps + ks - 1) / ks;
+    p->n_acc = 2 * p->BN <= (ks == 1 ? Pipe<1>::A_COL0 : Pipe<2>::A_COL0) ? 2 : 1;
     p->b_res = 0;
-    p->b_stages = S_U;
-    if (p->n_tiles == 1 && p->ksteps <= MAX_B_STAGES && p->m_tiles > 148) {
-        const SmemLayout L = smem_layout(p->BN, bits, p->s_p, p->ksteps);
+    p->b_stages = ks == 1 ? Pipe<1>::SU : Pipe<2>::SU;
+    if (p->n_tiles == 1 && p->rounds <= MAX_B_STAGES && p->m_tiles > 148) {
+        const SmemLayout L = smem_layout(p->BN, bits, p->s_p, p->rounds, ks);
         if (L.total + 1024 <= 227u * 1024u) {
             p->b_res = 1;
-            p->b_stages = p->ksteps;
+            p->b_stages = p->rounds;
         }
     }
 }
@@ -899,14 +923,14 @@ int pick_bn(int m_tiles, int ncols, int bits)
     return best;
 }
 
-template <int BITS, bool A_SIGNED, int EPI>
+template <int BITS, bool A_SIGNED, int EPI, int KS>
 int launch_tc(const CUtensorMap &tmap, const TcParams &p, cudaStream_t s)
 {
-    const SmemLayout L = smem_layout(p.BN, BITS, p.s_p, p.b_stages);
+    const SmemLayout L = smem_layout(p.BN, BITS, p.s_p, p.b_stages, KS);
     const int smem_bytes = (int)L.total + 1024;
     static bool configured = false;
     if (!configured) {
-        if (cudaFuncSetAttribute(dsq_tc_kernel<BITS, A_SIGNED, EPI>,
+        if (cudaFuncSetAttribute(dsq_tc_kernel<BITS, A_SIGNED, EPI, KS>,
                                  cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  227 * 1024) != cudaSuccess)
             return DSQ_ERR_CUDA;
@@ -914,37 +938,62 @@ int launch_tc(const CUtensorMap &tmap, const TcParams &p, cudaStream_t s)
     }
     int grid = p.m_tiles * p.n_tiles;
     if (grid > 148) grid = 148;
-    if (p.BN * p.n_acc > A_COL0) return DSQ_ERR_UNSUPPORTED;
-    dsq_tc_kernel<BITS, A_SIGNED, EPI><<<grid, NUM_THREADS, smem_bytes, s>>>(tmap, p);
+    if (p.BN * p.n_acc > Pipe<KS>::A_COL0 || L.total + 1024 > 227u * 1024u)
+        return DSQ_ERR_UNSUPPORTED;
+    dsq_tc_kernel<BITS, A_SIGNED, EPI, KS><<<grid, NUM_THREADS, smem_bytes, s>>>(tmap, p);
     return dsq_launch_status();
 }
 
-template <int BITS>
+template <int BITS, int KS>
 int launch_conv(int epi, const CUtensorMap &tmap, const TcParams &p, cudaStream_t s)
 {
     switch (epi) {
-    case EPI_CODES: return launch_tc<BITS, false, EPI_CODES>(tmap, p, s);
-    case EPI_CODES_RES: return launch_tc<BITS, false, EPI_CODES_RES>(tmap, p, s);
-    default: return launch_tc<BITS, false, EPI_GENERAL>(tmap, p, s);
+    case EPI_CODES: return launch_tc<BITS, false, EPI_CODES, KS>(tmap, p, s);
+    case EPI_CODES_RES: return launch_tc<BITS, false, EPI_CODES_RES, KS>(tmap, p, s);
+    default: return launch_tc<BITS, false, EPI_GENERAL, KS>(tmap, p, s);
     }
 }
 
-int dispatch_tc(int bits, int epi, const CUtensorMap &tmap, const TcParams &p, cudaStream_t s)
+int dispatch_tc(int bits, int epi, int ks, const CUtensorMap &tmap, const TcParams &p,
+                cudaStream_t s)
 {
     if (epi == EPI_GEMM) {
-        if (bits == 4) return launch_tc<4, true, EPI_GEMM>(tmap, p, s);
-        if (bits == 3) return launch_tc<3, true, EPI_GEMM>(tmap, p, s);
-        if (bits == 2) return launch_tc<2, true, EPI_GEMM>(tmap, p, s);
+        if (bits == 4) return ks == 2 ? launch_tc<4, true, EPI_GEMM, 2>(tmap, p, s)
+                                      : launch_tc<4, true, EPI_GEMM, 1>(tmap, p, s);
+        if (bits == 3) return launch_tc<3, true, EPI_GEMM, 1>(tmap, p, s);
+        if (bits == 2) return ks == 2 ? launch_tc<2, true, EPI_GEMM, 2>(tmap, p, s)
+                                      : launch_tc<2, true, EPI_GEMM, 1>(tmap, p, s);
         return DSQ_ERR_UNSUPPORTED;
     }
-    if (bits == 4) return launch_conv<4>(epi, tmap, p, s);
-    if (bits == 2) return launch_conv<2>(epi, tmap, p, s);
+    if (bits == 4) return ks == 2 ? launch_conv<4, 2>(epi, tmap, p, s) : launch_conv<4, 1>(epi, tmap, p, s);
+    if (bits == 2) return ks == 2 ? launch_conv<2, 2>(epi, tmap, p, s) : launch_conv<2, 1>(epi, tmap, p, s);
     return DSQ_ERR_UNSUPPORTED;
+}
+
+// K steps per barrier round: two when the N tile is narrow enough for the
+// doubled stages to fit tensor memory and shared memory
+int g_forced_ks = 0;
+int pick_ks(const TcParams &p, int bits)
+{
+    if (g_forced_ks) return (bits == 3 || p.BN > 128) ? 1 : g_forced_ks;
+    if (bits == 3 || p.BN > 128 || p.ksteps < 2) return 1;
+    // when the expanded B tile can stay resident with single K steps, the
+    // rounds are cheap already and single steps measured slightly faster
+    TcParams q = p;
+    choose_b_mode(&q, bits, 1);
+    return q.b_res ? 1 : 2;
 }
 
 }  // namespace
 
 extern "C" {
+
+int dsq_set_round_k_steps(int ks)
+{
+    if (ks != 0 && ks != 1 && ks != 2) return DSQ_ERR_SHAPE;
+    g_forced_ks = ks;
+    return DSQ_OK;
+}
 
 int dsq_set_tile_n(int bn)
 {
@@ -979,9 +1028,9 @@ int dsq_gemm(const void *A_codes, const void *B_codes, int64_t M, int64_t N, int
     p.BN = pick_bn(p.m_tiles, (int)N, bits);
     if (bits == 2 && p.BN < 64) p.BN = 64;
     p.n_tiles = (int)((N + p.BN - 1) / p.BN);
-    p.n_acc = 2 * p.BN <= A_COL0 ? 2 : 1;
-    p.s_p = p.BN > 192 ? 3 : 4;
-    choose_b_mode(&p, bits);
+    p.s_p = 3;
+    const int ks = pick_ks(p, bits);
+    choose_b_mode(&p, bits, ks);
     p.act = (const uint8_t *)A_codes;
     p.H = 1; p.W = (int)M; p.Ho = 1; p.Wo = (int)M;
     p.stride = 1; p.pad = 0; p.KW = 1; p.taps = 1; p.P = (int)pitch;
@@ -993,9 +1042,9 @@ int dsq_gemm(const void *A_codes, const void *B_codes, int64_t M, int64_t N, int
     p.D_f32 = D_f32;
     p.ws = (int *)workspace;
     CUtensorMap tmap;
-    int st = make_rows_tmap(&tmap, B_codes, pitch, (uint64_t)N, pitch, 16 * bits, p.BN);
+    int st = make_rows_tmap(&tmap, B_codes, pitch, (uint64_t)N, pitch, ks * 16 * bits, p.BN);
     if (st) return st;
-    return dispatch_tc(bits, EPI_GEMM, tmap, p, (cudaStream_t)stream);
+    return dispatch_tc(bits, EPI_GEMM, ks, tmap, p, (cudaStream_t)stream);
 }
 
 int dsq_conv2d(const void *act_codes, const dsq_nhwc_t *shape, const dsq_quant_t *act_q,
@@ -1040,9 +1089,9 @@ int dsq_conv2d(const void *act_codes, const dsq_nhwc_t *shape, const dsq_quant_t
     p.m_tiles = (int)((M + BM - 1) / BM);
     p.BN = pick_bn(p.m_tiles, conv->Cout, bits);
     p.n_tiles = (conv->Cout + p.BN - 1) / p.BN;
-    p.n_acc = 2 * p.BN <= A_COL0 ? 2 : 1;
-    p.s_p = p.BN > 192 ? 3 : 4;
-    choose_b_mode(&p, bits);
+    p.s_p = 3;
+    const int ks = pick_ks(p, bits);
+    choose_b_mode(&p, bits, ks);
     p.act = (const uint8_t *)act_codes;
     p.H = shape->H; p.W = shape->W; p.Ho = Ho; p.Wo = Wo;
     p.stride = conv->stride; p.pad = conv->pad; p.KW = conv->KW; p.taps = taps; p.P = (int)P;
@@ -1058,7 +1107,7 @@ int dsq_conv2d(const void *act_codes, const dsq_nhwc_t *shape, const dsq_quant_t
     }
     p.ws = (int *)workspace;
     CUtensorMap tmap;
-    st = make_rows_tmap(&tmap, w_packed, row_bytes, (uint64_t)conv->Cout, row_bytes, 16 * bits,
+    st = make_rows_tmap(&tmap, w_packed, row_bytes, (uint64_t)conv->Cout, row_bytes, ks * 16 * bits,
                         p.BN);
     if (st) return st;
     // largest |2*acc + S_a| below 2^22: the epilogue may convert integers to
@@ -1067,7 +1116,7 @@ int dsq_conv2d(const void *act_codes, const dsq_nhwc_t *shape, const dsq_quant_t
                           (2.0 * (double)(1 << (bits - 1)) + 1.0) < 4194304.0;
     const int epi = (y_f32 || acc_out || !y_codes) ? EPI_GENERAL
                     : (e.residual ? EPI_CODES_RES : EPI_CODES);
-    return dispatch_tc(bits, epi, tmap, p, (cudaStream_t)stream);
+    return dispatch_tc(bits, epi, ks, tmap, p, (cudaStream_t)stream);
 }
 
 int dsq_probe_i8_mma_rate(int iters, float *ms_out, double *macs_out, void *workspace,
