@@ -212,14 +212,16 @@ struct SmemLayout {
 constexpr int MAX_S_P = 4;
 constexpr int MAX_B_STAGES = 16;
 
-__host__ __device__ inline SmemLayout smem_layout(int BN, int bits, int s_p, int b_stages, int ks)
+__host__ __device__ inline SmemLayout smem_layout(int BN, int bits, int s_p, int b_stages, int ks,
+                                                int b_res)
 {
     SmemLayout L;
     uint32_t o = 0;
     L.b_tiles = o;  o += b_stages * ks * BN * BK_BYTES;
     L.b_packed = o; o += s_p * ks * BN * 16 * bits;
     L.a_ring = o;   o += NUM_A_GROUPS * (ks == 1 ? 3 : 2) * ks * BM * 16 * bits;
-    L.epi = o;      o += NUM_E_WARPS * 64 * 4;       // per-warp scale / bias staging
+    // per-warp scale / bias staging (the B warps join the epilogue when resident)
+    L.epi = o;      o += (NUM_E_WARPS + (b_res ? NUM_B_WARPS : 0)) * 64 * 4;
     o = (o + 127u) & ~127u;
     L.bars = o;     o += 8 * (2 * SU_MAX + MAX_B_STAGES + 2 * MAX_S_P + 4);
     L.tmem_slot = o; o += 8;
@@ -240,7 +242,7 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>(
         (reinterpret_cast<uintptr_t>(smem_raw) + 1023u) & ~(uintptr_t)1023u);
-    const SmemLayout L = smem_layout(p.BN, BITS, p.s_p, p.b_stages, KS);
+    const SmemLayout L = smem_layout(p.BN, BITS, p.s_p, p.b_stages, KS, p.b_res);
     const int S_P = p.s_p;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int BN = p.BN;
@@ -278,7 +280,7 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
         }
         for (int s = 0; s < 2; ++s) {
             mbar_init(bar_acc_full(s), 1);   // tcgen05.commit
-            mbar_init(bar_acc_empty(s), NUM_E_WARPS);
+            mbar_init(bar_acc_empty(s), p.b_res ? NUM_E_WARPS + NUM_B_WARPS : NUM_E_WARPS);
         }
         *ctl.abort_flag = 0;
         mbar_init_fence();
@@ -293,6 +295,7 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
 
+    int epi_idx = -1, epi_slot = 0;        // set for warps that run the epilogue
     if (warp == WARP_TMA) {
         // ---------------- B producer: TMA packed tiles --------------------
         if (lane == 0) {
@@ -539,8 +542,22 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
                 }
             }
         }
+        // with a resident B tile these eight warps are done after the first
+        // rounds: they join the epilogue (two more warps per TMEM lane quarter)
+        if (p.b_res && ok) {
+            epi_idx = 1 + ((warp - WARP_B0) >> 2);
+            epi_slot = NUM_E_WARPS + (warp - WARP_B0);
+        }
     } else {
+        epi_idx = 0;
+        epi_slot = warp - WARP_E0;
+    }
+
+    if (epi_idx >= 0) {
         // ---------------- epilogue -------------------------------------------
+        // epi_cnt warps share a lane quarter and take the 32-column chunks of a
+        // tile in turn
+        const int epi_cnt = p.b_res ? 3 : 1;
         const int quarter = warp & 3;                 // TMEM lanes 32q .. 32q+31
         const int row_in_tile = quarter * 32 + lane;
         uint32_t it = 0;
@@ -560,7 +577,7 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
             // per-warp staging of the chunk's 32 scale / bias values: lane i fetches
             // column i (prefetched one chunk ahead), the warp reads them back as
             // broadcast 128-bit shared loads
-            float *epi_scale = reinterpret_cast<float *>(smem + L.epi) + (warp - WARP_E0) * 64;
+            float *epi_scale = reinterpret_cast<float *>(smem + L.epi) + epi_slot * 64;
             float *epi_bias = epi_scale + 32;
             float sc_nx = 0.f, bi_nx = 0.f;
             auto fetch_cols = [&](int c0) {
@@ -572,16 +589,16 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
                     bi_nx = __ldg(p.e.bias + n);
                 }
             };
-            fetch_cols(0);
+            fetch_cols(epi_idx * 32);
 #pragma unroll 1
-            for (int c0 = 0; c0 < BN; c0 += 32) {
+            for (int c0 = epi_idx * 32; c0 < BN; c0 += 32 * epi_cnt) {
                 uint32_t r[32];
                 __syncwarp();
                 tmem_ld_32x32(taddr + c0, r);
                 if (EPI != EPI_GEMM) {
                     epi_scale[lane] = sc_nx;
                     epi_bias[lane] = bi_nx;
-                    fetch_cols(c0 + 32);
+                    fetch_cols(c0 + 32 * epi_cnt);
                     __syncwarp();
                 }
                 tmem_ld_wait();
@@ -895,7 +912,7 @@ void choose_b_mode(TcParams *p, int bits, int ks)
     p->b_res = 0;
     p->b_stages = ks == 1 ? Pipe<1>::SU : Pipe<2>::SU;
     if (p->n_tiles == 1 && p->rounds <= MAX_B_STAGES && p->m_tiles > 148) {
-        const SmemLayout L = smem_layout(p->BN, bits, p->s_p, p->rounds, ks);
+        const SmemLayout L = smem_layout(p->BN, bits, p->s_p, p->rounds, ks, 1);
         if (L.total + 1024 <= 227u * 1024u) {
             p->b_res = 1;
             p->b_stages = p->rounds;
@@ -926,7 +943,7 @@ int pick_bn(int m_tiles, int ncols, int bits)
 template <int BITS, bool A_SIGNED, int EPI, int KS>
 int launch_tc(const CUtensorMap &tmap, const TcParams &p, cudaStream_t s)
 {
-    const SmemLayout L = smem_layout(p.BN, BITS, p.s_p, p.b_stages, KS);
+    const SmemLayout L = smem_layout(p.BN, BITS, p.s_p, p.b_stages, KS, p.b_res);
     const int smem_bytes = (int)L.total + 1024;
     static bool configured = false;
     if (!configured) {
