@@ -934,7 +934,7 @@ int pick_bn(int m_tiles, int ncols, int bits)
         const int n_tiles = (ncols + bn - 1) / bn;
         const int64_t tiles = (int64_t)m_tiles * n_tiles;
         const int64_t waves = (tiles + 147) / 148;
-        const double cost = (double)waves * (64.0 + (bn > 192 ? 1.1 : 1.0) * bn);
+        const double cost = (double)waves * (100.0 + bn);
         if (cost < best_cost) { best_cost = cost; best = bn; }
     }
     return best;
