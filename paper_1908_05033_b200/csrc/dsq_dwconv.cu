@@ -1,9 +1,10 @@
 // Depthwise 3x3 convolution on packed codes, CUDA cores.  A depthwise
 // convolution has no shared contraction dimension across channels, so it is
-// not tensor-core work: each thread owns 8 channels of one output pixel (one
-// 32-bit word at 4 bits, one 16-bit half-word at 2 bits), walks the 3x3 taps
-// on packed words and applies the shared epilogue.  Inputs and outputs move
-// as packed codes only: bits/8 bytes per element each way.
+// not tensor-core work: each thread owns 8 channels (one 32-bit word at 4
+// bits, one 16-bit half-word at 2 bits) of four adjacent output pixels, walks
+// the 3x3 taps on packed words and applies the dequantise / requantise
+// epilogue.  Inputs and outputs move as packed codes only: bits/8 bytes per
+// element each way.
 #include "dsq_epilogue.cuh"
 
 namespace {
@@ -15,72 +16,119 @@ __device__ __forceinline__ uint32_t load_unit(const uint8_t *p)
     return __ldg(reinterpret_cast<const uint16_t *>(p));
 }
 
-template <int BITS>
+// One thread: 8 channels (one unit) of OW = 4 horizontally adjacent output
+// pixels.  The 3 x (OW-1)*stride+3 input window and the 9 weight units are
+// loaded once as packed words; then channel by channel the fields are
+// extracted (each activation field is used by up to three outputs) and the
+// four 9-tap sums are formed.  With the symmetric weight grid the weights are
+// taken as 2c+1, so the sum is 2*acc + S_a directly.  Per output element this
+// is about 30 integer / fp32 instructions against 1 byte of HBM traffic.
+template <int BITS, int STRIDE>
 __global__ void __launch_bounds__(256)
 dwconv3x3_kernel(const uint8_t *__restrict__ act, const uint8_t *__restrict__ wgt,
-                 int N, int H, int W, int C, int Ho, int Wo, int stride,
-                 int pitch, DsqEpi e)
+                 int N, int H, int W, int C, int Ho, int Wo, int pitch, DsqEpi e)
 {
     constexpr int UB = BITS;                 // bytes per 8-channel unit
     constexpr uint32_t MASK = (1u << BITS) - 1u;
+    constexpr int OW = 4;                    // outputs per thread along W
+    constexpr int IW = (OW - 1) * STRIDE + 3;
     const int units = pitch / UB;
-    const int64_t total = (int64_t)N * Ho * Wo * units;
+    const int strips = (Wo + OW - 1) / OW;
+    const int64_t total = (int64_t)N * Ho * strips * units;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total;
          i += (int64_t)gridDim.x * blockDim.x) {
         const int u = (int)(i % units);
-        const int64_t pix = i / units;
-        const int wo = (int)(pix % Wo);
-        const int ho = (int)((pix / Wo) % Ho);
-        const int n = (int)(pix / ((int64_t)Wo * Ho));
+        int64_t t = i / units;
+        const int sx = (int)(t % strips);
+        t /= strips;
+        const int ho = (int)(t % Ho);
+        const int n = (int)(t / Ho);
+        const int wo0 = sx * OW;
+        const int hi0 = ho * STRIDE - 1, wi0 = wo0 * STRIDE - 1;
 
-        int acc[8], sa[8];
+        uint32_t a[3][IW], wv[9];
 #pragma unroll
-        for (int f = 0; f < 8; ++f) acc[f] = sa[f] = 0;
-
+        for (int r = 0; r < 3; ++r) {
+            const int hi = hi0 + r;
 #pragma unroll
-        for (int kh = 0; kh < 3; ++kh) {
-            const int hi = ho * stride - 1 + kh;
-            if (hi < 0 || hi >= H) continue;
-#pragma unroll
-            for (int kw = 0; kw < 3; ++kw) {
-                const int wi = wo * stride - 1 + kw;
-                if (wi < 0 || wi >= W) continue;
-                const uint32_t a = load_unit<BITS>(
-                    act + (((int64_t)n * H + hi) * W + wi) * pitch + u * UB);
-                const uint32_t wv =
-                    load_unit<BITS>(wgt + (kh * 3 + kw) * pitch + u * UB);
-#pragma unroll
-                for (int f = 0; f < 8; ++f) {
-                    const int q = (int)((a >> (BITS * f)) & MASK);
-                    const int c = ((int)(wv << (32 - BITS * (f + 1)))) >> (32 - BITS);
-                    acc[f] += q * c;
-                    sa[f] += q;
-                }
+            for (int x = 0; x < IW; ++x) {
+                const int wi = wi0 + x;
+                a[r][x] = 0u;
+                if (hi >= 0 && hi < H && wi >= 0 && wi < W)
+                    a[r][x] = load_unit<BITS>(
+                        act + (((int64_t)n * H + hi) * W + wi) * pitch + u * UB);
             }
         }
+#pragma unroll
+        for (int k = 0; k < 9; ++k) wv[k] = load_unit<BITS>(wgt + k * pitch + u * UB);
 
-        uint32_t res = 0;
-        if (e.residual) res = load_unit<BITS>(e.residual + pix * pitch + u * UB);
-        uint32_t word = 0;
+        const int64_t pix0 = ((int64_t)n * Ho + ho) * Wo + wo0;
+        uint32_t res[OW], cw[OW];
+#pragma unroll
+        for (int o = 0; o < OW; ++o) {
+            cw[o] = 0u;
+            res[o] = 0u;
+            if (e.residual && wo0 + o < Wo)
+                res[o] = load_unit<BITS>(e.residual + (pix0 + o) * pitch + u * UB);
+        }
 #pragma unroll
         for (int f = 0; f < 8; ++f) {
             const int ch = 8 * u + f;
             if (ch >= C) continue;
-            const int v = e.half_offset ? 2 * acc[f] + sa[f] : acc[f];
+            int wq[9];
+#pragma unroll
+            for (int k = 0; k < 9; ++k) {
+                const int c = ((int)(wv[k] << (32 - BITS * (f + 1)))) >> (32 - BITS);
+                wq[k] = e.half_offset ? 2 * c + 1 : c;
+            }
+            int acc[OW];
+#pragma unroll
+            for (int o = 0; o < OW; ++o) acc[o] = 0;
+#pragma unroll
+            for (int r = 0; r < 3; ++r) {
+                int q[IW];
+#pragma unroll
+                for (int x = 0; x < IW; ++x) q[x] = (int)((a[r][x] >> (BITS * f)) & MASK);
+#pragma unroll
+                for (int o = 0; o < OW; ++o)
+#pragma unroll
+                    for (int kw = 0; kw < 3; ++kw) acc[o] += q[o * STRIDE + kw] * wq[r * 3 + kw];
+            }
             float sc = __ldg(e.scale + ch);
             if (e.half_offset) sc = __fmul_rn(sc, 0.5f);
-            float y = dsq_epi_y(v, sc, __ldg(e.bias + ch));
-            if (e.residual)
-                y = dsq_epi_residual(y, (res >> (BITS * f)) & MASK, e.res_delta,
-                                     e.res_lo);
-            if (e.acc_out) e.acc_out[pix * C + ch] = v;
-            if (e.y_f32) e.y_f32[pix * C + ch] = y;
-            if (e.has_requant) word |= dsq_code(y, e.rq) << (BITS * f);
+            const float bi = __ldg(e.bias + ch);
+#pragma unroll
+            for (int o = 0; o < OW; ++o) {
+                if (wo0 + o >= Wo) continue;
+                // |acc| <= 9*15*17: the 1.5*2^23 bias trick converts exactly
+                const float vf = __fsub_rn(__int_as_float(0x4B400000 + acc[o]), 12582912.0f);
+                float y = __fmaf_rn(vf, sc, bi);
+                if (e.residual) {
+                    const uint32_t qr = (res[o] >> (BITS * f)) & MASK;
+                    y = __fadd_rn(y, __fmaf_rn(__fsub_rn(__int_as_float(0x4B000000 | qr),
+                                                         8388608.0f),
+                                               e.res_delta, e.res_lo));
+                }
+                if (e.acc_out) e.acc_out[(pix0 + o) * C + ch] = acc[o];
+                if (e.y_f32) e.y_f32[(pix0 + o) * C + ch] = y;
+                if (e.has_requant) {
+                    const float xc = fminf(fmaxf(y, e.rq.lo), e.rq.hi);
+                    const float rr = __fmaf_rn(__fsub_rn(xc, e.rq.lo), e.rq.inv, 0.5f);
+                    const uint32_t q = min(
+                        (uint32_t)__float_as_int(__fadd_rd(rr, 8388608.0f)) - 0x4B000000u,
+                        (uint32_t)e.rq.qmax);
+                    cw[o] |= q << (BITS * f);
+                }
+            }
         }
         if (e.y_codes) {
-            uint8_t *dst = e.y_codes + pix * pitch + u * UB;
-            if (BITS == 4) *reinterpret_cast<uint32_t *>(dst) = word;
-            else *reinterpret_cast<uint16_t *>(dst) = (uint16_t)word;
+#pragma unroll
+            for (int o = 0; o < OW; ++o) {
+                if (wo0 + o >= Wo) continue;
+                uint8_t *dst = e.y_codes + (pix0 + o) * pitch + u * UB;
+                if (BITS == 4) *reinterpret_cast<uint32_t *>(dst) = cw[o];
+                else *reinterpret_cast<uint16_t *>(dst) = (uint16_t)cw[o];
+            }
         }
     }
 }
@@ -114,18 +162,19 @@ extern "C" int dsq_dwconv2d(const void *act_codes, const dsq_nhwc_t *shape,
     const int Ho = (shape->H + 2 - 3) / conv->stride + 1;
     const int Wo = (shape->W + 2 - 3) / conv->stride + 1;
     const int pitch = (int)dsq_row_pitch(shape->C, bits);
-    const int64_t total = (int64_t)shape->N * Ho * Wo * (pitch / bits);
+    const int64_t total = (int64_t)shape->N * Ho * ((Wo + 3) / 4) * (pitch / bits);
     int64_t g = (total + 255) / 256;
     if (g > 148 * 32) g = 148 * 32;
     if (g < 1) g = 1;
     cudaStream_t s = (cudaStream_t)stream;
-    if (bits == 4)
-        dwconv3x3_kernel<4><<<(int)g, 256, 0, s>>>(
-            (const uint8_t *)act_codes, (const uint8_t *)w_packed, shape->N,
-            shape->H, shape->W, shape->C, Ho, Wo, conv->stride, pitch, e);
-    else
-        dwconv3x3_kernel<2><<<(int)g, 256, 0, s>>>(
-            (const uint8_t *)act_codes, (const uint8_t *)w_packed, shape->N,
-            shape->H, shape->W, shape->C, Ho, Wo, conv->stride, pitch, e);
+    const uint8_t *a = (const uint8_t *)act_codes, *w = (const uint8_t *)w_packed;
+#define DSQ_DW_LAUNCH(B, S)                                                               \
+    dwconv3x3_kernel<B, S><<<(int)g, 256, 0, s>>>(a, w, shape->N, shape->H, shape->W, shape->C, \
+                                                  Ho, Wo, pitch, e)
+    if (bits == 4 && conv->stride == 1) DSQ_DW_LAUNCH(4, 1);
+    else if (bits == 4) DSQ_DW_LAUNCH(4, 2);
+    else if (conv->stride == 1) DSQ_DW_LAUNCH(2, 1);
+    else DSQ_DW_LAUNCH(2, 2);
+#undef DSQ_DW_LAUNCH
     return dsq_launch_status();
 }
