@@ -36,6 +36,11 @@ if ROOT not in sys.path:
 
 import dsq_inputs  # noqa: E402
 
+# DRAM traffic of the dominant kernel (dsq_tc_kernel) per launch in this
+# workload, from one ncu capture (profiles/bench_launch_list.txt); valid only
+# for the kernel sources it was taken on (checked by hash)
+TRAFFIC = {"bytes_per_launch": 4728037, "sources_sha256": "d1afa4523e5fc3d89452a4e737ce83b6b633f4ce36c430d033b114b1f7069966"}
+
 WORKLOAD = "resnet18-shaped stack, 4-bit W/A, batch 64, 56x56x64 stem output, 19 convs"
 METRIC = "4-bit ResNet-18 conv-stack throughput (effective low-bit conv TOPS alongside)"
 INT8_NOMINAL_TOPS = 4500.0
@@ -44,6 +49,20 @@ INT8_NOMINAL_TOPS = 4500.0
 # ---------------------------------------------------------------------------
 # helpers
 # ---------------------------------------------------------------------------
+def kernel_sources_sha256():
+    import hashlib
+    h = hashlib.sha256()
+    for f in ("dsq_tc.cu", "dsq_ptx.cuh", "dsq_epilogue.cuh", "dsq_common.cuh"):
+        h.update(open(os.path.join(ROOT, "paper_1908_05033_b200", "csrc", f), "rb").read())
+    return h.hexdigest()
+
+
+def measured_traffic():
+    if TRAFFIC["bytes_per_launch"] is None:
+        return None
+    return TRAFFIC["bytes_per_launch"] if TRAFFIC["sources_sha256"] == kernel_sources_sha256() else None
+
+
 def load_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -304,6 +323,53 @@ def kernel_times_eager(g, xs, torch, reps=5):
     return out
 
 
+def algorithmic_bytes_step(st, batch):
+    """Packed code bytes every conv of the stack must move for one batch: its
+    input codes, its residual codes, its output codes and its packed weights."""
+    shapes = st.tensor_shapes()
+    b = st.bits / 8.0
+    total = 0.0
+    for L in st.layers:
+        if L.kind == "pool":
+            continue
+        Hi, Wi, Ci = shapes[L.src]
+        Ho, Wo, Co = shapes[L.dst]
+        total += batch * (Hi * Wi * Ci + Ho * Wo * Co) * b
+        if L.residual is not None:
+            total += batch * Ho * Wo * Co * b
+        total += Co * L.ksize * L.ksize * (1 if L.kind == "dw" else Ci) * b
+    return total
+
+
+def time_other_stack(st, wid, torch, dev, steps=50):
+    """ms per step and images/s of another workload's stack (graph replay)."""
+    from paper_1908_05033_b200.stack import GpuStack
+    params = dsq_inputs.stack_params(st, workload_id=wid)
+    x = torch.from_numpy(dsq_inputs.stack_input(st, workload_id=wid)).to(dev)
+    g = GpuStack(st, params, device=dev)
+    side = torch.cuda.Stream(device=dev)
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        g.forward(x)
+        torch.cuda.synchronize()
+        gr = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(gr, stream=side):
+            g.forward(x)
+    torch.cuda.synchronize()
+    for _ in range(5):
+        gr.replay()
+    e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        gr.replay()
+    e1.record(); torch.cuda.synchronize()
+    g.check()
+    ms = e0.elapsed_time(e1) / steps
+    return {"ms_per_step": ms, "img_per_s": st.batch / (ms * 1e-3),
+            "effective_tops": 2.0 * st.macs_per_image() * st.batch / (ms * 1e-3) / 1e12,
+            "batch": st.batch, "bits": st.bits, "launches_per_step": g.n_launches()}
+
+
 def run_ours(args):
     import torch
     rank, world, local = dist_setup(args.gpus)
@@ -370,7 +436,8 @@ def run_ours(args):
                        "(int8:bf16 nominal ratio); nominal 4500, own MMA-only probe in extras",
         "avg_launch_ms": conv_in_step_ms / n_conv,
         "how": "graph step time minus the quantise kernel's eager event time, over 19 launches",
-        "traffic": None,
+        "traffic": measured_traffic(),
+        "algorithmic_bytes_per_launch": algorithmic_bytes_step(st, batch) / n_conv,
     }
 
     line = {
@@ -460,6 +527,10 @@ def run_ours(args):
                                   "frac_of_2x_bf16_burst": gt / (2 * peaks["bf16_tflops"]),
                                   "l2": "256 MB flush between launches"}
         dsq.check_workspace(ws, "extras")
+        del Ap, Bp, Cm, flush
+        extras["mobilenetv2_stack_b4_batch64"] = time_other_stack(
+            dsq_inputs.mobilenetv2_stack(), 4, torch, dev)
+        extras["vgg16_stack_b2_batch32"] = time_other_stack(dsq_inputs.vgg16_stack(), 5, torch, dev)
         extras["quantize_in_step_ms"] = quant_ms
         extras["conv_kernels_in_step_ms"] = conv_ms
         extras["per_layer_ms"] = {n: round(t, 4) for _, n, t in kt}
