@@ -51,15 +51,24 @@ namespace {
 
 constexpr int BM = 128;               // tile rows = MMA M
 constexpr int BK_BYTES = 128;         // int8 bytes per row per K step (128 codes)
-// A barrier round covers KS K steps of 128 codes (KS = 1 or 2, template
-// parameter): with small N tiles the fixed cost of a round (barrier hand-offs,
-// MMA issue) outweighs its work, so two K steps share one round.
+// Pipeline modes (template parameter PM).  A barrier round covers KS K steps of
+// 128 codes: with the fixed cost of a round (barrier hand-offs, MMA issue) near
+// a thousand cycles, two K steps per round pay whenever they fit.
+//   PM 1: KS = 1, 4 stages, two A groups          (any N tile, 3-bit rows)
+//   PM 2: KS = 2, 3 stages, two A groups          (N tile <= 128)
+//   PM 3: KS = 2, 2 stages, one A group ("wide")  (N tile 192 / 256: shared memory
+//         holds two double stages of B only; the second A group's warps help
+//         the epilogue instead)
 constexpr int SU_MAX = 4;
-template <int KS> struct Pipe {
-    static constexpr int SU = KS == 1 ? 4 : 3;       // stages of expanded operands
-    static constexpr int A_D = KS == 1 ? 2 : 1;      // own A rounds in flight per thread
-    static constexpr int A_RING = A_D + 1;           // packed A ring slots per group
-    static constexpr int A_COL0 = 512 - SU * 32 * KS;   // A stages: top TMEM columns
+template <int PM> struct Pipe {
+    static constexpr int KS = PM == 1 ? 1 : 2;
+    static constexpr bool WIDE = PM == 3;
+    static constexpr int SU = PM == 1 ? 4 : PM == 2 ? 3 : 2;   // stages of expanded operands
+    static constexpr int GROUPS = WIDE ? 1 : 2;              // A groups in use
+    static constexpr int A_D = PM == 1 ? 2 : 1;              // own A rounds in flight per thread
+    static constexpr int A_RING = A_D + 1;                   // packed A ring slots per group
+    static constexpr int A_COL0 = 512 - SU * 32 * KS;        // A stages: top TMEM columns
+    static constexpr int S_P = WIDE ? 2 : 3;                 // packed B ring slots
 };
 constexpr int TMEM_COLS = 512;
 
@@ -85,6 +94,8 @@ struct TcParams {
     // b_res = 1: the whole expanded B tile (all K steps) stays in shared memory
     // for the life of the CTA (one N tile, few K steps: small weight matrices)
     int b_res, b_stages;
+    int epw;                          // epilogue warps per TMEM lane quarter (1..3)
+    int smem_bytes;                   // dynamic shared memory given to the launch
     // A gather geometry (a GEMM is a 1x1 convolution over an M x 1 image)
     const uint8_t *act;
     int H, W, Ho, Wo, stride, pad, KW, taps, P;
@@ -213,15 +224,15 @@ constexpr int MAX_S_P = 4;
 constexpr int MAX_B_STAGES = 16;
 
 __host__ __device__ inline SmemLayout smem_layout(int BN, int bits, int s_p, int b_stages, int ks,
-                                                int b_res)
+                                                int a_slots, int epw)
 {
     SmemLayout L;
     uint32_t o = 0;
     L.b_tiles = o;  o += b_stages * ks * BN * BK_BYTES;
     L.b_packed = o; o += s_p * ks * BN * 16 * bits;
-    L.a_ring = o;   o += NUM_A_GROUPS * (ks == 1 ? 3 : 2) * ks * BM * 16 * bits;
+    L.a_ring = o;   o += a_slots * ks * BM * 16 * bits;
     // per-warp scale / bias staging (the B warps join the epilogue when resident)
-    L.epi = o;      o += (NUM_E_WARPS + (b_res ? NUM_B_WARPS : 0)) * 64 * 4;
+    L.epi = o;      o += 4 * epw * 64 * 4;
     o = (o + 127u) & ~127u;
     L.bars = o;     o += 8 * (2 * SU_MAX + MAX_B_STAGES + 2 * MAX_S_P + 4);
     L.tmem_slot = o; o += 8;
@@ -230,19 +241,29 @@ __host__ __device__ inline SmemLayout smem_layout(int BN, int bits, int s_p, int
     return L;
 }
 
-template <int BITS, bool A_SIGNED, int EPI, int KS>
+template <int BITS, bool A_SIGNED, int EPI, int PM>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
 {
     constexpr bool B_SIGNED = !A_SIGNED;
     constexpr int CH = Chunks<BITS>::CH;
-    constexpr int S_U = Pipe<KS>::SU, A_D = Pipe<KS>::A_D, A_RING = Pipe<KS>::A_RING;
-    constexpr int A_COL0 = Pipe<KS>::A_COL0;
+    constexpr int KS = Pipe<PM>::KS, GROUPS = Pipe<PM>::GROUPS;
+    constexpr bool WIDE = Pipe<PM>::WIDE;
+    constexpr int S_U = Pipe<PM>::SU, A_D = Pipe<PM>::A_D, A_RING = Pipe<PM>::A_RING;
+    constexpr int A_COL0 = Pipe<PM>::A_COL0;
     static_assert(KS == 1 || BITS != 3, "3-bit rows use single K steps");
-    extern __shared__ uint8_t smem_raw[];
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>(
         (reinterpret_cast<uintptr_t>(smem_raw) + 1023u) & ~(uintptr_t)1023u);
-    const SmemLayout L = smem_layout(p.BN, BITS, p.s_p, p.b_stages, KS, p.b_res);
+    const SmemLayout L =
+        smem_layout(p.BN, BITS, p.s_p, p.b_stages, KS, GROUPS * A_RING, p.epw);
+    // the layout must fit behind the 1024-byte aligned base (the host adds
+    // slack only while it stays within the 227 KB limit); same answer in every
+    // thread, taken before any barrier exists
+    if ((uint32_t)(smem - smem_raw) + L.total > (uint32_t)p.smem_bytes) {
+        if (threadIdx.x == 0) atomicCAS(p.ws + DSQ_WS_STATUS, 0, (int)DSQ_ERR_UNSUPPORTED);
+        return;
+    }
     const int S_P = p.s_p;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int BN = p.BN;
@@ -280,7 +301,7 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
         }
         for (int s = 0; s < 2; ++s) {
             mbar_init(bar_acc_full(s), 1);   // tcgen05.commit
-            mbar_init(bar_acc_empty(s), p.b_res ? NUM_E_WARPS + NUM_B_WARPS : NUM_E_WARPS);
+            mbar_init(bar_acc_empty(s), 4 * p.epw);
         }
         *ctl.abort_flag = 0;
         mbar_init_fence();
@@ -359,6 +380,7 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
         // steps in flight, thread-local completion) -> registers -> expand ->
         // tensor memory (tcgen05.st), completed and published at once.
         const int group = (warp - WARP_A0) >> 2;
+        if (group < GROUPS) {
         const int quarter = warp & 3;              // TMEM lane quarter of this warp
         const int row = quarter * 32 + lane;
         constexpr int SLOT_BYTES = KS * CH * BM * 16;   // ring slot = KS*CH planes x 128 rows x 16 B
@@ -417,8 +439,9 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
             }
         };
         const uint32_t n_steps = (uint32_t)my_tiles_all * p.rounds;
-        // own steps: g = group, group + 2, ...
-        const uint32_t n_own = n_steps > (uint32_t)group ? (n_steps - group + 1) / 2 : 0u;
+        // own steps: g = group, group + GROUPS, ...
+        const uint32_t n_own =
+            GROUPS == 1 ? n_steps : (n_steps > (uint32_t)group ? (n_steps - group + 1) / 2 : 0u);
         int rd_slot = 0, pend_s = -1;
         bool ok = true;
         auto publish = [&]() {
@@ -428,15 +451,15 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
             if (lane == 0) mbar_arrive(bar_a_full(pend_s));
             pend_s = -1;
         };
-        if (group == 1) walk_step(false);          // step 0 belongs to group 0
+        if (GROUPS == 2 && group == 1) walk_step(false);   // step 0 belongs to group 0
         // iteration i issues own step i and consumes own step i - A_D
 #pragma unroll 1
         for (uint32_t i = 0; ok && i < n_own + A_D; ++i) {
             walk_step(true);                       // own step (no-op past the end)
             cp_async_commit();                     // one group per own step
-            walk_step(false);                      // the other group's step
+            if (GROUPS == 2) walk_step(false);     // the other group's step
             if (i < (uint32_t)A_D) continue;
-            const uint32_t g = 2 * (i - A_D) + group;
+            const uint32_t g = GROUPS * (i - A_D) + group;
             cp_async_wait<A_D>();                  // own step i - A_D has landed
             const int s = g % S_U;
             const uint32_t ph = (g / S_U) & 1u;
@@ -464,6 +487,11 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
             publish();                             // the other group's step overlaps this
         }
         cp_async_wait<0>();
+        } else if (WIDE) {
+            // the unused second A group helps the epilogue
+            epi_idx = 1;
+            epi_slot = NUM_E_WARPS + (warp - WARP_A0 - 4);
+        }
     } else if (warp < WARP_E0) {
         // ---------------- B: expand packed shared tiles ---------------------
         const int tid = threadIdx.x - WARP_B0 * 32;
@@ -472,7 +500,7 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
         // c % CH; the swizzle term (row & 7) does not depend on i
         constexpr int CHK = KS * CH;
         constexpr int ROWS_PER_IT = (BITS == 3) ? NUM_B_THREADS : NUM_B_THREADS / CHK;
-        constexpr int MAX_IT = (BITS == 3) ? 1 : (256 * CH) / NUM_B_THREADS;
+        constexpr int MAX_IT = (BITS == 3) ? 1 : (WIDE ? 2 : 1) * (256 * CH) / NUM_B_THREADS;
         const int row0 = (BITS == 3) ? tid : tid / CHK;
         const int h = (BITS == 3) ? 0 : (tid % CHK) / CH;
         const int j = (BITS == 3) ? 0 : tid % CH;
@@ -557,7 +585,7 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
         // ---------------- epilogue -------------------------------------------
         // epi_cnt warps share a lane quarter and take the 32-column chunks of a
         // tile in turn
-        const int epi_cnt = p.b_res ? 3 : 1;
+        const int epi_cnt = p.epw;
         const int quarter = warp & 3;                 // TMEM lanes 32q .. 32q+31
         const int row_in_tile = quarter * 32 + lane;
         uint32_t it = 0;
@@ -905,17 +933,33 @@ int make_rows_tmap(CUtensorMap *map, const void *base, uint64_t row_bytes, uint6
 // Resident B: one N tile and few K steps, so the expanded B tile of every K
 // step fits in shared memory next to the rings; it is then expanded once per
 // CTA instead of once per M tile.
-void choose_b_mode(TcParams *p, int bits, int ks)
+struct PipeInfo { int ks, su, a_slots, a_col0, s_p, wide; };
+PipeInfo pipe_info(int pm)
 {
-    p->rounds = (p->ksteps + ks - 1) / ks;
-    p->n_acc = 2 * p->BN <= (ks == 1 ? Pipe<1>::A_COL0 : Pipe<2>::A_COL0) ? 2 : 1;
+    switch (pm) {
+    case 1: return {Pipe<1>::KS, Pipe<1>::SU, Pipe<1>::GROUPS * Pipe<1>::A_RING, Pipe<1>::A_COL0, Pipe<1>::S_P, 0};
+    case 2: return {Pipe<2>::KS, Pipe<2>::SU, Pipe<2>::GROUPS * Pipe<2>::A_RING, Pipe<2>::A_COL0, Pipe<2>::S_P, 0};
+    default: return {Pipe<3>::KS, Pipe<3>::SU, Pipe<3>::GROUPS * Pipe<3>::A_RING, Pipe<3>::A_COL0, Pipe<3>::S_P, 1};
+    }
+}
+
+// Fills the fields that depend on the pipeline mode; picks resident B where it
+// fits (one N tile, few rounds, more M tiles than SMs).
+void choose_b_mode(TcParams *p, int bits, int pm)
+{
+    const PipeInfo pi = pipe_info(pm);
+    p->rounds = (p->ksteps + pi.ks - 1) / pi.ks;
+    p->n_acc = 2 * p->BN <= pi.a_col0 ? 2 : 1;
+    p->s_p = pi.s_p;
     p->b_res = 0;
-    p->b_stages = ks == 1 ? Pipe<1>::SU : Pipe<2>::SU;
-    if (p->n_tiles == 1 && p->rounds <= MAX_B_STAGES && p->m_tiles > 148) {
-        const SmemLayout L = smem_layout(p->BN, bits, p->s_p, p->rounds, ks, 1);
+    p->b_stages = pi.su;
+    p->epw = pi.wide ? 2 : 1;
+    if (!pi.wide && p->n_tiles == 1 && p->rounds <= MAX_B_STAGES && p->m_tiles > 148) {
+        const SmemLayout L = smem_layout(p->BN, bits, p->s_p, p->rounds, pi.ks, pi.a_slots, 3);
         if (L.total + 1024 <= 227u * 1024u) {
             p->b_res = 1;
             p->b_stages = p->rounds;
+            p->epw = 3;
         }
     }
 }
@@ -940,14 +984,17 @@ int pick_bn(int m_tiles, int ncols, int bits)
     return best;
 }
 
-template <int BITS, bool A_SIGNED, int EPI, int KS>
+template <int BITS, bool A_SIGNED, int EPI, int PM>
 int launch_tc(const CUtensorMap &tmap, const TcParams &p, cudaStream_t s)
 {
-    const SmemLayout L = smem_layout(p.BN, BITS, p.s_p, p.b_stages, KS, p.b_res);
-    const int smem_bytes = (int)L.total + 1024;
+    const SmemLayout L = smem_layout(p.BN, BITS, p.s_p, p.b_stages, Pipe<PM>::KS,
+                                     Pipe<PM>::GROUPS * Pipe<PM>::A_RING, p.epw);
+    if (L.total > 227u * 1024u) return DSQ_ERR_UNSUPPORTED;
+    int smem_bytes = (int)L.total + 1024;            // slack for the 1024-byte alignment
+    if (smem_bytes > 227 * 1024) smem_bytes = 227 * 1024;
     static bool configured = false;
     if (!configured) {
-        if (cudaFuncSetAttribute(dsq_tc_kernel<BITS, A_SIGNED, EPI, KS>,
+        if (cudaFuncSetAttribute(dsq_tc_kernel<BITS, A_SIGNED, EPI, PM>,
                                  cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  227 * 1024) != cudaSuccess)
             return DSQ_ERR_CUDA;
@@ -955,45 +1002,53 @@ int launch_tc(const CUtensorMap &tmap, const TcParams &p, cudaStream_t s)
     }
     int grid = p.m_tiles * p.n_tiles;
     if (grid > 148) grid = 148;
-    if (p.BN * p.n_acc > Pipe<KS>::A_COL0 || L.total + 1024 > 227u * 1024u)
-        return DSQ_ERR_UNSUPPORTED;
-    dsq_tc_kernel<BITS, A_SIGNED, EPI, KS><<<grid, NUM_THREADS, smem_bytes, s>>>(tmap, p);
+    if (p.BN * p.n_acc > Pipe<PM>::A_COL0) return DSQ_ERR_UNSUPPORTED;
+    TcParams q = p;
+    q.smem_bytes = smem_bytes;
+    dsq_tc_kernel<BITS, A_SIGNED, EPI, PM><<<grid, NUM_THREADS, smem_bytes, s>>>(tmap, q);
     return dsq_launch_status();
 }
 
-template <int BITS, int KS>
+template <int BITS, int PM>
 int launch_conv(int epi, const CUtensorMap &tmap, const TcParams &p, cudaStream_t s)
 {
     switch (epi) {
-    case EPI_CODES: return launch_tc<BITS, false, EPI_CODES, KS>(tmap, p, s);
-    case EPI_CODES_RES: return launch_tc<BITS, false, EPI_CODES_RES, KS>(tmap, p, s);
-    default: return launch_tc<BITS, false, EPI_GENERAL, KS>(tmap, p, s);
+    case EPI_CODES: return launch_tc<BITS, false, EPI_CODES, PM>(tmap, p, s);
+    case EPI_CODES_RES: return launch_tc<BITS, false, EPI_CODES_RES, PM>(tmap, p, s);
+    default: return launch_tc<BITS, false, EPI_GENERAL, PM>(tmap, p, s);
     }
 }
 
-int dispatch_tc(int bits, int epi, int ks, const CUtensorMap &tmap, const TcParams &p,
-                cudaStream_t s)
+template <int BITS>
+int launch_bits(int epi, int pm, const CUtensorMap &tmap, const TcParams &p, cudaStream_t s)
 {
     if (epi == EPI_GEMM) {
-        if (bits == 4) return ks == 2 ? launch_tc<4, true, EPI_GEMM, 2>(tmap, p, s)
-                                      : launch_tc<4, true, EPI_GEMM, 1>(tmap, p, s);
-        if (bits == 3) return launch_tc<3, true, EPI_GEMM, 1>(tmap, p, s);
-        if (bits == 2) return ks == 2 ? launch_tc<2, true, EPI_GEMM, 2>(tmap, p, s)
-                                      : launch_tc<2, true, EPI_GEMM, 1>(tmap, p, s);
-        return DSQ_ERR_UNSUPPORTED;
+        if (pm == 3) return launch_tc<BITS, true, EPI_GEMM, 3>(tmap, p, s);
+        if (pm == 2) return launch_tc<BITS, true, EPI_GEMM, 2>(tmap, p, s);
+        return launch_tc<BITS, true, EPI_GEMM, 1>(tmap, p, s);
     }
-    if (bits == 4) return ks == 2 ? launch_conv<4, 2>(epi, tmap, p, s) : launch_conv<4, 1>(epi, tmap, p, s);
-    if (bits == 2) return ks == 2 ? launch_conv<2, 2>(epi, tmap, p, s) : launch_conv<2, 1>(epi, tmap, p, s);
+    if (pm == 3) return launch_conv<BITS, 3>(epi, tmap, p, s);
+    if (pm == 2) return launch_conv<BITS, 2>(epi, tmap, p, s);
+    return launch_conv<BITS, 1>(epi, tmap, p, s);
+}
+
+int dispatch_tc(int bits, int epi, int pm, const CUtensorMap &tmap, const TcParams &p,
+                cudaStream_t s)
+{
+    if (bits == 4) return launch_bits<4>(epi, pm, tmap, p, s);
+    if (bits == 2) return launch_bits<2>(epi, pm, tmap, p, s);
+    if (bits == 3 && epi == EPI_GEMM) return launch_tc<3, true, EPI_GEMM, 1>(tmap, p, s);
     return DSQ_ERR_UNSUPPORTED;
 }
 
-// K steps per barrier round: two when the N tile is narrow enough for the
-// doubled stages to fit tensor memory and shared memory
+// Pipeline mode for a problem (see Pipe<PM>); g_forced_ks: 0 automatic, 1 forces
+// single K steps, 2 forces double steps wherever they are possible.
 int g_forced_ks = 0;
-int pick_ks(const TcParams &p, int bits)
+int pick_pm(const TcParams &p, int bits)
 {
-    if (g_forced_ks) return (bits == 3 || p.BN > 128) ? 1 : g_forced_ks;
-    if (bits == 3 || p.BN > 128 || p.ksteps < 2) return 1;
+    if (bits == 3 || p.ksteps < 2 || g_forced_ks == 1) return 1;
+    if (p.BN > 128) return p.ksteps >= 4 ? 3 : 1;
+    if (g_forced_ks == 2) return 2;
     // when the expanded B tile can stay resident with single K steps, the
     // rounds are cheap already and single steps measured slightly faster
     TcParams q = p;
@@ -1045,9 +1100,9 @@ int dsq_gemm(const void *A_codes, const void *B_codes, int64_t M, int64_t N, int
     p.BN = pick_bn(p.m_tiles, (int)N, bits);
     if (bits == 2 && p.BN < 64) p.BN = 64;
     p.n_tiles = (int)((N + p.BN - 1) / p.BN);
-    p.s_p = 3;
-    const int ks = pick_ks(p, bits);
-    choose_b_mode(&p, bits, ks);
+    const int pm = pick_pm(p, bits);
+    const int ks = pm == 1 ? 1 : 2;
+    choose_b_mode(&p, bits, pm);
     p.act = (const uint8_t *)A_codes;
     p.H = 1; p.W = (int)M; p.Ho = 1; p.Wo = (int)M;
     p.stride = 1; p.pad = 0; p.KW = 1; p.taps = 1; p.P = (int)pitch;
@@ -1061,7 +1116,7 @@ int dsq_gemm(const void *A_codes, const void *B_codes, int64_t M, int64_t N, int
     CUtensorMap tmap;
     int st = make_rows_tmap(&tmap, B_codes, pitch, (uint64_t)N, pitch, ks * 16 * bits, p.BN);
     if (st) return st;
-    return dispatch_tc(bits, EPI_GEMM, ks, tmap, p, (cudaStream_t)stream);
+    return dispatch_tc(bits, EPI_GEMM, pm, tmap, p, (cudaStream_t)stream);
 }
 
 int dsq_conv2d(const void *act_codes, const dsq_nhwc_t *shape, const dsq_quant_t *act_q,
@@ -1106,9 +1161,9 @@ int dsq_conv2d(const void *act_codes, const dsq_nhwc_t *shape, const dsq_quant_t
     p.m_tiles = (int)((M + BM - 1) / BM);
     p.BN = pick_bn(p.m_tiles, conv->Cout, bits);
     p.n_tiles = (conv->Cout + p.BN - 1) / p.BN;
-    p.s_p = 3;
-    const int ks = pick_ks(p, bits);
-    choose_b_mode(&p, bits, ks);
+    const int pm = pick_pm(p, bits);
+    const int ks = pm == 1 ? 1 : 2;
+    choose_b_mode(&p, bits, pm);
     p.act = (const uint8_t *)act_codes;
     p.H = shape->H; p.W = shape->W; p.Ho = Ho; p.Wo = Wo;
     p.stride = conv->stride; p.pad = conv->pad; p.KW = conv->KW; p.taps = taps; p.P = (int)P;
@@ -1133,7 +1188,7 @@ int dsq_conv2d(const void *act_codes, const dsq_nhwc_t *shape, const dsq_quant_t
                           (2.0 * (double)(1 << (bits - 1)) + 1.0) < 4194304.0;
     const int epi = (y_f32 || acc_out || !y_codes) ? EPI_GENERAL
                     : (e.residual ? EPI_CODES_RES : EPI_CODES);
-    return dispatch_tc(bits, epi, ks, tmap, p, (cudaStream_t)stream);
+    return dispatch_tc(bits, epi, pm, tmap, p, (cudaStream_t)stream);
 }
 
 int dsq_probe_i8_mma_rate(int iters, float *ms_out, double *macs_out, void *workspace,
