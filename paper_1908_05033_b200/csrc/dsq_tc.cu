@@ -495,14 +495,16 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
     } else if (warp < WARP_E0) {
         // ---------------- B: expand packed shared tiles ---------------------
         const int tid = threadIdx.x - WARP_B0 * 32;
-        // a packed row of the round holds CHK = KS*CH chunks; chunk c = tid +
-        // NUM_B_THREADS*i -> row = c / CHK, K step h = (c % CHK) / CH, chunk j =
-        // c % CH; the swizzle term (row & 7) does not depend on i
+        // a packed row of the round holds CHK = KS*CH chunks.  Thread (row0, j)
+        // owns chunk j of every K step of rows row0 + i*ROWS_PER_IT: the eight
+        // lanes of a 128-bit store phase then cover two rows x four chunks of
+        // one K step, i.e. eight different 16-byte bank groups of the swizzled
+        // tile (lanes split over two K steps would collide pairwise, the K steps
+        // being a multiple of 128 bytes apart); (row & 7) does not depend on i
         constexpr int CHK = KS * CH;
-        constexpr int ROWS_PER_IT = (BITS == 3) ? NUM_B_THREADS : NUM_B_THREADS / CHK;
-        constexpr int MAX_IT = (BITS == 3) ? 1 : (WIDE ? 2 : 1) * (256 * CH) / NUM_B_THREADS;
-        const int row0 = (BITS == 3) ? tid : tid / CHK;
-        const int h = (BITS == 3) ? 0 : (tid % CHK) / CH;
+        constexpr int ROWS_PER_IT = (BITS == 3) ? NUM_B_THREADS : NUM_B_THREADS / CH;
+        constexpr int MAX_IT = (BITS == 3) ? 1 : (256 * CH) / NUM_B_THREADS;
+        const int row0 = (BITS == 3) ? tid : tid / CH;
         const int j = (BITS == 3) ? 0 : tid % CH;
         const int sw = row0 & 7;
         const int n_it = (BN + ROWS_PER_IT - 1) / ROWS_PER_IT;
@@ -539,26 +541,33 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
                     }
                 } else {
                     constexpr int OUT = Chunks<BITS>::OUT;
-                    uint4 v[MAX_IT];
+                    uint4 v[MAX_IT][KS];
 #pragma unroll
                     for (int i = 0; i < MAX_IT; ++i)
-                        if (i < n_it && row0 + i * ROWS_PER_IT < BN)
-                            v[i] = reinterpret_cast<const uint4 *>(src)[tid + i * NUM_B_THREADS];
+                        if (i < n_it && row0 + i * ROWS_PER_IT < BN) {
+#pragma unroll
+                            for (int h = 0; h < KS; ++h)
+                                v[i][h] = reinterpret_cast<const uint4 *>(
+                                    src)[(row0 + i * ROWS_PER_IT) * CHK + h * CH + j];
+                        }
                     if (!p.b_res && !(ok = wait_bar(bar_u_empty(su), phu ^ 1u, ctl, 7))) break;
-                    uint8_t *rowp = dst + h * b_sub_bytes + row0 * BK_BYTES;
+                    uint8_t *rowp = dst + row0 * BK_BYTES;
 #pragma unroll
                     for (int i = 0; i < MAX_IT; ++i) {
                         if (i < n_it && row0 + i * ROWS_PER_IT < BN) {
 #pragma unroll
-                            for (int c = 0; c < OUT; ++c) {
-                                const uint4 o = make_uint4(
-                                    expand_word<BITS, B_SIGNED>(v[i].x, c, p.orv),
-                                    expand_word<BITS, B_SIGNED>(v[i].y, c, p.orv),
-                                    expand_word<BITS, B_SIGNED>(v[i].z, c, p.orv),
-                                    expand_word<BITS, B_SIGNED>(v[i].w, c, p.orv));
-                                *reinterpret_cast<uint4 *>(rowp + i * ROWS_PER_IT * BK_BYTES +
-                                                           (((j * OUT + c) ^ sw) << 4)) = o;
-                            }
+                            for (int h = 0; h < KS; ++h)
+#pragma unroll
+                                for (int c = 0; c < OUT; ++c) {
+                                    const uint4 o = make_uint4(
+                                        expand_word<BITS, B_SIGNED>(v[i][h].x, c, p.orv),
+                                        expand_word<BITS, B_SIGNED>(v[i][h].y, c, p.orv),
+                                        expand_word<BITS, B_SIGNED>(v[i][h].z, c, p.orv),
+                                        expand_word<BITS, B_SIGNED>(v[i][h].w, c, p.orv));
+                                    *reinterpret_cast<uint4 *>(
+                                        rowp + h * b_sub_bytes + i * ROWS_PER_IT * BK_BYTES +
+                                        (((j * OUT + c) ^ sw) << 4)) = o;
+                                }
                         }
                     }
                 }
