@@ -79,7 +79,14 @@ __device__ __forceinline__ uint4 lds_128(uint32_t addr)
                  : "memory");
     return v;
 }
-
+// 256-bit global store (one full 32-byte sector per lane); dst 32-byte aligned
+__device__ __forceinline__ void stg_256(void *dst, uint32_t a, uint32_t b, uint32_t c, uint32_t d,
+                                        uint32_t e, uint32_t f, uint32_t g, uint32_t h)
+{
+    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst), "r"(a),
+                 "r"(b), "r"(c), "r"(d), "r"(e), "r"(f), "r"(g), "r"(h)
+                 : "memory");
+}
 
 // ---- proxy / tcgen05 fences ------------------------------------------------
 // Make generic-proxy shared-memory writes visible to the async proxy (TMA,

@@ -648,7 +648,14 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
                     if (n0 >= p.Ncols) continue;
                     if (p.C_i32) {
                         int32_t *dst = p.C_i32 + m * p.Ncols + n0;
-                        if (full) {
+                        if (full && (reinterpret_cast<uintptr_t>(dst) & 31u) == 0) {
+                            // one full 32-byte sector per lane and store
+#pragma unroll
+                            for (int v = 0; v < 4; ++v)
+                                stg_256(dst + 8 * v, r[8 * v], r[8 * v + 1], r[8 * v + 2],
+                                        r[8 * v + 3], r[8 * v + 4], r[8 * v + 5], r[8 * v + 6],
+                                        r[8 * v + 7]);
+                        } else if (full) {
 #pragma unroll
                             for (int v = 0; v < 8; ++v)
                                 reinterpret_cast<int4 *>(dst)[v] =
@@ -662,7 +669,18 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
                     }
                     if (p.D_f32) {
                         float *dst = p.D_f32 + m * p.Ncols + n0;
-                        if (full) {
+                        if (full && (reinterpret_cast<uintptr_t>(dst) & 31u) == 0) {
+#pragma unroll
+                            for (int v = 0; v < 4; ++v) {
+                                uint32_t f[8];
+#pragma unroll
+                                for (int u = 0; u < 8; ++u)
+                                    f[u] = __float_as_uint(
+                                        __fmul_rn((float)(int)r[8 * v + u], rs));
+                                stg_256(dst + 8 * v, f[0], f[1], f[2], f[3], f[4], f[5], f[6],
+                                        f[7]);
+                            }
+                        } else if (full) {
 #pragma unroll
                             for (int v = 0; v < 8; ++v)
                                 reinterpret_cast<float4 *>(dst)[v] =
