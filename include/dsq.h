@@ -271,6 +271,13 @@ int dsq_set_tile_n(int bn);
  * the N tile is at most 128 wide).  Results do not depend on it. */
 int dsq_set_round_k_steps(int ks);
 
+/* Third tuning hook: CTA pairs.  With 256-wide N tiles the tensor-core
+ * kernels run as clusters of two CTAs that share one 256 x 256 tile
+ * (tcgen05 cta_group::2; each SM expands half of the B operand).  mode 0:
+ * automatic, 1: never, 2: wherever the shapes allow.  Results do not depend
+ * on it. */
+int dsq_set_cta_pairs(int mode);
+
 /* ---- misc --------------------------------------------------------------- */
 const char *dsq_status_string(int status);
 int dsq_version(void);

@@ -76,6 +76,7 @@ _SIGNATURES = {
                                      C.POINTER(C.c_double), _vp, _sz, _vp]),
     "dsq_set_tile_n": (_int, [_int]),
     "dsq_set_round_k_steps": (_int, [_int]),
+    "dsq_set_cta_pairs": (_int, [_int]),
     "dsq_status_string": (C.c_char_p, [_int]),
     "dsq_version": (_int, []),
 }
@@ -320,6 +321,10 @@ def dsq_gemm(A, B, M, N, K, bits, ws, row_scale=None, want_i32=True,
 
 def dsq_set_round_k_steps(ks):
     _check(lib.dsq_set_round_k_steps(ks), "dsq_set_round_k_steps")
+
+
+def dsq_set_cta_pairs(mode):
+    _check(lib.dsq_set_cta_pairs(mode), "dsq_set_cta_pairs")
 
 
 def dsq_set_tile_n(bn):

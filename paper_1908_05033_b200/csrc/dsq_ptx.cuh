@@ -54,6 +54,37 @@ __device__ __forceinline__ uint64_t global_timer_ns()
     return t;
 }
 
+// ---- thread-block clusters (CTA pairs) ---------------------------------------
+__device__ __forceinline__ uint32_t cluster_ctarank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// Barrier over all threads of all CTAs of the cluster (every thread calls it).
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\t"
+                 "barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// Address of this CTA's shared-memory location `addr` as seen in CTA `rank` of
+// the cluster (shared::cluster window).
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+// Arrive on an mbarrier of any CTA of the cluster (shared::cluster address).
+// Default semantics (release at CTA scope): what the arriving thread wrote to
+// its own shared / tensor memory is complete before the arrival is seen, which
+// is all the peer's MMA thread needs before it lets the tensor core read that
+// memory.  (A cluster-scope release costs over a thousand cycles per arrival.)
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
+{
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+
 // ---- cp.async (16-byte, L2 only); src_bytes = 0 writes zeros -----------------
 __device__ __forceinline__ void cp_async_16(uint32_t dst, const void *src, uint32_t src_bytes)
 {
@@ -122,24 +153,43 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *m,
 }
 
 // ---- tensor memory ---------------------------------------------------------
-// Executed by one full warp.  ncols: power of two, 32..512.
+// Executed by one full warp.  ncols: power of two, 32..512.  CG = 2: the
+// same warp of both CTAs of a pair executes it, and both get the same columns.
+template <int CG = 1>
 __device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols)
 {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
-                     dst_smem),
-                 "r"(ncols)
-                 : "memory");
-}
-__device__ __forceinline__ void tmem_relinquish()
-{
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::
+    if (CG == 1)
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                         dst_smem),
+                     "r"(ncols)
+                     : "memory");
+    else
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                         dst_smem),
+                     "r"(ncols)
                      : "memory");
 }
+template <int CG = 1>
+__device__ __forceinline__ void tmem_relinquish()
+{
+    if (CG == 1)
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::
+                         : "memory");
+    else
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::
+                         : "memory");
+}
+template <int CG = 1>
 __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols)
 {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr),
-                 "r"(ncols)
-                 : "memory");
+    if (CG == 1)
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr),
+                     "r"(ncols)
+                     : "memory");
+    else
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr),
+                     "r"(ncols)
+                     : "memory");
 }
 
 // ---- tcgen05.mma kind::i8 --------------------------------------------------
@@ -158,11 +208,31 @@ __device__ __forceinline__ void mma_i8(uint32_t d_tmem, uint64_t a_desc,
 }
 // Arrive on an mbarrier once all previously issued tcgen05.mma of this thread
 // have completed (implies tcgen05.fence::before_thread_sync).
+// CG = 2: tracks the pair's instructions; `bar` may be a shared::cluster
+// address of either CTA.
+template <int CG = 1>
 __device__ __forceinline__ void mma_commit(uint32_t bar)
 {
+    if (CG == 1)
+        asm volatile(
+            "tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(
+                bar)
+            : "memory");
+    else
+        asm volatile(
+            "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(
+                bar)
+            : "memory");
+}
+
+// Same for a CTA pair: one instruction signals the barrier at this shared-memory
+// offset in every CTA of `cta_mask` (bit r = CTA rank r of the cluster).
+__device__ __forceinline__ void mma_commit_pair(uint32_t bar, uint16_t cta_mask)
+{
     asm volatile(
-        "tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(
-            bar)
+        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 "
+        "[%0], %1;" ::"r"(bar),
+        "h"(cta_mask)
         : "memory");
 }
 
@@ -184,10 +254,12 @@ __device__ __forceinline__ void mma_i8_ts(uint32_t d_tmem, uint32_t a_tmem,
 // A advances 8 tensor-memory columns and the B descriptor 32 bytes (2 units of
 // 16 bytes in its low word) per instruction.  Only the first one takes the
 // caller's accumulate flag.  Keeps the issuing thread's instruction count low.
+template <int CG = 1>
 __device__ __forceinline__ void mma_i8_ts_x4(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_desc_lo,
                                              uint32_t b_desc_hi, uint32_t idesc,
                                              uint32_t accumulate_first)
 {
+    if (CG == 1) {
     asm volatile(
         "{\n\t.reg .pred p0, p1;\n\t.reg .b64 d0, d1, d2, d3;\n\t"
         ".reg .b32 l1, l2, l3, a1, a2, a3;\n\t"
@@ -202,6 +274,22 @@ __device__ __forceinline__ void mma_i8_ts_x4(uint32_t d_tmem, uint32_t a_tmem, u
         "tcgen05.mma.cta_group::1.kind::i8 [%0], [a3], d3, %4, p1;\n\t}" ::"r"(d_tmem),
         "r"(a_tmem), "r"(b_desc_lo), "r"(b_desc_hi), "r"(idesc), "r"(accumulate_first)
         : "memory");
+    } else {
+    asm volatile(
+        "{\n\t.reg .pred p0, p1;\n\t.reg .b64 d0, d1, d2, d3;\n\t"
+        ".reg .b32 l1, l2, l3, a1, a2, a3;\n\t"
+        "setp.ne.b32 p0, %5, 0;\n\tsetp.eq.b32 p1, %5, %5;\n\t"
+        "add.u32 l1, %2, 2;\n\tadd.u32 l2, %2, 4;\n\tadd.u32 l3, %2, 6;\n\t"
+        "add.u32 a1, %1, 8;\n\tadd.u32 a2, %1, 16;\n\tadd.u32 a3, %1, 24;\n\t"
+        "mov.b64 d0, {%2, %3};\n\tmov.b64 d1, {l1, %3};\n\t"
+        "mov.b64 d2, {l2, %3};\n\tmov.b64 d3, {l3, %3};\n\t"
+        "tcgen05.mma.cta_group::2.kind::i8 [%0], [%1], d0, %4, p0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::i8 [%0], [a1], d1, %4, p1;\n\t"
+        "tcgen05.mma.cta_group::2.kind::i8 [%0], [a2], d2, %4, p1;\n\t"
+        "tcgen05.mma.cta_group::2.kind::i8 [%0], [a3], d3, %4, p1;\n\t}" ::"r"(d_tmem),
+        "r"(a_tmem), "r"(b_desc_lo), "r"(b_desc_hi), "r"(idesc), "r"(accumulate_first)
+        : "memory");
+    }
 }
 
 // 32 lanes x 32 columns store: thread t of the warp writes lane (base + t),
@@ -274,14 +362,14 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t smem_addr)
 }
 
 // Instruction descriptor for kind::i8: s32 accumulator, K-major A and B.
-__host__ __device__ inline uint32_t idesc_i8(int n, bool a_signed, bool b_signed)
+__host__ __device__ inline uint32_t idesc_i8(int n, bool a_signed, bool b_signed, int m = 128)
 {
     uint32_t d = 0;
     d |= 2u << 4;                              // D format: S32
     d |= (a_signed ? 1u : 0u) << 7;            // A: 0 = u8, 1 = s8
     d |= (b_signed ? 1u : 0u) << 10;           // B
     d |= (uint32_t)(n >> 3) << 17;             // N / 8
-    d |= (uint32_t)(128 >> 4) << 24;           // M / 16
+    d |= (uint32_t)(m >> 4) << 24;             // M / 16 (256: both CTAs of a pair)
     return d;
 }
 

@@ -59,16 +59,28 @@ constexpr int BK_BYTES = 128;         // int8 bytes per row per K step (128 code
 //   PM 3: KS = 2, 2 stages, one A group ("wide")  (N tile 192 / 256: shared memory
 //         holds two double stages of B only; the second A group's warps help
 //         the epilogue instead)
+//   PM 4: KS = 2, 3 stages, two A groups, CTA PAIR: the two CTAs of a cluster
+//         work on one 256 x 256 tile with tcgen05.mma.cta_group::2.  Each CTA
+//         gathers and expands its 128 A rows and HALF of the B rows (128 output
+//         channels), the even CTA issues the instructions for both, and each
+//         keeps the accumulators of its own 128 rows.  Per tensor-core clock
+//         every SM then expands half as much B, which is what bounds the
+//         single-CTA modes at wide N tiles.
 constexpr int SU_MAX = 4;
 template <int PM> struct Pipe {
     static constexpr int KS = PM == 1 ? 1 : 2;
     static constexpr bool WIDE = PM == 3;
-    static constexpr int SU = PM == 1 ? 4 : PM == 2 ? 3 : 2;   // stages of expanded operands
+    static constexpr bool PAIR = PM == 4;
+    static constexpr int SU = PM == 1 ? 4 : PM == 3 ? 2 : 3;   // stages of expanded operands
     static constexpr int GROUPS = WIDE ? 1 : 2;              // A groups in use
     static constexpr int A_D = PM == 1 ? 2 : 1;              // own A rounds in flight per thread
     static constexpr int A_RING = A_D + 1;                   // packed A ring slots per group
     static constexpr int A_COL0 = 512 - SU * 32 * KS;        // A stages: top TMEM columns
     static constexpr int S_P = WIDE ? 2 : 3;                 // packed B ring slots
+    // coalesced A gather (adjacent lanes fetch one row's contiguous chunks): fewer
+    // memory requests, more instructions in the A threads; pays where the A
+    // threads have slack
+    static constexpr bool COAL = PAIR;
 };
 constexpr int TMEM_COLS = 512;
 
@@ -99,6 +111,7 @@ struct TcParams {
     // A gather geometry (a GEMM is a 1x1 convolution over an M x 1 image)
     const uint8_t *act;
     int H, W, Ho, Wo, stride, pad, KW, taps, P;
+    int a_lcr;                        // log2 of the A gather's run length in 16-byte chunks
     // epilogue
     int mode, shift, out_pitch, small_acc;
     DsqEpi e;
@@ -248,31 +261,39 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
     constexpr bool B_SIGNED = !A_SIGNED;
     constexpr int CH = Chunks<BITS>::CH;
     constexpr int KS = Pipe<PM>::KS, GROUPS = Pipe<PM>::GROUPS;
-    constexpr bool WIDE = Pipe<PM>::WIDE;
+    constexpr bool WIDE = Pipe<PM>::WIDE, PAIR = Pipe<PM>::PAIR;
+    constexpr int CG = PAIR ? 2 : 1;          // CTAs per tcgen05 instruction
+    constexpr int BMT = BM * CG;              // tile rows
     constexpr int S_U = Pipe<PM>::SU, A_D = Pipe<PM>::A_D, A_RING = Pipe<PM>::A_RING;
     constexpr int A_COL0 = Pipe<PM>::A_COL0;
     static_assert(KS == 1 || BITS != 3, "3-bit rows use single K steps");
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>(
         (reinterpret_cast<uintptr_t>(smem_raw) + 1023u) & ~(uintptr_t)1023u);
+    const int BN = p.BN;
+    const int BNL = BN / CG;                  // B rows this CTA expands
     const SmemLayout L =
-        smem_layout(p.BN, BITS, p.s_p, p.b_stages, KS, GROUPS * A_RING, p.epw);
+        smem_layout(BNL, BITS, p.s_p, p.b_stages, KS, GROUPS * A_RING, p.epw);
     // the layout must fit behind the 1024-byte aligned base (the host adds
     // slack only while it stays within the 227 KB limit); same answer in every
-    // thread, taken before any barrier exists
+    // thread of every CTA, taken before any barrier exists
     if ((uint32_t)(smem - smem_raw) + L.total > (uint32_t)p.smem_bytes) {
         if (threadIdx.x == 0) atomicCAS(p.ws + DSQ_WS_STATUS, 0, (int)DSQ_ERR_UNSUPPORTED);
         return;
     }
     const int S_P = p.s_p;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int BN = p.BN;
+    // a pair is the two CTAs of a cluster; rank 0 issues the MMAs
+    const uint32_t rank = PAIR ? cluster_ctarank() : 0u;
+    const int tile0 = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+    const int tstep = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
+    const int row_base = (int)rank * BM;      // first tile row of this CTA
     const int total_tiles = p.m_tiles * p.n_tiles;
-    const uint32_t b_sub_bytes = BN * BK_BYTES;              // one K step of the tile
+    const uint32_t b_sub_bytes = BNL * BK_BYTES;             // one K step of the (half) tile
     const uint32_t b_tile_bytes = KS * b_sub_bytes;          // one round
-    const uint32_t b_packed_bytes = KS * BN * 16 * BITS;
+    const uint32_t b_packed_bytes = KS * BNL * 16 * BITS;
     int my_tiles_all = 0;
-    for (int t = blockIdx.x; t < total_tiles; t += gridDim.x) ++my_tiles_all;
+    for (int t = tile0; t < total_tiles; t += tstep) ++my_tiles_all;
     // B is produced for every step of every tile, or once (resident mode)
     const uint32_t n_b_steps =
         my_tiles_all == 0 ? 0u : (p.b_res ? (uint32_t)p.rounds : (uint32_t)my_tiles_all * p.rounds);
@@ -288,31 +309,46 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
     auto bar_acc_empty = [&](int s) { return bars + 8u * (BAR_P + 2 * MAX_S_P + 2 + s); };
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + L.tmem_slot);
     Ctl ctl{reinterpret_cast<volatile int *>(smem + L.abort_flag), p.ws};
+    // The consumer of a_full / b_full / acc_empty is the MMA thread of rank 0:
+    // in a pair both CTAs arrive on rank 0's barriers.
+    auto arrive_leader = [&](uint32_t bar) {
+        if (PAIR) mbar_arrive_cluster(map_to_cta(bar, 0u));
+        else mbar_arrive(bar);
+    };
+    // completion of the issued MMAs, signalled to this barrier in both CTAs
+    auto commit_all = [&](uint32_t bar) {
+        if (PAIR) mma_commit_pair(bar, (uint16_t)3);
+        else mma_commit<1>(bar);
+    };
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S_U; ++s) {
-            mbar_init(bar_a_full(s), 4);     // the four warps of one A group
+            // operands of a round: the four warps of one A group and (unless the
+            // expanded B tile is resident) the B warps, of every CTA of the pair
+            mbar_init(bar_a_full(s), (4 + (p.b_res ? 0 : NUM_B_WARPS)) * CG);
             mbar_init(bar_u_empty(s), 1);    // tcgen05.commit
         }
-        for (int s = 0; s < MAX_B_STAGES; ++s) mbar_init(bar_b_full(s), NUM_B_WARPS);
+        for (int s = 0; s < MAX_B_STAGES; ++s) mbar_init(bar_b_full(s), NUM_B_WARPS * CG);
         for (int s = 0; s < S_P; ++s) {
             mbar_init(bar_p_full(s), 1);     // TMA producer (+ transaction bytes)
             mbar_init(bar_p_empty(s), NUM_B_WARPS);
         }
         for (int s = 0; s < 2; ++s) {
             mbar_init(bar_acc_full(s), 1);   // tcgen05.commit
-            mbar_init(bar_acc_empty(s), 4 * p.epw);
+            mbar_init(bar_acc_empty(s), 4 * p.epw * CG);
         }
         *ctl.abort_flag = 0;
         mbar_init_fence();
     }
     if (warp == WARP_MMA) {
-        tmem_alloc(smem_u32((const void *)tmem_slot), TMEM_COLS);
-        tmem_relinquish();
+        tmem_alloc<CG>(smem_u32((const void *)tmem_slot), TMEM_COLS);
+        tmem_relinquish<CG>();
     }
     if (warp == WARP_TMA && lane == 0) tma_prefetch_desc(&tmap_b);
     tc_fence_before_sync();
     __syncthreads();
+    // no arrival may reach the peer before its barriers exist
+    if (PAIR) cluster_sync_all();
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
 
@@ -321,15 +357,16 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
         // ---------------- B producer: TMA packed tiles --------------------
         if (lane == 0) {
             uint32_t g = 0, ph = 0;
-            int s = 0, ks = 0, tile = blockIdx.x;
+            int s = 0, ks = 0, tile = tile0;
 #pragma unroll 1
             for (; g < n_b_steps; ++g) {
                 if (!wait_bar(bar_p_empty(s), ph ^ 1u, ctl, 1)) break;
                 mbar_arrive_expect_tx(bar_p_full(s), b_packed_bytes);
                 tma_load_2d(smem_u32(smem + L.b_packed + s * b_packed_bytes), &tmap_b,
-                            ks * (KS * 16 * BITS), (tile % p.n_tiles) * BN, bar_p_full(s));
+                            ks * (KS * 16 * BITS), (tile % p.n_tiles) * BN + (int)rank * BNL,
+                            bar_p_full(s));
                 if (++s == S_P) { s = 0; ph ^= 1u; }
-                if (++ks == p.rounds) { ks = 0; tile += gridDim.x; }
+                if (++ks == p.rounds) { ks = 0; tile += tstep; }
             }
             // let outstanding copies land before the CTA can exit
             const uint32_t issued = g;
@@ -338,14 +375,14 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
         }
     } else if (warp == WARP_MMA) {
         // ---------------- MMA issuer ---------------------------------------
-        if (lane == 0) {
-            const uint32_t idesc = idesc_i8(BN, A_SIGNED, B_SIGNED);
+        if (lane == 0 && rank == 0) {
+            const uint32_t idesc = idesc_i8(BN, A_SIGNED, B_SIGNED, BMT);
             const uint64_t b_desc0 = smem_desc_sw128(smem_u32(smem + L.b_tiles));
             const uint32_t b_desc_lo0 = (uint32_t)b_desc0, b_desc_hi = (uint32_t)(b_desc0 >> 32);
             uint32_t g = 0, it = 0;
             bool ok = true;
 #pragma unroll 1
-            for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++it) {
+            for (int tile = tile0; ok && tile < total_tiles; tile += tstep, ++it) {
                 const int as = p.n_acc == 2 ? (it & 1) : 0;
                 const uint32_t aph = (p.n_acc == 2 ? (it >> 1) : it) & 1u;
                 if (!(ok = wait_bar(bar_acc_empty(as), aph ^ 1u, ctl, 3))) break;
@@ -356,19 +393,21 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
                     const int s = g % S_U;
                     const uint32_t ph = (g / S_U) & 1u;
                     const int bs = p.b_res ? ks : s;
-                    if (!p.b_res || it == 0)
-                        if (!(ok = wait_bar(bar_b_full(bs), p.b_res ? 0u : ph, ctl, 10))) break;
-                    if (!(ok = wait_bar(bar_a_full(s), ph, ctl, 4))) break;
+                    if (p.b_res && it == 0)
+                        if (!(ok = wait_bar(bar_b_full(bs), 0u, ctl, 10))) break;
+                    // common case without the call: the operands are there already
+                    if (!mbar_try_wait(bar_a_full(s), ph))
+                        if (!(ok = wait_bar(bar_a_full(s), ph, ctl, 4))) break;
                     tc_fence_after_sync();
                     // per K step 4 instructions, 32 bytes of K each
 #pragma unroll
                     for (int h = 0; h < KS; ++h)
-                        mma_i8_ts_x4(d_tmem, tmem_base + A_COL0 + (s * KS + h) * 32,
+                        mma_i8_ts_x4<CG>(d_tmem, tmem_base + A_COL0 + (s * KS + h) * 32,
                                      b_desc_lo0 + (bs * KS + h) * (b_sub_bytes >> 4), b_desc_hi,
                                      idesc, (uint32_t)(ks | h));
-                    mma_commit(bar_u_empty(s));
+                    commit_all(bar_u_empty(s));
                 }
-                if (ok) mma_commit(bar_acc_full(as));
+                if (ok) commit_all(bar_acc_full(as));
             }
         }
     } else if (warp < WARP_B0) {
@@ -376,9 +415,16 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
         // Group k (four warps, one per TMEM lane quarter) handles the K steps with
         // step index = k (mod 2), so two steps are in flight at once and the
         // per-step latency chain of one group overlaps the other's.  Per step:
-        // global --cp.async--> private 16-byte cells of a shared ring (A_D own
-        // steps in flight, thread-local completion) -> registers -> expand ->
-        // tensor memory (tcgen05.st), completed and published at once.
+        // global --cp.async--> 16-byte cells of a shared ring (A_D own steps in
+        // flight) -> registers -> expand -> tensor memory (tcgen05.st),
+        // completed and published at once.
+        //
+        // The copies are issued coalesced: a row's codes of one filter tap are
+        // contiguous, so a run of 2^a_lcr chunks is fetched by that many adjacent
+        // lanes (the row's owner hands the run's address over by shuffle), and a
+        // warp instruction covers a few rows x up to 128 contiguous bytes instead
+        // of 32 rows x 16 bytes: an eighth of the L1 requests and of the
+        // shared-memory write cycles.  Each thread then reads its own row.
         const int group = (warp - WARP_A0) >> 2;
         if (group < GROUPS) {
         const int quarter = warp & 3;              // TMEM lane quarter of this warp
@@ -388,8 +434,12 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
             smem_u32(smem + L.a_ring) + group * (A_RING * SLOT_BYTES) + row * 16;
         // walk position over the flattened (tile, K step) sequence; starts one
         // tile back with ld_ks at its end, so that the first step advances
-        int ld_tile = (int)blockIdx.x - (int)gridDim.x, ld_ks = p.rounds, ld_slot = 0;
+        int ld_tile = tile0 - tstep, ld_ks = p.rounds, ld_slot = 0;
         int tap = 0, kw = 0, off = 0;
+        const int lcr = p.a_lcr, crm = (1 << lcr) - 1;
+        const int lane_row = lane >> lcr, lane_c = lane & crm;
+        const uint32_t ring0 = smem_u32(smem + L.a_ring) + group * (A_RING * SLOT_BYTES) +
+                               quarter * (32 * 16);
         uint32_t tap_mask = 0;                     // bit t: filter tap t is inside the image
         const uint8_t *src = p.act;
         const int64_t row_jump = (int64_t)(p.W - p.KW) * p.P;
@@ -397,7 +447,7 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
             tap = kw = off = 0;
             tap_mask = 0;
             if (t >= total_tiles) return;
-            const int m = (t / p.n_tiles) * BM + row;
+            const int m = (t / p.n_tiles) * BMT + row_base + row;
             if (m < p.M) {
                 const int wo = m % p.Wo;
                 const int ho = (m / p.Wo) % p.Ho;
@@ -415,23 +465,53 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
         auto walk_step = [&](bool load) {
             if (ld_ks == p.rounds) {
                 ld_ks = 0;
-                ld_tile += gridDim.x;
+                ld_tile += tstep;
                 set_tile(ld_tile);
             }
             if (ld_tile < total_tiles) {
-                const uint32_t dst = cell0 + ld_slot * SLOT_BYTES;
+                const uint32_t dst = ring0 + ld_slot * SLOT_BYTES;
+                unsigned long long run = 0ull;     // this row's current run (0: zero fill)
+                if (!Pipe<PM>::COAL) {
+                    // every thread fetches its own row, chunk by chunk
+#pragma unroll
+                    for (int j = 0; j < KS * CH; ++j) {
+                        if (load) {
+                            const bool ok = tap < 32 && ((tap_mask >> tap) & 1u);
+                            cp_async_16(dst + lane * 16 + j * (BM * 16), ok ? src : p.act,
+                                        ok ? 16u : 0u);
+                        }
+                        off += 16;
+                        src += 16;
+                        if (off == p.P) {
+                            off = 0;
+                            ++tap;
+                            if (++kw == p.KW) { kw = 0; src += row_jump; }
+                        }
+                    }
+                } else
 #pragma unroll
                 for (int j = 0; j < KS * CH; ++j) {
-                    if (load) {
+                    if ((j & crm) == 0) {          // a new run of 2^lcr chunks starts
                         const bool ok = tap < 32 && ((tap_mask >> tap) & 1u);
-                        cp_async_16(dst + j * (BM * 16), ok ? src : p.act, ok ? 16u : 0u);
+                        run = ok ? (unsigned long long)reinterpret_cast<uintptr_t>(src) : 0ull;
+                        off += 16 << lcr;
+                        src += 16 << lcr;
+                        if (off == p.P) {
+                            off = 0;
+                            ++tap;
+                            if (++kw == p.KW) { kw = 0; src += row_jump; }
+                        }
                     }
-                    off += 16;
-                    src += 16;
-                    if (off == p.P) {
-                        off = 0;
-                        ++tap;
-                        if (++kw == p.KW) { kw = 0; src += row_jump; }
+                    if (load) {
+                        // lane -> (row of this warp, chunk of the run)
+                        const int rsel = ((j & crm) << (5 - lcr)) + lane_row;
+                        const unsigned long long ptr = __shfl_sync(0xffffffffu, run, rsel);
+                        const int cj = (j & ~crm) + lane_c;
+                        cp_async_16(dst + cj * (BM * 16) + rsel * 16,
+                                    ptr ? reinterpret_cast<const uint8_t *>((uintptr_t)ptr) +
+                                              16 * lane_c
+                                        : p.act,
+                                    ptr ? 16u : 0u);
                     }
                 }
                 ++ld_ks;
@@ -448,7 +528,7 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
             tmem_st_wait();
             tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar_a_full(pend_s));
+            if (lane == 0) arrive_leader(bar_a_full(pend_s));
             pend_s = -1;
         };
         if (GROUPS == 2 && group == 1) walk_step(false);   // step 0 belongs to group 0
@@ -461,6 +541,7 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
             if (i < (uint32_t)A_D) continue;
             const uint32_t g = GROUPS * (i - A_D) + group;
             cp_async_wait<A_D>();                  // own step i - A_D has landed
+            if (Pipe<PM>::COAL) __syncwarp();      // ... the other lanes' copies of my row too
             const int s = g % S_U;
             const uint32_t ph = (g / S_U) & 1u;
 #pragma unroll
@@ -507,7 +588,7 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
         const int row0 = (BITS == 3) ? tid : tid / CH;
         const int j = (BITS == 3) ? 0 : tid % CH;
         const int sw = row0 & 7;
-        const int n_it = (BN + ROWS_PER_IT - 1) / ROWS_PER_IT;
+        const int n_it = (BNL + ROWS_PER_IT - 1) / ROWS_PER_IT;
         uint32_t php = 0;
         int sp = -1;
         bool ok = true;
@@ -522,7 +603,7 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
                 uint8_t *dst = smem + L.b_tiles + su * b_tile_bytes;
                 if (BITS == 3) {
                     uint32_t w[12];
-                    if (row0 < BN) {
+                    if (row0 < BNL) {
                         const uint4 *r4 = reinterpret_cast<const uint4 *>(src + row0 * 48);
 #pragma unroll
                         for (int l = 0; l < 3; ++l) {
@@ -532,7 +613,7 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
                         }
                     }
                     if (!p.b_res && !(ok = wait_bar(bar_u_empty(su), phu ^ 1u, ctl, 7))) break;
-                    if (row0 < BN) {
+                    if (row0 < BNL) {
                         uint8_t *rowp = dst + row0 * BK_BYTES;
 #pragma unroll
                         for (int q = 0; q < 8; ++q)
@@ -544,7 +625,7 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
                     uint4 v[MAX_IT][KS];
 #pragma unroll
                     for (int i = 0; i < MAX_IT; ++i)
-                        if (i < n_it && row0 + i * ROWS_PER_IT < BN) {
+                        if (i < n_it && row0 + i * ROWS_PER_IT < BNL) {
 #pragma unroll
                             for (int h = 0; h < KS; ++h)
                                 v[i][h] = reinterpret_cast<const uint4 *>(
@@ -554,7 +635,7 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
                     uint8_t *rowp = dst + row0 * BK_BYTES;
 #pragma unroll
                     for (int i = 0; i < MAX_IT; ++i) {
-                        if (i < n_it && row0 + i * ROWS_PER_IT < BN) {
+                        if (i < n_it && row0 + i * ROWS_PER_IT < BNL) {
 #pragma unroll
                             for (int h = 0; h < KS; ++h)
 #pragma unroll
@@ -574,7 +655,7 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
                 fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0) {
-                    mbar_arrive(bar_b_full(su));
+                    arrive_leader(p.b_res ? bar_b_full(su) : bar_a_full(su));
                     mbar_arrive(bar_p_empty(sp));
                 }
             }
@@ -600,11 +681,11 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
         uint32_t it = 0;
         bool ok = true;
 #pragma unroll 1
-        for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++it) {
+        for (int tile = tile0; ok && tile < total_tiles; tile += tstep, ++it) {
             const int as = p.n_acc == 2 ? (it & 1) : 0;
             const uint32_t aph = (p.n_acc == 2 ? (it >> 1) : it) & 1u;
             const int m_tile = tile / p.n_tiles, n_tile = tile % p.n_tiles;
-            const int64_t m = (int64_t)m_tile * BM + row_in_tile;
+            const int64_t m = (int64_t)m_tile * BMT + row_base + row_in_tile;
             const bool row_ok = m < p.M;
             if (!(ok = wait_bar(bar_acc_full(as), aph, ctl, 8))) break;
             tc_fence_after_sync();
@@ -842,17 +923,20 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
             }
             tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar_acc_empty(as));
+            if (lane == 0) arrive_leader(bar_acc_empty(as));
         }
     }
 
     // ---------------- teardown ---------------------------------------------
     tc_fence_before_sync();
     __syncthreads();
+    // a CTA of a pair stays until its peer has stopped signalling its barriers
+    // and reading operands from its shared and tensor memory
+    if (PAIR) cluster_sync_all();
     if (warp == WARP_MMA) {
         __syncwarp();
         tc_fence_after_sync();
-        tmem_dealloc(tmem_base, TMEM_COLS);
+        tmem_dealloc<CG>(tmem_base, TMEM_COLS);
     }
 }
 
@@ -960,10 +1044,11 @@ int make_rows_tmap(CUtensorMap *map, const void *base, uint64_t row_bytes, uint6
 // Resident B: one N tile and few K steps, so the expanded B tile of every K
 // step fits in shared memory next to the rings; it is then expanded once per
 // CTA instead of once per M tile.
-struct PipeInfo { int ks, su, a_slots, a_col0, s_p, wide; };
+struct PipeInfo { int ks, su, a_slots, a_col0, s_p, wide, pair; };
 PipeInfo pipe_info(int pm)
 {
     switch (pm) {
+    case 4: return {Pipe<4>::KS, Pipe<4>::SU, Pipe<4>::GROUPS * Pipe<4>::A_RING, Pipe<4>::A_COL0, Pipe<4>::S_P, 0, 1};
     case 1: return {Pipe<1>::KS, Pipe<1>::SU, Pipe<1>::GROUPS * Pipe<1>::A_RING, Pipe<1>::A_COL0, Pipe<1>::S_P, 0};
     case 2: return {Pipe<2>::KS, Pipe<2>::SU, Pipe<2>::GROUPS * Pipe<2>::A_RING, Pipe<2>::A_COL0, Pipe<2>::S_P, 0};
     default: return {Pipe<3>::KS, Pipe<3>::SU, Pipe<3>::GROUPS * Pipe<3>::A_RING, Pipe<3>::A_COL0, Pipe<3>::S_P, 1};
@@ -981,7 +1066,7 @@ void choose_b_mode(TcParams *p, int bits, int pm)
     p->b_res = 0;
     p->b_stages = pi.su;
     p->epw = pi.wide ? 2 : 1;
-    if (!pi.wide && p->n_tiles == 1 && p->rounds <= MAX_B_STAGES && p->m_tiles > 148) {
+    if (!pi.wide && !pi.pair && p->n_tiles == 1 && p->rounds <= MAX_B_STAGES && p->m_tiles > 148) {
         const SmemLayout L = smem_layout(p->BN, bits, p->s_p, p->rounds, pi.ks, pi.a_slots, 3);
         if (L.total + 1024 <= 227u * 1024u) {
             p->b_res = 1;
@@ -989,6 +1074,18 @@ void choose_b_mode(TcParams *p, int bits, int pm)
             p->epw = 3;
         }
     }
+}
+
+// Run length of the coalesced A gather: the largest power of two of 16-byte
+// chunks that divides both a pixel's packed row (so a run never straddles two
+// filter taps) and the chunks of a round.
+int a_run_log2(int P, int bits, int ks)
+{
+    if (bits == 3) return 0;
+    const int chk = ks * bits, q = P / 16;
+    int l = 0;
+    while (l < 3 && (2 << l) <= chk && q % (2 << l) == 0) ++l;
+    return l;
 }
 
 int g_forced_bn = 0;   // dsq_set_tile_n
@@ -1014,8 +1111,9 @@ int pick_bn(int m_tiles, int ncols, int bits)
 template <int BITS, bool A_SIGNED, int EPI, int PM>
 int launch_tc(const CUtensorMap &tmap, const TcParams &p, cudaStream_t s)
 {
-    const SmemLayout L = smem_layout(p.BN, BITS, p.s_p, p.b_stages, Pipe<PM>::KS,
-                                     Pipe<PM>::GROUPS * Pipe<PM>::A_RING, p.epw);
+    constexpr bool PAIR = Pipe<PM>::PAIR;
+    const SmemLayout L = smem_layout(PAIR ? p.BN / 2 : p.BN, BITS, p.s_p, p.b_stages,
+                                     Pipe<PM>::KS, Pipe<PM>::GROUPS * Pipe<PM>::A_RING, p.epw);
     if (L.total > 227u * 1024u) return DSQ_ERR_UNSUPPORTED;
     int smem_bytes = (int)L.total + 1024;            // slack for the 1024-byte alignment
     if (smem_bytes > 227 * 1024) smem_bytes = 227 * 1024;
@@ -1032,6 +1130,28 @@ int launch_tc(const CUtensorMap &tmap, const TcParams &p, cudaStream_t s)
     if (p.BN * p.n_acc > Pipe<PM>::A_COL0) return DSQ_ERR_UNSUPPORTED;
     TcParams q = p;
     q.smem_bytes = smem_bytes;
+    if (PAIR) {
+        // one cluster of two CTAs (the two SMs of a TPC) per tile in flight
+        if (grid > 74) grid = 74;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(2 * grid);
+        cfg.blockDim = dim3(NUM_THREADS);
+        cfg.dynamicSmemBytes = (size_t)smem_bytes;
+        cfg.stream = s;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        if (cudaLaunchKernelEx(&cfg, dsq_tc_kernel<BITS, A_SIGNED, EPI, PM>, tmap, q) !=
+            cudaSuccess) {
+            cudaGetLastError();
+            return DSQ_ERR_CUDA;
+        }
+        return dsq_launch_status();
+    }
     dsq_tc_kernel<BITS, A_SIGNED, EPI, PM><<<grid, NUM_THREADS, smem_bytes, s>>>(tmap, q);
     return dsq_launch_status();
 }
@@ -1050,10 +1170,12 @@ template <int BITS>
 int launch_bits(int epi, int pm, const CUtensorMap &tmap, const TcParams &p, cudaStream_t s)
 {
     if (epi == EPI_GEMM) {
+        if (pm == 4) return launch_tc<BITS, true, EPI_GEMM, 4>(tmap, p, s);
         if (pm == 3) return launch_tc<BITS, true, EPI_GEMM, 3>(tmap, p, s);
         if (pm == 2) return launch_tc<BITS, true, EPI_GEMM, 2>(tmap, p, s);
         return launch_tc<BITS, true, EPI_GEMM, 1>(tmap, p, s);
     }
+    if (pm == 4) return launch_conv<BITS, 4>(epi, tmap, p, s);
     if (pm == 3) return launch_conv<BITS, 3>(epi, tmap, p, s);
     if (pm == 2) return launch_conv<BITS, 2>(epi, tmap, p, s);
     return launch_conv<BITS, 1>(epi, tmap, p, s);
@@ -1071,9 +1193,12 @@ int dispatch_tc(int bits, int epi, int pm, const CUtensorMap &tmap, const TcPara
 // Pipeline mode for a problem (see Pipe<PM>); g_forced_ks: 0 automatic, 1 forces
 // single K steps, 2 forces double steps wherever they are possible.
 int g_forced_ks = 0;
+int g_pair_mode = 0;    // dsq_set_cta_pairs: 0 automatic, 1 never, 2 wherever possible
 int pick_pm(const TcParams &p, int bits)
 {
     if (bits == 3 || p.ksteps < 2 || g_forced_ks == 1) return 1;
+    // CTA pairs: 256-wide N tiles and at least two 128-row tiles to put together
+    if (p.BN == 256 && p.M > BM && g_pair_mode != 1) return 4;
     if (p.BN > 128) return p.ksteps >= 4 ? 3 : 1;
     if (g_forced_ks == 2) return 2;
     // when the expanded B tile can stay resident with single K steps, the
@@ -1091,6 +1216,13 @@ int dsq_set_round_k_steps(int ks)
 {
     if (ks != 0 && ks != 1 && ks != 2) return DSQ_ERR_SHAPE;
     g_forced_ks = ks;
+    return DSQ_OK;
+}
+
+int dsq_set_cta_pairs(int mode)
+{
+    if (mode < 0 || mode > 2) return DSQ_ERR_SHAPE;
+    g_pair_mode = mode;
     return DSQ_OK;
 }
 
@@ -1129,10 +1261,12 @@ int dsq_gemm(const void *A_codes, const void *B_codes, int64_t M, int64_t N, int
     p.n_tiles = (int)((N + p.BN - 1) / p.BN);
     const int pm = pick_pm(p, bits);
     const int ks = pm == 1 ? 1 : 2;
+    if (pm == 4) p.m_tiles = (int)((M + 2 * BM - 1) / (2 * BM));
     choose_b_mode(&p, bits, pm);
     p.act = (const uint8_t *)A_codes;
     p.H = 1; p.W = (int)M; p.Ho = 1; p.Wo = (int)M;
     p.stride = 1; p.pad = 0; p.KW = 1; p.taps = 1; p.P = (int)pitch;
+    p.a_lcr = a_run_log2(p.P, bits, ks);
     p.mode = MODE_GEMM;
     p.shift = 8 - bits;
     p.orv = 0;
@@ -1141,7 +1275,8 @@ int dsq_gemm(const void *A_codes, const void *B_codes, int64_t M, int64_t N, int
     p.D_f32 = D_f32;
     p.ws = (int *)workspace;
     CUtensorMap tmap;
-    int st = make_rows_tmap(&tmap, B_codes, pitch, (uint64_t)N, pitch, ks * 16 * bits, p.BN);
+    int st = make_rows_tmap(&tmap, B_codes, pitch, (uint64_t)N, pitch, ks * 16 * bits,
+                            pm == 4 ? p.BN / 2 : p.BN);
     if (st) return st;
     return dispatch_tc(bits, EPI_GEMM, pm, tmap, p, (cudaStream_t)stream);
 }
@@ -1190,10 +1325,12 @@ int dsq_conv2d(const void *act_codes, const dsq_nhwc_t *shape, const dsq_quant_t
     p.n_tiles = (conv->Cout + p.BN - 1) / p.BN;
     const int pm = pick_pm(p, bits);
     const int ks = pm == 1 ? 1 : 2;
+    if (pm == 4) p.m_tiles = (int)((M + 2 * BM - 1) / (2 * BM));
     choose_b_mode(&p, bits, pm);
     p.act = (const uint8_t *)act_codes;
     p.H = shape->H; p.W = shape->W; p.Ho = Ho; p.Wo = Wo;
     p.stride = conv->stride; p.pad = conv->pad; p.KW = conv->KW; p.taps = taps; p.P = (int)P;
+    p.a_lcr = a_run_log2(p.P, bits, ks);
     p.mode = MODE_CONV;
     p.e = e;
     p.out_pitch = (int)dsq_row_pitch(conv->Cout, bits);
@@ -1207,7 +1344,7 @@ int dsq_conv2d(const void *act_codes, const dsq_nhwc_t *shape, const dsq_quant_t
     p.ws = (int *)workspace;
     CUtensorMap tmap;
     st = make_rows_tmap(&tmap, w_packed, row_bytes, (uint64_t)conv->Cout, row_bytes, ks * 16 * bits,
-                        p.BN);
+                        pm == 4 ? p.BN / 2 : p.BN);
     if (st) return st;
     // largest |2*acc + S_a| below 2^22: the epilogue may convert integers to
     // float through the 1.5 * 2^23 bias trick, which is exact there
