@@ -81,6 +81,11 @@ template <int PM> struct Pipe {
     // memory requests, more instructions in the A threads; pays where the A
     // threads have slack
     static constexpr bool COAL = PAIR;
+    // B warps: one group of eight expands every round, or (pair mode, where a
+    // round is only 128 rows per CTA) two groups of four take alternate rounds,
+    // so that two rounds' latency chains (barrier, shared loads, stores, fence,
+    // arrival) overlap
+    static constexpr int B_GROUPS = PAIR ? 2 : 1;
 };
 constexpr int TMEM_COLS = 512;
 
@@ -112,6 +117,10 @@ struct TcParams {
     const uint8_t *act;
     int H, W, Ho, Wo, stride, pad, KW, taps, P;
     int a_lcr;                        // log2 of the A gather's run length in 16-byte chunks
+    // a_tma = 1: the A rows of a tile are rows of a plain 2-D matrix (GEMM, 1x1
+    // stride-1 convolution): TMA brings each round's 128 x (KS*CH*16)-byte box
+    // into the A ring (swizzled), and the A threads only read their rows
+    int a_tma, a_swz_shift, a_swz_mask;
     // epilogue
     int mode, shift, out_pitch, small_acc;
     DsqEpi e;
@@ -234,6 +243,7 @@ struct SmemLayout {
 };
 
 constexpr int MAX_S_P = 4;
+constexpr int MAX_A_SLOTS = 6;
 constexpr int MAX_B_STAGES = 16;
 
 __host__ __device__ inline SmemLayout smem_layout(int BN, int bits, int s_p, int b_stages, int ks,
@@ -247,25 +257,30 @@ __host__ __device__ inline SmemLayout smem_layout(int BN, int bits, int s_p, int
     // per-warp scale / bias staging (the B warps join the epilogue when resident)
     L.epi = o;      o += 4 * epw * 64 * 4;
     o = (o + 127u) & ~127u;
-    L.bars = o;     o += 8 * (2 * SU_MAX + MAX_B_STAGES + 2 * MAX_S_P + 4);
+    L.bars = o;     o += 8 * (2 * SU_MAX + MAX_B_STAGES + 2 * MAX_S_P + 4 + 2 * MAX_A_SLOTS);
     L.tmem_slot = o; o += 8;
     L.abort_flag = o; o += 8;
     L.total = o;
     return L;
 }
 
-template <int BITS, bool A_SIGNED, int EPI, int PM>
+template <int BITS, bool A_SIGNED, int EPI, int PM, bool A_TMA>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
-dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
+dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
+              const __grid_constant__ CUtensorMap tmap_a, const TcParams p)
 {
     constexpr bool B_SIGNED = !A_SIGNED;
     constexpr int CH = Chunks<BITS>::CH;
     constexpr int KS = Pipe<PM>::KS, GROUPS = Pipe<PM>::GROUPS;
     constexpr bool WIDE = Pipe<PM>::WIDE, PAIR = Pipe<PM>::PAIR;
+    constexpr int B_GROUPS = Pipe<PM>::B_GROUPS;
     constexpr int CG = PAIR ? 2 : 1;          // CTAs per tcgen05 instruction
     constexpr int BMT = BM * CG;              // tile rows
     constexpr int S_U = Pipe<PM>::SU, A_D = Pipe<PM>::A_D, A_RING = Pipe<PM>::A_RING;
     constexpr int A_COL0 = Pipe<PM>::A_COL0;
+    constexpr int A_SLOTS = GROUPS * A_RING;                // packed A ring slots
+    constexpr int A_SLOT_BYTES = KS * CH * BM * 16;         // one round of 128 rows
+    static_assert(A_SLOTS <= MAX_A_SLOTS, "A ring barriers");
     static_assert(KS == 1 || BITS != 3, "3-bit rows use single K steps");
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>(
@@ -307,6 +322,10 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
     auto bar_p_empty = [&](int s) { return bars + 8u * (BAR_P + MAX_S_P + s); };
     auto bar_acc_full = [&](int s) { return bars + 8u * (BAR_P + 2 * MAX_S_P + s); };
     auto bar_acc_empty = [&](int s) { return bars + 8u * (BAR_P + 2 * MAX_S_P + 2 + s); };
+    auto bar_ar_full = [&](int s) { return bars + 8u * (BAR_P + 2 * MAX_S_P + 4 + s); };
+    auto bar_ar_empty = [&](int s) {
+        return bars + 8u * (BAR_P + 2 * MAX_S_P + 4 + MAX_A_SLOTS + s);
+    };
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + L.tmem_slot);
     Ctl ctl{reinterpret_cast<volatile int *>(smem + L.abort_flag), p.ws};
     // The consumer of a_full / b_full / acc_empty is the MMA thread of rank 0:
@@ -325,13 +344,17 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
         for (int s = 0; s < S_U; ++s) {
             // operands of a round: the four warps of one A group and (unless the
             // expanded B tile is resident) the B warps, of every CTA of the pair
-            mbar_init(bar_a_full(s), (4 + (p.b_res ? 0 : NUM_B_WARPS)) * CG);
+            mbar_init(bar_a_full(s), (4 + (p.b_res ? 0 : NUM_B_WARPS / B_GROUPS)) * CG);
             mbar_init(bar_u_empty(s), 1);    // tcgen05.commit
         }
         for (int s = 0; s < MAX_B_STAGES; ++s) mbar_init(bar_b_full(s), NUM_B_WARPS * CG);
         for (int s = 0; s < S_P; ++s) {
             mbar_init(bar_p_full(s), 1);     // TMA producer (+ transaction bytes)
-            mbar_init(bar_p_empty(s), NUM_B_WARPS);
+            mbar_init(bar_p_empty(s), NUM_B_WARPS / B_GROUPS);
+        }
+        for (int s = 0; s < A_SLOTS; ++s) {
+            mbar_init(bar_ar_full(s), 1);    // TMA producer (+ transaction bytes)
+            mbar_init(bar_ar_empty(s), 4);   // the four warps of the slot's A group
         }
         for (int s = 0; s < 2; ++s) {
             mbar_init(bar_acc_full(s), 1);   // tcgen05.commit
@@ -344,7 +367,10 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
         tmem_alloc<CG>(smem_u32((const void *)tmem_slot), TMEM_COLS);
         tmem_relinquish<CG>();
     }
-    if (warp == WARP_TMA && lane == 0) tma_prefetch_desc(&tmap_b);
+    if (warp == WARP_TMA && lane == 0) {
+        tma_prefetch_desc(&tmap_b);
+        if (A_TMA) tma_prefetch_desc(&tmap_a);
+    }
     tc_fence_before_sync();
     __syncthreads();
     // no arrival may reach the peer before its barriers exist
@@ -354,24 +380,42 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
 
     int epi_idx = -1, epi_slot = 0;        // set for warps that run the epilogue
     if (warp == WARP_TMA) {
-        // ---------------- B producer: TMA packed tiles --------------------
+        // ---------------- producer: TMA packed B tiles (and A boxes) ---------
         if (lane == 0) {
-            uint32_t g = 0, ph = 0;
-            int s = 0, ks = 0, tile = tile0;
+            const uint32_t n_a_steps = A_TMA ? (uint32_t)my_tiles_all * p.rounds : 0u;
+            const uint32_t n_steps = n_b_steps > n_a_steps ? n_b_steps : n_a_steps;
+            const uint32_t ring = smem_u32(smem + L.a_ring);
+            uint32_t g = 0, ph = 0, issued_b = 0, issued_a = 0;
+            int s = 0, ks = 0, tile = tile0;       // B position
+            int ka = 0, tile_a = tile0;            // A position
 #pragma unroll 1
-            for (; g < n_b_steps; ++g) {
-                if (!wait_bar(bar_p_empty(s), ph ^ 1u, ctl, 1)) break;
-                mbar_arrive_expect_tx(bar_p_full(s), b_packed_bytes);
-                tma_load_2d(smem_u32(smem + L.b_packed + s * b_packed_bytes), &tmap_b,
-                            ks * (KS * 16 * BITS), (tile % p.n_tiles) * BN + (int)rank * BNL,
-                            bar_p_full(s));
-                if (++s == S_P) { s = 0; ph ^= 1u; }
-                if (++ks == p.rounds) { ks = 0; tile += tstep; }
+            for (; g < n_steps; ++g) {
+                if (g < n_b_steps) {
+                    if (!wait_bar(bar_p_empty(s), ph ^ 1u, ctl, 1)) break;
+                    mbar_arrive_expect_tx(bar_p_full(s), b_packed_bytes);
+                    tma_load_2d(smem_u32(smem + L.b_packed + s * b_packed_bytes), &tmap_b,
+                                ks * (KS * 16 * BITS),
+                                (tile % p.n_tiles) * BN + (int)rank * BNL, bar_p_full(s));
+                    ++issued_b;
+                    if (++s == S_P) { s = 0; ph ^= 1u; }
+                    if (++ks == p.rounds) { ks = 0; tile += tstep; }
+                }
+                if (A_TMA && g < n_a_steps) {
+                    const int sl = (int)(g % A_SLOTS);
+                    if (!wait_bar(bar_ar_empty(sl), ((g / A_SLOTS) & 1u) ^ 1u, ctl, 11)) break;
+                    mbar_arrive_expect_tx(bar_ar_full(sl), A_SLOT_BYTES);
+                    tma_load_2d(ring + sl * A_SLOT_BYTES, &tmap_a, ka * (KS * 16 * BITS),
+                                (tile_a / p.n_tiles) * BMT + row_base, bar_ar_full(sl));
+                    ++issued_a;
+                    if (++ka == p.rounds) { ka = 0; tile_a += tstep; }
+                }
             }
             // let outstanding copies land before the CTA can exit
-            const uint32_t issued = g;
-            for (uint32_t k = (issued > (uint32_t)S_P ? issued - S_P : 0); k < issued; ++k)
+            for (uint32_t k = (issued_b > (uint32_t)S_P ? issued_b - S_P : 0); k < issued_b; ++k)
                 wait_bar(bar_p_full(k % S_P), (k / S_P) & 1u, ctl, 2);
+            for (uint32_t k = (issued_a > (uint32_t)A_SLOTS ? issued_a - A_SLOTS : 0);
+                 k < issued_a; ++k)
+                wait_bar(bar_ar_full(k % A_SLOTS), (k / A_SLOTS) & 1u, ctl, 2);
         }
     } else if (warp == WARP_MMA) {
         // ---------------- MMA issuer ---------------------------------------
@@ -429,7 +473,7 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
         if (group < GROUPS) {
         const int quarter = warp & 3;              // TMEM lane quarter of this warp
         const int row = quarter * 32 + lane;
-        constexpr int SLOT_BYTES = KS * CH * BM * 16;   // ring slot = KS*CH planes x 128 rows x 16 B
+        constexpr int SLOT_BYTES = A_SLOT_BYTES;   // ring slot = KS*CH planes x 128 rows x 16 B
         const uint32_t cell0 =
             smem_u32(smem + L.a_ring) + group * (A_RING * SLOT_BYTES) + row * 16;
         // walk position over the flattened (tile, K step) sequence; starts one
@@ -470,28 +514,13 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
             }
             if (ld_tile < total_tiles) {
                 const uint32_t dst = ring0 + ld_slot * SLOT_BYTES;
+                // The walk advances run by run (2^lcr chunks that are contiguous in
+                // memory and lie in one filter tap), which keeps its dependent chain
+                // of address / tap updates short.
                 unsigned long long run = 0ull;     // this row's current run (0: zero fill)
-                if (!Pipe<PM>::COAL) {
-                    // every thread fetches its own row, chunk by chunk
-#pragma unroll
-                    for (int j = 0; j < KS * CH; ++j) {
-                        if (load) {
-                            const bool ok = tap < 32 && ((tap_mask >> tap) & 1u);
-                            cp_async_16(dst + lane * 16 + j * (BM * 16), ok ? src : p.act,
-                                        ok ? 16u : 0u);
-                        }
-                        off += 16;
-                        src += 16;
-                        if (off == p.P) {
-                            off = 0;
-                            ++tap;
-                            if (++kw == p.KW) { kw = 0; src += row_jump; }
-                        }
-                    }
-                } else
 #pragma unroll
                 for (int j = 0; j < KS * CH; ++j) {
-                    if ((j & crm) == 0) {          // a new run of 2^lcr chunks starts
+                    if ((j & crm) == 0) {          // a new run starts
                         const bool ok = tap < 32 && ((tap_mask >> tap) & 1u);
                         run = ok ? (unsigned long long)reinterpret_cast<uintptr_t>(src) : 0ull;
                         off += 16 << lcr;
@@ -502,7 +531,8 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
                             if (++kw == p.KW) { kw = 0; src += row_jump; }
                         }
                     }
-                    if (load) {
+                    if (!load) continue;
+                    if (Pipe<PM>::COAL) {
                         // lane -> (row of this warp, chunk of the run)
                         const int rsel = ((j & crm) << (5 - lcr)) + lane_row;
                         const unsigned long long ptr = __shfl_sync(0xffffffffu, run, rsel);
@@ -512,6 +542,13 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
                                               16 * lane_c
                                         : p.act,
                                     ptr ? 16u : 0u);
+                    } else {
+                        // every thread fetches its own row
+                        cp_async_16(dst + lane * 16 + j * (BM * 16),
+                                    run ? reinterpret_cast<const uint8_t *>((uintptr_t)run) +
+                                              16 * (j & crm)
+                                        : p.act,
+                                    run ? 16u : 0u);
                     }
                 }
                 ++ld_ks;
@@ -531,17 +568,28 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
             if (lane == 0) arrive_leader(bar_a_full(pend_s));
             pend_s = -1;
         };
-        if (GROUPS == 2 && group == 1) walk_step(false);   // step 0 belongs to group 0
+        // TMA mode: slot = 128 rows of KS*CH chunks, chunk index XOR-swizzled
+        constexpr bool a_tma = A_TMA;
+        const uint32_t tma_row = smem_u32(smem + L.a_ring) + row * (KS * CH * 16);
+        const int swz = (row >> p.a_swz_shift) & p.a_swz_mask;
+        if (!a_tma && GROUPS == 2 && group == 1) walk_step(false);   // step 0 belongs to group 0
         // iteration i issues own step i and consumes own step i - A_D
 #pragma unroll 1
         for (uint32_t i = 0; ok && i < n_own + A_D; ++i) {
-            walk_step(true);                       // own step (no-op past the end)
-            cp_async_commit();                     // one group per own step
-            if (GROUPS == 2) walk_step(false);     // the other group's step
+            if (!a_tma) {
+                walk_step(true);                   // own step (no-op past the end)
+                cp_async_commit();                 // one group per own step
+                if (GROUPS == 2) walk_step(false); // the other group's step
+            }
             if (i < (uint32_t)A_D) continue;
             const uint32_t g = GROUPS * (i - A_D) + group;
-            cp_async_wait<A_D>();                  // own step i - A_D has landed
-            if (Pipe<PM>::COAL) __syncwarp();      // ... the other lanes' copies of my row too
+            const int aslot = (int)(g % A_SLOTS);
+            if (a_tma) {
+                if (!(ok = wait_bar(bar_ar_full(aslot), (g / A_SLOTS) & 1u, ctl, 12))) break;
+            } else {
+                cp_async_wait<A_D>();              // own step i - A_D has landed
+                if (Pipe<PM>::COAL) __syncwarp();  // ... the other lanes' copies of my row too
+            }
             const int s = g % S_U;
             const uint32_t ph = (g / S_U) & 1u;
 #pragma unroll
@@ -551,7 +599,10 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
                     uint4 cur[CH];
 #pragma unroll
                     for (int j = 0; j < CH; ++j)
-                        cur[j] = lds_128(cell0 + rd_slot * SLOT_BYTES + (h * CH + j) * (BM * 16));
+                        cur[j] = a_tma ? lds_128(tma_row + aslot * SLOT_BYTES +
+                                                 (((h * CH + j) ^ swz) << 4))
+                                       : lds_128(cell0 + rd_slot * SLOT_BYTES +
+                                                 (h * CH + j) * (BM * 16));
                     expand_row_regs<BITS, A_SIGNED>(cur, p.orv, o);
                 }
                 if (h == 0) {
@@ -564,6 +615,10 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
             }
             if (!ok) break;
             if (++rd_slot == A_RING) rd_slot = 0;
+            if (a_tma) {                           // the slot may be refilled
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_ar_empty(aslot));
+            }
             pend_s = s;
             publish();                             // the other group's step overlaps this
         }
@@ -575,7 +630,9 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
         }
     } else if (warp < WARP_E0) {
         // ---------------- B: expand packed shared tiles ---------------------
-        const int tid = threadIdx.x - WARP_B0 * 32;
+        constexpr int BT = NUM_B_THREADS / B_GROUPS;      // threads expanding one round
+        const int bgroup = B_GROUPS == 1 ? 0 : (warp - WARP_B0) / (NUM_B_WARPS / B_GROUPS);
+        const int tid = threadIdx.x - WARP_B0 * 32 - bgroup * BT;
         // a packed row of the round holds CHK = KS*CH chunks.  Thread (row0, j)
         // owns chunk j of every K step of rows row0 + i*ROWS_PER_IT: the eight
         // lanes of a 128-bit store phase then cover two rows x four chunks of
@@ -583,19 +640,20 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
         // tile (lanes split over two K steps would collide pairwise, the K steps
         // being a multiple of 128 bytes apart); (row & 7) does not depend on i
         constexpr int CHK = KS * CH;
-        constexpr int ROWS_PER_IT = (BITS == 3) ? NUM_B_THREADS : NUM_B_THREADS / CH;
-        constexpr int MAX_IT = (BITS == 3) ? 1 : (256 * CH) / NUM_B_THREADS;
+        constexpr int ROWS_PER_IT = (BITS == 3) ? BT : BT / CH;
+        constexpr int MAX_IT = (BITS == 3) ? 1 : ((PAIR ? 128 : 256) * CH) / BT;
         const int row0 = (BITS == 3) ? tid : tid / CH;
         const int j = (BITS == 3) ? 0 : tid % CH;
         const int sw = row0 & 7;
         const int n_it = (BNL + ROWS_PER_IT - 1) / ROWS_PER_IT;
         uint32_t php = 0;
-        int sp = -1;
+        int sp = bgroup - B_GROUPS;
         bool ok = true;
         {
 #pragma unroll 1
-            for (uint32_t g = 0; g < n_b_steps; ++g) {
-                if (++sp == S_P) { sp = 0; php ^= 1u; }
+            for (uint32_t g = bgroup; g < n_b_steps; g += B_GROUPS) {
+                sp += B_GROUPS;                      // sp = g % S_P, php = (g / S_P) & 1
+                if (sp >= S_P) { sp -= S_P; php ^= 1u; }
                 const int su = p.b_res ? (int)g : (int)(g % S_U);
                 const uint32_t phu = (g / S_U) & 1u;
                 if (!(ok = wait_bar(bar_p_full(sp), php, ctl, 6))) break;
@@ -1025,8 +1083,11 @@ EncodeTiledFn get_encode_fn()
 }
 
 // 2-D byte map over packed rows: inner dimension = row bytes, outer = rows.
+struct TcMaps { CUtensorMap b, a; };
+
 int make_rows_tmap(CUtensorMap *map, const void *base, uint64_t row_bytes, uint64_t rows,
-                   uint64_t pitch, uint32_t box_bytes, uint32_t box_rows)
+                   uint64_t pitch, uint32_t box_bytes, uint32_t box_rows,
+                   CUtensorMapSwizzle swizzle = CU_TENSOR_MAP_SWIZZLE_NONE)
 {
     EncodeTiledFn fn = get_encode_fn();
     if (!fn) return DSQ_ERR_CUDA;
@@ -1036,7 +1097,7 @@ int make_rows_tmap(CUtensorMap *map, const void *base, uint64_t row_bytes, uint6
     cuuint32_t estr[2] = {1, 1};
     CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(base), dims,
                     strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                    CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                    swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? DSQ_OK : DSQ_ERR_CUDA;
 }
@@ -1088,6 +1149,31 @@ int a_run_log2(int P, int bits, int ks)
     return l;
 }
 
+// TMA-fed A ring: possible when the tile's A rows are rows of one 2-D matrix and
+// a round of a row is 32, 64 or 128 bytes (a swizzle span).  Fills p->a_tma and the
+// swizzle fields, and encodes the map.
+int setup_a_tma(TcParams *p, CUtensorMap *map, const void *A, int64_t rows, int bits, int ks,
+                bool plain_rows)
+{
+    p->a_tma = 0;
+    p->a_swz_shift = 0;
+    p->a_swz_mask = 0;
+    const int round_bytes = ks * bits * 16;
+    if (!plain_rows || bits == 3) return DSQ_OK;
+    // round_bytes is 32, 64 or 128: one swizzle span, so that the row-per-thread
+    // reads of the ring are free of bank conflicts
+    const int st = make_rows_tmap(map, A, (uint64_t)p->P, (uint64_t)rows, (uint64_t)p->P,
+                                  (uint32_t)round_bytes, BM,
+                                  round_bytes == 128  ? CU_TENSOR_MAP_SWIZZLE_128B
+                                  : round_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B
+                                                      : CU_TENSOR_MAP_SWIZZLE_32B);
+    if (st) return st;
+    p->a_tma = 1;
+    p->a_swz_shift = round_bytes == 128 ? 0 : round_bytes == 64 ? 1 : 2;
+    p->a_swz_mask = round_bytes == 128 ? 7 : round_bytes == 64 ? 3 : 1;
+    return DSQ_OK;
+}
+
 int g_forced_bn = 0;   // dsq_set_tile_n
 
 int pick_bn(int m_tiles, int ncols, int bits)
@@ -1108,9 +1194,10 @@ int pick_bn(int m_tiles, int ncols, int bits)
     return best;
 }
 
-template <int BITS, bool A_SIGNED, int EPI, int PM>
-int launch_tc(const CUtensorMap &tmap, const TcParams &p, cudaStream_t s)
+template <int BITS, bool A_SIGNED, int EPI, int PM, bool A_TMA>
+int launch_tc(const TcMaps &tmap, const TcParams &p, cudaStream_t s)
 {
+    if ((p.a_tma != 0) != A_TMA) return DSQ_ERR_UNSUPPORTED;
     constexpr bool PAIR = Pipe<PM>::PAIR;
     const SmemLayout L = smem_layout(PAIR ? p.BN / 2 : p.BN, BITS, p.s_p, p.b_stages,
                                      Pipe<PM>::KS, Pipe<PM>::GROUPS * Pipe<PM>::A_RING, p.epw);
@@ -1119,7 +1206,7 @@ int launch_tc(const CUtensorMap &tmap, const TcParams &p, cudaStream_t s)
     if (smem_bytes > 227 * 1024) smem_bytes = 227 * 1024;
     static bool configured = false;
     if (!configured) {
-        if (cudaFuncSetAttribute(dsq_tc_kernel<BITS, A_SIGNED, EPI, PM>,
+        if (cudaFuncSetAttribute(dsq_tc_kernel<BITS, A_SIGNED, EPI, PM, A_TMA>,
                                  cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  227 * 1024) != cudaSuccess)
             return DSQ_ERR_CUDA;
@@ -1145,35 +1232,43 @@ int launch_tc(const CUtensorMap &tmap, const TcParams &p, cudaStream_t s)
         attr[0].val.clusterDim.z = 1;
         cfg.attrs = attr;
         cfg.numAttrs = 1;
-        if (cudaLaunchKernelEx(&cfg, dsq_tc_kernel<BITS, A_SIGNED, EPI, PM>, tmap, q) !=
+        if (cudaLaunchKernelEx(&cfg, dsq_tc_kernel<BITS, A_SIGNED, EPI, PM, A_TMA>, tmap.b, tmap.a, q) !=
             cudaSuccess) {
             cudaGetLastError();
             return DSQ_ERR_CUDA;
         }
         return dsq_launch_status();
     }
-    dsq_tc_kernel<BITS, A_SIGNED, EPI, PM><<<grid, NUM_THREADS, smem_bytes, s>>>(tmap, q);
+    dsq_tc_kernel<BITS, A_SIGNED, EPI, PM, A_TMA><<<grid, NUM_THREADS, smem_bytes, s>>>(tmap.b, tmap.a, q);
     return dsq_launch_status();
 }
 
 template <int BITS, int PM>
-int launch_conv(int epi, const CUtensorMap &tmap, const TcParams &p, cudaStream_t s)
+int launch_conv(int epi, const TcMaps &tmap, const TcParams &p, cudaStream_t s)
 {
+    if (p.a_tma) {
+        switch (epi) {
+        case EPI_CODES: return launch_tc<BITS, false, EPI_CODES, PM, true>(tmap, p, s);
+        case EPI_CODES_RES: return launch_tc<BITS, false, EPI_CODES_RES, PM, true>(tmap, p, s);
+        default: return launch_tc<BITS, false, EPI_GENERAL, PM, true>(tmap, p, s);
+        }
+    }
     switch (epi) {
-    case EPI_CODES: return launch_tc<BITS, false, EPI_CODES, PM>(tmap, p, s);
-    case EPI_CODES_RES: return launch_tc<BITS, false, EPI_CODES_RES, PM>(tmap, p, s);
-    default: return launch_tc<BITS, false, EPI_GENERAL, PM>(tmap, p, s);
+    case EPI_CODES: return launch_tc<BITS, false, EPI_CODES, PM, false>(tmap, p, s);
+    case EPI_CODES_RES: return launch_tc<BITS, false, EPI_CODES_RES, PM, false>(tmap, p, s);
+    default: return launch_tc<BITS, false, EPI_GENERAL, PM, false>(tmap, p, s);
     }
 }
 
 template <int BITS>
-int launch_bits(int epi, int pm, const CUtensorMap &tmap, const TcParams &p, cudaStream_t s)
+int launch_bits(int epi, int pm, const TcMaps &tmap, const TcParams &p, cudaStream_t s)
 {
     if (epi == EPI_GEMM) {
-        if (pm == 4) return launch_tc<BITS, true, EPI_GEMM, 4>(tmap, p, s);
-        if (pm == 3) return launch_tc<BITS, true, EPI_GEMM, 3>(tmap, p, s);
-        if (pm == 2) return launch_tc<BITS, true, EPI_GEMM, 2>(tmap, p, s);
-        return launch_tc<BITS, true, EPI_GEMM, 1>(tmap, p, s);
+        // 2- and 4-bit GEMMs always fetch A with TMA
+        if (pm == 4) return launch_tc<BITS, true, EPI_GEMM, 4, true>(tmap, p, s);
+        if (pm == 3) return launch_tc<BITS, true, EPI_GEMM, 3, true>(tmap, p, s);
+        if (pm == 2) return launch_tc<BITS, true, EPI_GEMM, 2, true>(tmap, p, s);
+        return launch_tc<BITS, true, EPI_GEMM, 1, true>(tmap, p, s);
     }
     if (pm == 4) return launch_conv<BITS, 4>(epi, tmap, p, s);
     if (pm == 3) return launch_conv<BITS, 3>(epi, tmap, p, s);
@@ -1181,12 +1276,12 @@ int launch_bits(int epi, int pm, const CUtensorMap &tmap, const TcParams &p, cud
     return launch_conv<BITS, 1>(epi, tmap, p, s);
 }
 
-int dispatch_tc(int bits, int epi, int pm, const CUtensorMap &tmap, const TcParams &p,
+int dispatch_tc(int bits, int epi, int pm, const TcMaps &tmap, const TcParams &p,
                 cudaStream_t s)
 {
     if (bits == 4) return launch_bits<4>(epi, pm, tmap, p, s);
     if (bits == 2) return launch_bits<2>(epi, pm, tmap, p, s);
-    if (bits == 3 && epi == EPI_GEMM) return launch_tc<3, true, EPI_GEMM, 1>(tmap, p, s);
+    if (bits == 3 && epi == EPI_GEMM) return launch_tc<3, true, EPI_GEMM, 1, false>(tmap, p, s);
     return DSQ_ERR_UNSUPPORTED;
 }
 
@@ -1274,9 +1369,12 @@ int dsq_gemm(const void *A_codes, const void *B_codes, int64_t M, int64_t N, int
     p.row_scale = row_scale;
     p.D_f32 = D_f32;
     p.ws = (int *)workspace;
-    CUtensorMap tmap;
-    int st = make_rows_tmap(&tmap, B_codes, pitch, (uint64_t)N, pitch, ks * 16 * bits,
+    TcMaps tmap;
+    int st = make_rows_tmap(&tmap.b, B_codes, pitch, (uint64_t)N, pitch, ks * 16 * bits,
                             pm == 4 ? p.BN / 2 : p.BN);
+    if (st) return st;
+    tmap.a = tmap.b;
+    st = setup_a_tma(&p, &tmap.a, A_codes, M, bits, ks, true);
     if (st) return st;
     return dispatch_tc(bits, EPI_GEMM, pm, tmap, p, (cudaStream_t)stream);
 }
@@ -1342,9 +1440,14 @@ int dsq_conv2d(const void *act_codes, const dsq_nhwc_t *shape, const dsq_quant_t
         p.orv = 0;
     }
     p.ws = (int *)workspace;
-    CUtensorMap tmap;
-    st = make_rows_tmap(&tmap, w_packed, row_bytes, (uint64_t)conv->Cout, row_bytes, ks * 16 * bits,
-                        pm == 4 ? p.BN / 2 : p.BN);
+    TcMaps tmap;
+    st = make_rows_tmap(&tmap.b, w_packed, row_bytes, (uint64_t)conv->Cout, row_bytes,
+                        ks * 16 * bits, pm == 4 ? p.BN / 2 : p.BN);
+    if (st) return st;
+    tmap.a = tmap.b;
+    // a 1x1 stride-1 unpadded convolution reads the pixel rows as they lie
+    st = setup_a_tma(&p, &tmap.a, act_codes, M, bits, ks,
+                     conv->KH == 1 && conv->stride == 1 && conv->pad == 0);
     if (st) return st;
     // largest |2*acc + S_a| below 2^22: the epilogue may convert integers to
     // float through the 1.5 * 2^23 bias trick, which is exact there
