@@ -152,6 +152,24 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *m,
         : "memory");
 }
 
+// 4-D im2col load over an NHWC tensor (dims C, W, H, N): `pixelsPerColumn`
+// pixels x `channelsPerPixel` bytes.  (w, h) is the position of the filter
+// window's corner for the first pixel (output position * stride - pad); the
+// pixels that follow are the next window positions in W, then H, then N order
+// inside the map's bounding box.  (off_w, off_h) selects the filter tap; a
+// pixel outside the image is filled with zeros.  c * element size must be a
+// multiple of 16 bytes.
+__device__ __forceinline__ void tma_load_im2col_4d(uint32_t dst, const CUtensorMap *m, int c,
+                                                   int w, int h, int n, uint16_t off_w,
+                                                   uint16_t off_h, uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.im2col.mbarrier::complete_tx::bytes"
+        " [%0], [%1, {%2, %3, %4, %5}], [%6], {%7, %8};" ::"r"(dst),
+        "l"(m), "r"(c), "r"(w), "r"(h), "r"(n), "r"(bar), "h"(off_w), "h"(off_h)
+        : "memory");
+}
+
 // ---- tensor memory ---------------------------------------------------------
 // Executed by one full warp.  ncols: power of two, 32..512.  CG = 2: the
 // same warp of both CTAs of a pair executes it, and both get the same columns.

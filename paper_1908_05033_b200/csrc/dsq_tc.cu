@@ -89,13 +89,14 @@ template <int PM> struct Pipe {
 };
 constexpr int TMEM_COLS = 512;
 
-constexpr int WARP_TMA = 0, WARP_MMA = 1, WARP_A0 = 2, WARP_B0 = 10, WARP_E0 = 18;
+constexpr int WARP_TMA = 0, WARP_MMA = 1, WARP_A0 = 2, WARP_B0 = 10, WARP_E0 = 18,
+              WARP_TMA_A = 22;
 // two groups of four A warps take alternate K steps
 constexpr int NUM_A_GROUPS = 2, NUM_A_WARPS = 4 * NUM_A_GROUPS, NUM_B_WARPS = 8, NUM_E_WARPS = 4;
 constexpr int NUM_B_THREADS = NUM_B_WARPS * 32;
-constexpr int NUM_WARPS = 22;
+constexpr int NUM_WARPS = 23;
 static_assert(WARP_A0 + NUM_A_WARPS == WARP_B0 && WARP_B0 + NUM_B_WARPS == WARP_E0 &&
-                  WARP_E0 + NUM_E_WARPS == NUM_WARPS,
+                  WARP_E0 + NUM_E_WARPS == WARP_TMA_A && WARP_TMA_A + 1 == NUM_WARPS,
               "warp roles");
 constexpr int NUM_THREADS = NUM_WARPS * 32;
 constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;   // a wait gives up after 2 s
@@ -117,10 +118,18 @@ struct TcParams {
     const uint8_t *act;
     int H, W, Ho, Wo, stride, pad, KW, taps, P;
     int a_lcr;                        // log2 of the A gather's run length in 16-byte chunks
-    // a_tma = 1: the A rows of a tile are rows of a plain 2-D matrix (GEMM, 1x1
-    // stride-1 convolution): TMA brings each round's 128 x (KS*CH*16)-byte box
-    // into the A ring (swizzled), and the A threads only read their rows
-    int a_tma, a_swz_shift, a_swz_mask;
+    // a_tma != 0: TMA brings each round's 128 rows of packed A into the A ring and
+    // the A threads only read their rows.  A round is a_nsub boxes of 128 rows x
+    // a_sub bytes (a_sub = 16 << a_lc <= 128, one swizzle span), stored one after
+    // the other.
+    //   1: the rows are rows of a plain 2-D matrix (GEMM, 1x1 stride-1
+    //      convolution): one box per round
+    //   2: im2col over the NHWC tensor: a box is one run of a_sub bytes of one
+    //      filter tap of 128 consecutive output pixels (a_sub divides the pixel
+    //      pitch, so a box never straddles two taps); K columns past the last
+    //      tap are not loaded, the A threads put zeros there (a_kchunks = 16-byte
+    //      chunks of a row that exist)
+    int a_tma, a_lc, a_nsub, a_kchunks;
     // epilogue
     int mode, shift, out_pitch, small_acc;
     DsqEpi e;
@@ -380,39 +389,72 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
 
     int epi_idx = -1, epi_slot = 0;        // set for warps that run the epilogue
     if (warp == WARP_TMA) {
-        // ---------------- producer: TMA packed B tiles (and A boxes) ---------
+        // ---------------- producer: TMA packed B tiles -----------------------
+        // (the A boxes have a producer thread of their own in another warp: every
+        // wait / expect / issue of one thread is a chain of shared-memory
+        // pipeline round trips, a few hundred cycles each while the unpack warps
+        // keep that pipeline busy)
         if (lane == 0) {
-            const uint32_t n_a_steps = A_TMA ? (uint32_t)my_tiles_all * p.rounds : 0u;
-            const uint32_t n_steps = n_b_steps > n_a_steps ? n_b_steps : n_a_steps;
-            const uint32_t ring = smem_u32(smem + L.a_ring);
-            uint32_t g = 0, ph = 0, issued_b = 0, issued_a = 0;
-            int s = 0, ks = 0, tile = tile0;       // B position
-            int ka = 0, tile_a = tile0;            // A position
+            uint32_t g = 0, ph = 0, issued_b = 0;
+            int s = 0, ks = 0, tile = tile0;
 #pragma unroll 1
-            for (; g < n_steps; ++g) {
-                if (g < n_b_steps) {
-                    if (!wait_bar(bar_p_empty(s), ph ^ 1u, ctl, 1)) break;
-                    mbar_arrive_expect_tx(bar_p_full(s), b_packed_bytes);
-                    tma_load_2d(smem_u32(smem + L.b_packed + s * b_packed_bytes), &tmap_b,
-                                ks * (KS * 16 * BITS),
-                                (tile % p.n_tiles) * BN + (int)rank * BNL, bar_p_full(s));
-                    ++issued_b;
-                    if (++s == S_P) { s = 0; ph ^= 1u; }
-                    if (++ks == p.rounds) { ks = 0; tile += tstep; }
-                }
-                if (A_TMA && g < n_a_steps) {
-                    const int sl = (int)(g % A_SLOTS);
-                    if (!wait_bar(bar_ar_empty(sl), ((g / A_SLOTS) & 1u) ^ 1u, ctl, 11)) break;
-                    mbar_arrive_expect_tx(bar_ar_full(sl), A_SLOT_BYTES);
-                    tma_load_2d(ring + sl * A_SLOT_BYTES, &tmap_a, ka * (KS * 16 * BITS),
-                                (tile_a / p.n_tiles) * BMT + row_base, bar_ar_full(sl));
-                    ++issued_a;
-                    if (++ka == p.rounds) { ka = 0; tile_a += tstep; }
-                }
+            for (; g < n_b_steps; ++g) {
+                if (!wait_bar(bar_p_empty(s), ph ^ 1u, ctl, 1)) break;
+                mbar_arrive_expect_tx(bar_p_full(s), b_packed_bytes);
+                tma_load_2d(smem_u32(smem + L.b_packed + s * b_packed_bytes), &tmap_b,
+                            ks * (KS * 16 * BITS),
+                            (tile % p.n_tiles) * BN + (int)rank * BNL, bar_p_full(s));
+                ++issued_b;
+                if (++s == S_P) { s = 0; ph ^= 1u; }
+                if (++ks == p.rounds) { ks = 0; tile += tstep; }
             }
             // let outstanding copies land before the CTA can exit
             for (uint32_t k = (issued_b > (uint32_t)S_P ? issued_b - S_P : 0); k < issued_b; ++k)
                 wait_bar(bar_p_full(k % S_P), (k / S_P) & 1u, ctl, 2);
+        }
+    } else if (warp == WARP_TMA_A) {
+        // ---------------- producer: TMA packed A boxes -----------------------
+        if (A_TMA && lane == 0) {
+            const uint32_t n_a_steps = (uint32_t)my_tiles_all * p.rounds;
+            const uint32_t ring = smem_u32(smem + L.a_ring);
+            uint32_t g = 0, issued_a = 0;
+            int ka = 0, tile_a = tile0;
+            int i2c_w = 0, i2c_h = 0, i2c_n = 0, i2c_c = 0, i2c_kw = 0, i2c_kh = 0;
+#pragma unroll 1
+            for (; g < n_a_steps; ++g) {
+                const int sl = (int)(g % A_SLOTS);
+                if (!wait_bar(bar_ar_empty(sl), ((g / A_SLOTS) & 1u) ^ 1u, ctl, 11)) break;
+                const int m0 = (tile_a / p.n_tiles) * BMT + row_base;
+                if (p.a_tma == 1) {
+                    mbar_arrive_expect_tx(bar_ar_full(sl), A_SLOT_BYTES);
+                    tma_load_2d(ring + sl * A_SLOT_BYTES, &tmap_a, ka * (KS * 16 * BITS), m0,
+                                bar_ar_full(sl));
+                } else {
+                    if (ka == 0) {                 // first pixel of the tile, first tap
+                        const int wo = m0 % p.Wo, t = m0 / p.Wo;
+                        i2c_w = wo * p.stride - p.pad;
+                        i2c_h = (t % p.Ho) * p.stride - p.pad;
+                        i2c_n = t / p.Ho;
+                        i2c_c = 0; i2c_kw = 0; i2c_kh = 0;
+                    }
+                    const int sub = 16 << p.a_lc;
+                    const int left = (p.a_kchunks * 16 - ka * (KS * 16 * BITS)) / sub;
+                    const int nb = left < p.a_nsub ? left : p.a_nsub;
+                    mbar_arrive_expect_tx(bar_ar_full(sl), (uint32_t)(nb * BM * sub));
+                    for (int i = 0; i < nb; ++i) {
+                        tma_load_im2col_4d(ring + sl * A_SLOT_BYTES + i * (BM * sub), &tmap_a,
+                                           i2c_c, i2c_w, i2c_h, i2c_n, (uint16_t)i2c_kw,
+                                           (uint16_t)i2c_kh, bar_ar_full(sl));
+                        i2c_c += sub;
+                        if (i2c_c == p.P) {
+                            i2c_c = 0;
+                            if (++i2c_kw == p.KW) { i2c_kw = 0; ++i2c_kh; }
+                        }
+                    }
+                }
+                ++issued_a;
+                if (++ka == p.rounds) { ka = 0; tile_a += tstep; }
+            }
             for (uint32_t k = (issued_a > (uint32_t)A_SLOTS ? issued_a - A_SLOTS : 0);
                  k < issued_a; ++k)
                 wait_bar(bar_ar_full(k % A_SLOTS), (k / A_SLOTS) & 1u, ctl, 2);
@@ -570,8 +612,16 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
         };
         // TMA mode: slot = 128 rows of KS*CH chunks, chunk index XOR-swizzled
         constexpr bool a_tma = A_TMA;
-        const uint32_t tma_row = smem_u32(smem + L.a_ring) + row * (KS * CH * 16);
-        const int swz = (row >> p.a_swz_shift) & p.a_swz_mask;
+        // chunk jj of the round lies in box jj >> a_lc, at chunk (jj ^ swizzle) of
+        // this thread's row of that box
+        const int lc = p.a_lc;
+        const uint32_t tma_row = smem_u32(smem + L.a_ring) + ((uint32_t)row << (4 + lc));
+        const int swz = (row >> (3 - lc)) & ((1 << lc) - 1);
+        auto tma_chunk = [&](int jj) {
+            return tma_row + ((uint32_t)(jj >> lc) << (11 + lc)) +
+                   (uint32_t)((((jj & ((1 << lc) - 1)) ^ swz)) << 4);
+        };
+        int kr = group % p.rounds;                 // K round of the step being consumed
         if (!a_tma && GROUPS == 2 && group == 1) walk_step(false);   // step 0 belongs to group 0
         // iteration i issues own step i and consumes own step i - A_D
 #pragma unroll 1
@@ -592,17 +642,31 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
             }
             const int s = g % S_U;
             const uint32_t ph = (g / S_U) & 1u;
+            // chunks of this round that exist (im2col: nothing is loaded past the
+            // last filter tap)
+            int kvalid = KS * CH;
+            if (a_tma) {
+                if (p.a_tma == 2) kvalid = p.a_kchunks - kr * (KS * CH);
+                kr += GROUPS;
+                if (kr >= p.rounds) kr -= p.rounds;
+                if (kr >= p.rounds) kr -= p.rounds;
+            }
 #pragma unroll
             for (int h = 0; h < KS; ++h) {
                 uint32_t o[32];
                 {
                     uint4 cur[CH];
 #pragma unroll
-                    for (int j = 0; j < CH; ++j)
-                        cur[j] = a_tma ? lds_128(tma_row + aslot * SLOT_BYTES +
-                                                 (((h * CH + j) ^ swz) << 4))
-                                       : lds_128(cell0 + rd_slot * SLOT_BYTES +
-                                                 (h * CH + j) * (BM * 16));
+                    for (int j = 0; j < CH; ++j) {
+                        if (a_tma) {
+                            cur[j] = (h * CH + j < kvalid)
+                                         ? lds_128(tma_chunk(h * CH + j) + aslot * SLOT_BYTES)
+                                         : make_uint4(0u, 0u, 0u, 0u);
+                        } else {
+                            cur[j] = lds_128(cell0 + rd_slot * SLOT_BYTES +
+                                             (h * CH + j) * (BM * 16));
+                        }
+                    }
                     expand_row_regs<BITS, A_SIGNED>(cur, p.orv, o);
                 }
                 if (h == 0) {
@@ -1149,28 +1213,79 @@ int a_run_log2(int P, int bits, int ks)
     return l;
 }
 
-// TMA-fed A ring: possible when the tile's A rows are rows of one 2-D matrix and
-// a round of a row is 32, 64 or 128 bytes (a swizzle span).  Fills p->a_tma and the
-// swizzle fields, and encodes the map.
+typedef CUresult (*EncodeIm2colFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *,
+                                   const cuuint64_t *, const cuuint64_t *, const int *,
+                                   const int *, cuuint32_t, cuuint32_t, const cuuint32_t *,
+                                   CUtensorMapInterleave, CUtensorMapSwizzle,
+                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeIm2colFn get_encode_im2col_fn()
+{
+    static EncodeIm2colFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void *sym = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeIm2col", &sym, cudaEnableDefault, &qres) ==
+                cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeIm2colFn>(sym);
+    }
+    return fn;
+}
+
+CUtensorMapSwizzle swizzle_for_span(int bytes)
+{
+    return bytes == 128  ? CU_TENSOR_MAP_SWIZZLE_128B
+           : bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B
+           : bytes == 32 ? CU_TENSOR_MAP_SWIZZLE_32B
+                         : CU_TENSOR_MAP_SWIZZLE_NONE;
+}
+
+// TMA-fed A ring.  A round of a row (32, 64 or 128 packed bytes) is cut into
+// boxes of 128 rows x `sub` bytes, sub a power of two between 16 and 128 (one
+// swizzle span, so that the row-per-thread reads of the ring are free of bank
+// conflicts).  Plain rows (GEMM, 1x1 stride-1 unpadded convolution): one 2-D
+// box per round.  Any other convolution: im2col boxes over the NHWC tensor,
+// `sub` the largest such power of two that divides the pixel pitch.
 int setup_a_tma(TcParams *p, CUtensorMap *map, const void *A, int64_t rows, int bits, int ks,
-                bool plain_rows)
+                bool plain_rows, const dsq_nhwc_t *shape, int ksize)
 {
     p->a_tma = 0;
-    p->a_swz_shift = 0;
-    p->a_swz_mask = 0;
+    p->a_lc = 0;
+    p->a_nsub = 1;
+    p->a_kchunks = 0;
     const int round_bytes = ks * bits * 16;
-    if (!plain_rows || bits == 3) return DSQ_OK;
-    // round_bytes is 32, 64 or 128: one swizzle span, so that the row-per-thread
-    // reads of the ring are free of bank conflicts
-    const int st = make_rows_tmap(map, A, (uint64_t)p->P, (uint64_t)rows, (uint64_t)p->P,
-                                  (uint32_t)round_bytes, BM,
-                                  round_bytes == 128  ? CU_TENSOR_MAP_SWIZZLE_128B
-                                  : round_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B
-                                                      : CU_TENSOR_MAP_SWIZZLE_32B);
-    if (st) return st;
-    p->a_tma = 1;
-    p->a_swz_shift = round_bytes == 128 ? 0 : round_bytes == 64 ? 1 : 2;
-    p->a_swz_mask = round_bytes == 128 ? 7 : round_bytes == 64 ? 3 : 1;
+    if (bits == 3) return DSQ_OK;
+    if (plain_rows) {
+        const int st = make_rows_tmap(map, A, (uint64_t)p->P, (uint64_t)rows, (uint64_t)p->P,
+                                      (uint32_t)round_bytes, BM, swizzle_for_span(round_bytes));
+        if (st) return st;
+        p->a_tma = 1;
+        p->a_lc = round_bytes == 128 ? 3 : round_bytes == 64 ? 2 : 1;
+        return DSQ_OK;
+    }
+    int sub = 128;
+    while (sub > 16 && (p->P % sub != 0 || round_bytes % sub != 0)) sub >>= 1;
+    EncodeIm2colFn fn = get_encode_im2col_fn();
+    if (!fn) return DSQ_ERR_CUDA;
+    const cuuint64_t P = (cuuint64_t)p->P;
+    cuuint64_t dims[4] = {P, (cuuint64_t)shape->W, (cuuint64_t)shape->H, (cuuint64_t)shape->N};
+    cuuint64_t strides[3] = {P, P * shape->W, P * shape->W * shape->H};
+    // window-corner positions run from -pad to (extent - 1) + pad - (ksize - 1)
+    int lower[2] = {-p->pad, -p->pad};
+    int upper[2] = {p->pad - (ksize - 1), p->pad - (ksize - 1)};
+    cuuint32_t estr[4] = {1, (cuuint32_t)p->stride, (cuuint32_t)p->stride, 1};
+    const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void *>(A), dims,
+                          strides, lower, upper, (cuuint32_t)sub, BM, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_for_span(sub),
+                          CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return DSQ_ERR_CUDA;
+    p->a_tma = 2;
+    p->a_lc = sub == 128 ? 3 : sub == 64 ? 2 : sub == 32 ? 1 : 0;
+    p->a_nsub = round_bytes / sub;
+    p->a_kchunks = p->taps * (p->P / 16);
     return DSQ_OK;
 }
 
@@ -1374,7 +1489,7 @@ int dsq_gemm(const void *A_codes, const void *B_codes, int64_t M, int64_t N, int
                             pm == 4 ? p.BN / 2 : p.BN);
     if (st) return st;
     tmap.a = tmap.b;
-    st = setup_a_tma(&p, &tmap.a, A_codes, M, bits, ks, true);
+    st = setup_a_tma(&p, &tmap.a, A_codes, M, bits, ks, true, nullptr, 1);
     if (st) return st;
     return dispatch_tc(bits, EPI_GEMM, pm, tmap, p, (cudaStream_t)stream);
 }
@@ -1447,7 +1562,7 @@ int dsq_conv2d(const void *act_codes, const dsq_nhwc_t *shape, const dsq_quant_t
     tmap.a = tmap.b;
     // a 1x1 stride-1 unpadded convolution reads the pixel rows as they lie
     st = setup_a_tma(&p, &tmap.a, act_codes, M, bits, ks,
-                     conv->KH == 1 && conv->stride == 1 && conv->pad == 0);
+                     conv->KH == 1 && conv->stride == 1 && conv->pad == 0, shape, conv->KH);
     if (st) return st;
     // largest |2*acc + S_a| below 2^22: the epilogue may convert integers to
     // float through the 1.5 * 2^23 bias trick, which is exact there
