@@ -113,6 +113,9 @@ struct TcParams {
     // for the life of the CTA (one N tile, few K steps: small weight matrices)
     int b_res, b_stages;
     int epw;                          // epilogue warps per TMEM lane quarter (1..3)
+    // join = 1: on the CTA's last tile the A and B warps join the epilogue (needs
+    // a scale / bias staging slot for each of the 20 warps in shared memory)
+    int join;
     int smem_bytes;                   // dynamic shared memory given to the launch
     // A gather geometry (a GEMM is a 1x1 convolution over an M x 1 image)
     const uint8_t *act;
@@ -255,18 +258,21 @@ constexpr int MAX_S_P = 4;
 constexpr int MAX_A_SLOTS = 6;
 constexpr int MAX_B_STAGES = 16;
 
+constexpr int JOIN_CNT = 5;               // warps per lane quarter in a joined epilogue
+__host__ __device__ inline int epi_slots(int join, int epw) { return join ? 4 * JOIN_CNT : 4 * epw; }
+
 __host__ __device__ inline SmemLayout smem_layout(int BN, int bits, int s_p, int b_stages, int ks,
-                                                int a_slots, int epw)
+                                                int a_slots, int epi_slots)
 {
     SmemLayout L;
     uint32_t o = 0;
     L.b_tiles = o;  o += b_stages * ks * BN * BK_BYTES;
     L.b_packed = o; o += s_p * ks * BN * 16 * bits;
     L.a_ring = o;   o += a_slots * ks * BM * 16 * bits;
-    // per-warp scale / bias staging (the B warps join the epilogue when resident)
-    L.epi = o;      o += 4 * epw * 64 * 4;
+    // per-warp scale / bias staging (any warp may take part in an epilogue)
+    L.epi = o;      o += epi_slots * 64 * 4;
     o = (o + 127u) & ~127u;
-    L.bars = o;     o += 8 * (2 * SU_MAX + MAX_B_STAGES + 2 * MAX_S_P + 4 + 2 * MAX_A_SLOTS);
+    L.bars = o;     o += 8 * (2 * SU_MAX + MAX_B_STAGES + 2 * MAX_S_P + 4 + 2 * MAX_A_SLOTS + 1);
     L.tmem_slot = o; o += 8;
     L.abort_flag = o; o += 8;
     L.total = o;
@@ -297,7 +303,7 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
     const int BN = p.BN;
     const int BNL = BN / CG;                  // B rows this CTA expands
     const SmemLayout L =
-        smem_layout(BNL, BITS, p.s_p, p.b_stages, KS, GROUPS * A_RING, p.epw);
+        smem_layout(BNL, BITS, p.s_p, p.b_stages, KS, GROUPS * A_RING, epi_slots(p.join, p.epw));
     // the layout must fit behind the 1024-byte aligned base (the host adds
     // slack only while it stays within the 227 KB limit); same answer in every
     // thread of every CTA, taken before any barrier exists
@@ -335,6 +341,8 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
     auto bar_ar_empty = [&](int s) {
         return bars + 8u * (BAR_P + 2 * MAX_S_P + 4 + MAX_A_SLOTS + s);
     };
+    // completes once, when the accumulators of this CTA's last tile are final
+    const uint32_t bar_last_full = bars + 8u * (BAR_P + 2 * MAX_S_P + 4 + 2 * MAX_A_SLOTS);
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + L.tmem_slot);
     Ctl ctl{reinterpret_cast<volatile int *>(smem + L.abort_flag), p.ws};
     // The consumer of a_full / b_full / acc_empty is the MMA thread of rank 0:
@@ -369,6 +377,7 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
             mbar_init(bar_acc_full(s), 1);   // tcgen05.commit
             mbar_init(bar_acc_empty(s), 4 * p.epw * CG);
         }
+        mbar_init(bar_last_full, 1);         // tcgen05.commit
         *ctl.abort_flag = 0;
         mbar_init_fence();
     }
@@ -387,7 +396,13 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
 
-    int epi_idx = -1, epi_slot = 0;        // set for warps that run the epilogue
+    // Epilogue roles.  epi_idx >= 0: the warp takes part in the epilogue of every
+    // tile (p.epw warps per TMEM lane quarter).  join_idx >= 0: it takes part in
+    // the epilogue of the CTA's LAST tile, where nothing is left to overlap with,
+    // so the A and B warps, done with their rounds, help out (JOIN_CNT warps per
+    // quarter: a lone warp issues an instruction every few cycles at best).
+    int epi_idx = -1, join_idx = -1;
+    int epi_slot = warp - WARP_A0;         // joined: one slot per A / B / epilogue warp
     if (warp == WARP_TMA) {
         // ---------------- producer: TMA packed B tiles -----------------------
         // (the A boxes have a producer thread of their own in another warp: every
@@ -493,7 +508,10 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
                                      idesc, (uint32_t)(ks | h));
                     commit_all(bar_u_empty(s));
                 }
-                if (ok) commit_all(bar_acc_full(as));
+                if (ok) {
+                    commit_all(bar_acc_full(as));
+                    if (tile + tstep >= total_tiles) commit_all(bar_last_full);
+                }
             }
         }
     } else if (warp < WARP_B0) {
@@ -687,10 +705,12 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
             publish();                             // the other group's step overlaps this
         }
         cp_async_wait<0>();
+        if (ok && p.join) join_idx = 1 + group;
         } else if (WIDE) {
             // the unused second A group helps the epilogue
             epi_idx = 1;
-            epi_slot = NUM_E_WARPS + (warp - WARP_A0 - 4);
+            join_idx = 2;
+            if (!p.join) epi_slot = NUM_E_WARPS + (warp - WARP_A0 - 4);
         }
     } else if (warp < WARP_E0) {
         // ---------------- B: expand packed shared tiles ---------------------
@@ -786,30 +806,40 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
         // rounds: they join the epilogue (two more warps per TMEM lane quarter)
         if (p.b_res && ok) {
             epi_idx = 1 + ((warp - WARP_B0) >> 2);
-            epi_slot = NUM_E_WARPS + (warp - WARP_B0);
+            if (!p.join) epi_slot = NUM_E_WARPS + (warp - WARP_B0);
         }
+        if (ok && p.join) join_idx = 3 + ((warp - WARP_B0) >> 2);
     } else {
         epi_idx = 0;
-        epi_slot = warp - WARP_E0;
+        join_idx = 0;
+        if (!p.join) epi_slot = warp - WARP_E0;
     }
 
-    if (epi_idx >= 0) {
+    if (epi_idx >= 0 || join_idx >= 0) {
         // ---------------- epilogue -------------------------------------------
         // epi_cnt warps share a lane quarter and take the 32-column chunks of a
         // tile in turn
-        const int epi_cnt = p.epw;
         const int quarter = warp & 3;                 // TMEM lanes 32q .. 32q+31
         const int row_in_tile = quarter * 32 + lane;
         uint32_t it = 0;
         bool ok = true;
 #pragma unroll 1
         for (int tile = tile0; ok && tile < total_tiles; tile += tstep, ++it) {
+            const bool last = tile + tstep >= total_tiles;
+            const bool joined = last && p.join;
+            const int my_idx = joined ? join_idx : epi_idx;
+            const int epi_cnt = joined ? JOIN_CNT : p.epw;
+            if (my_idx < 0) continue;
             const int as = p.n_acc == 2 ? (it & 1) : 0;
             const uint32_t aph = (p.n_acc == 2 ? (it >> 1) : it) & 1u;
             const int m_tile = tile / p.n_tiles, n_tile = tile % p.n_tiles;
             const int64_t m = (int64_t)m_tile * BMT + row_base + row_in_tile;
             const bool row_ok = m < p.M;
-            if (!(ok = wait_bar(bar_acc_full(as), aph, ctl, 8))) break;
+            // helpers have not followed the accumulator barriers' phases: they wait
+            // on the single-use barrier of the last tile
+            if (!(ok = epi_idx >= 0 ? wait_bar(bar_acc_full(as), aph, ctl, 8)
+                                    : wait_bar(bar_last_full, 0u, ctl, 13)))
+                break;
             tc_fence_after_sync();
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + as * BN;
             float rs = 0.f;
@@ -829,9 +859,9 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
                     bi_nx = __ldg(p.e.bias + n);
                 }
             };
-            fetch_cols(epi_idx * 32);
+            fetch_cols(my_idx * 32);
 #pragma unroll 1
-            for (int c0 = epi_idx * 32; c0 < BN; c0 += 32 * epi_cnt) {
+            for (int c0 = my_idx * 32; c0 < BN; c0 += 32 * epi_cnt) {
                 uint32_t r[32];
                 __syncwarp();
                 tmem_ld_32x32(taddr + c0, r);
@@ -1045,7 +1075,7 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
             }
             tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) arrive_leader(bar_acc_empty(as));
+            if (lane == 0 && epi_idx >= 0) arrive_leader(bar_acc_empty(as));
         }
     }
 
@@ -1192,13 +1222,17 @@ void choose_b_mode(TcParams *p, int bits, int pm)
     p->b_stages = pi.su;
     p->epw = pi.wide ? 2 : 1;
     if (!pi.wide && !pi.pair && p->n_tiles == 1 && p->rounds <= MAX_B_STAGES && p->m_tiles > 148) {
-        const SmemLayout L = smem_layout(p->BN, bits, p->s_p, p->rounds, pi.ks, pi.a_slots, 3);
+        const SmemLayout L = smem_layout(p->BN, bits, p->s_p, p->rounds, pi.ks, pi.a_slots,
+                                         epi_slots(1, 3));
         if (L.total + 1024 <= 227u * 1024u) {
             p->b_res = 1;
             p->b_stages = p->rounds;
             p->epw = 3;
         }
     }
+    const SmemLayout Lj = smem_layout(pi.pair ? p->BN / 2 : p->BN, bits, p->s_p, p->b_stages, pi.ks,
+                                      pi.a_slots, epi_slots(1, p->epw));
+    p->join = Lj.total + 1024 <= 227u * 1024u;
 }
 
 // Run length of the coalesced A gather: the largest power of two of 16-byte
@@ -1315,7 +1349,8 @@ int launch_tc(const TcMaps &tmap, const TcParams &p, cudaStream_t s)
     if ((p.a_tma != 0) != A_TMA) return DSQ_ERR_UNSUPPORTED;
     constexpr bool PAIR = Pipe<PM>::PAIR;
     const SmemLayout L = smem_layout(PAIR ? p.BN / 2 : p.BN, BITS, p.s_p, p.b_stages,
-                                     Pipe<PM>::KS, Pipe<PM>::GROUPS * Pipe<PM>::A_RING, p.epw);
+                                     Pipe<PM>::KS, Pipe<PM>::GROUPS * Pipe<PM>::A_RING,
+                                     epi_slots(p.join, p.epw));
     if (L.total > 227u * 1024u) return DSQ_ERR_UNSUPPORTED;
     int smem_bytes = (int)L.total + 1024;            // slack for the 1024-byte alignment
     if (smem_bytes > 227 * 1024) smem_bytes = 227 * 1024;
