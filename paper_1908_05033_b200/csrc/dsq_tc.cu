@@ -66,17 +66,25 @@ constexpr int BK_BYTES = 128;         // int8 bytes per row per K step (128 code
 //         keeps the accumulators of its own 128 rows.  Per tensor-core clock
 //         every SM then expands half as much B, which is what bounds the
 //         single-CTA modes at wide N tiles.
+//   PM 5: KS = 5, 2 stages, two A groups, ONE round per tile ("whole K"): small
+//         convolutions (K <= 640 codes, e.g. 3x3 over 64 channels) with a
+//         resident B tile.  Every hand-off between the roles (a barrier wait, an
+//         expect, a TMA issue, a commit) costs a few hundred cycles whatever the
+//         amount of data behind it, so a tile pays for them once instead of
+//         once per K step; the two A groups take alternate tiles.
 constexpr int SU_MAX = 4;
 template <int PM> struct Pipe {
-    static constexpr int KS = PM == 1 ? 1 : 2;
+    static constexpr int KS = PM == 1 ? 1 : PM == 5 ? 5 : 2;
     static constexpr bool WIDE = PM == 3;
     static constexpr bool PAIR = PM == 4;
-    static constexpr int SU = PM == 1 ? 4 : PM == 3 ? 2 : 3;   // stages of expanded operands
+    static constexpr bool WHOLE_K = PM == 5;
+    // stages of expanded operands
+    static constexpr int SU = PM == 1 ? 4 : (PM == 3 || PM == 5) ? 2 : 3;
     static constexpr int GROUPS = WIDE ? 1 : 2;              // A groups in use
     static constexpr int A_D = PM == 1 ? 2 : 1;              // own A rounds in flight per thread
     static constexpr int A_RING = A_D + 1;                   // packed A ring slots per group
     static constexpr int A_COL0 = 512 - SU * 32 * KS;        // A stages: top TMEM columns
-    static constexpr int S_P = WIDE ? 2 : 3;                 // packed B ring slots
+    static constexpr int S_P = WHOLE_K ? 1 : WIDE ? 2 : 3;   // packed B ring slots
     // coalesced A gather (adjacent lanes fetch one row's contiguous chunks): fewer
     // memory requests, more instructions in the A threads; pays where the A
     // threads have slack
@@ -416,6 +424,15 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
             for (; g < n_b_steps; ++g) {
                 if (!wait_bar(bar_p_empty(s), ph ^ 1u, ctl, 1)) break;
                 mbar_arrive_expect_tx(bar_p_full(s), b_packed_bytes);
+                if (Pipe<PM>::WHOLE_K) {
+                    // a box is at most 256 bytes wide: one box per K step, stored
+                    // [K step][row][16 * BITS bytes]
+                    for (int h = 0; h < KS; ++h)
+                        tma_load_2d(smem_u32(smem + L.b_packed + s * b_packed_bytes) +
+                                        h * (BNL * 16 * BITS),
+                                    &tmap_b, (ks * KS + h) * (16 * BITS),
+                                    (tile % p.n_tiles) * BN + (int)rank * BNL, bar_p_full(s));
+                } else
                 tma_load_2d(smem_u32(smem + L.b_packed + s * b_packed_bytes), &tmap_b,
                             ks * (KS * 16 * BITS),
                             (tile % p.n_tiles) * BN + (int)rank * BNL, bar_p_full(s));
@@ -762,14 +779,34 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
                             *reinterpret_cast<uint4 *>(rowp + ((q ^ sw) << 4)) =
                                 expand3_chunk<B_SIGNED>(w, q, p.orv);
                     }
+                } else if (KS > 2) {
+                    // whole-K mode (resident tile, expanded once per CTA): K step
+                    // by K step, packed layout [K step][row][CH chunks]
+                    constexpr int OUT = Chunks<BITS>::OUT;
+#pragma unroll 1
+                    for (int h = 0; h < KS; ++h)
+#pragma unroll 1
+                        for (int r = row0; r < BNL; r += ROWS_PER_IT) {
+                            const uint4 v = reinterpret_cast<const uint4 *>(
+                                src)[(h * BNL + r) * CH + j];
+                            uint8_t *rowp = dst + h * b_sub_bytes + r * BK_BYTES;
+#pragma unroll
+                            for (int c = 0; c < OUT; ++c)
+                                *reinterpret_cast<uint4 *>(rowp + (((j * OUT + c) ^ sw) << 4)) =
+                                    make_uint4(expand_word<BITS, B_SIGNED>(v.x, c, p.orv),
+                                               expand_word<BITS, B_SIGNED>(v.y, c, p.orv),
+                                               expand_word<BITS, B_SIGNED>(v.z, c, p.orv),
+                                               expand_word<BITS, B_SIGNED>(v.w, c, p.orv));
+                        }
                 } else {
                     constexpr int OUT = Chunks<BITS>::OUT;
-                    uint4 v[MAX_IT][KS];
+                    constexpr int KSV = KS > 2 ? 1 : KS;   // (whole-K mode never gets here)
+                    uint4 v[MAX_IT][KSV];
 #pragma unroll
                     for (int i = 0; i < MAX_IT; ++i)
                         if (i < n_it && row0 + i * ROWS_PER_IT < BNL) {
 #pragma unroll
-                            for (int h = 0; h < KS; ++h)
+                            for (int h = 0; h < KSV; ++h)
                                 v[i][h] = reinterpret_cast<const uint4 *>(
                                     src)[(row0 + i * ROWS_PER_IT) * CHK + h * CH + j];
                         }
@@ -779,7 +816,7 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
                     for (int i = 0; i < MAX_IT; ++i) {
                         if (i < n_it && row0 + i * ROWS_PER_IT < BNL) {
 #pragma unroll
-                            for (int h = 0; h < KS; ++h)
+                            for (int h = 0; h < KSV; ++h)
 #pragma unroll
                                 for (int c = 0; c < OUT; ++c) {
                                     const uint4 o = make_uint4(
@@ -1199,10 +1236,11 @@ int make_rows_tmap(CUtensorMap *map, const void *base, uint64_t row_bytes, uint6
 // Resident B: one N tile and few K steps, so the expanded B tile of every K
 // step fits in shared memory next to the rings; it is then expanded once per
 // CTA instead of once per M tile.
-struct PipeInfo { int ks, su, a_slots, a_col0, s_p, wide, pair; };
+struct PipeInfo { int ks, su, a_slots, a_col0, s_p, wide, pair, whole_k; };
 PipeInfo pipe_info(int pm)
 {
     switch (pm) {
+    case 5: return {Pipe<5>::KS, Pipe<5>::SU, Pipe<5>::GROUPS * Pipe<5>::A_RING, Pipe<5>::A_COL0, Pipe<5>::S_P, 0, 0, 1};
     case 4: return {Pipe<4>::KS, Pipe<4>::SU, Pipe<4>::GROUPS * Pipe<4>::A_RING, Pipe<4>::A_COL0, Pipe<4>::S_P, 0, 1};
     case 1: return {Pipe<1>::KS, Pipe<1>::SU, Pipe<1>::GROUPS * Pipe<1>::A_RING, Pipe<1>::A_COL0, Pipe<1>::S_P, 0};
     case 2: return {Pipe<2>::KS, Pipe<2>::SU, Pipe<2>::GROUPS * Pipe<2>::A_RING, Pipe<2>::A_COL0, Pipe<2>::S_P, 0};
@@ -1230,6 +1268,7 @@ void choose_b_mode(TcParams *p, int bits, int pm)
             p->epw = 3;
         }
     }
+    if (pi.whole_k && !p->b_res) p->rounds = -1;     // the caller falls back to another mode
     const SmemLayout Lj = smem_layout(pi.pair ? p->BN / 2 : p->BN, bits, p->s_p, p->b_stages, pi.ks,
                                       pi.a_slots, epi_slots(1, p->epw));
     p->join = Lj.total + 1024 <= 227u * 1024u;
@@ -1420,6 +1459,13 @@ int launch_bits(int epi, int pm, const TcMaps &tmap, const TcParams &p, cudaStre
         if (pm == 2) return launch_tc<BITS, true, EPI_GEMM, 2, true>(tmap, p, s);
         return launch_tc<BITS, true, EPI_GEMM, 1, true>(tmap, p, s);
     }
+    if (pm == 5) {
+        switch (epi) {
+        case EPI_CODES: return launch_tc<BITS, false, EPI_CODES, 5, true>(tmap, p, s);
+        case EPI_CODES_RES: return launch_tc<BITS, false, EPI_CODES_RES, 5, true>(tmap, p, s);
+        default: return launch_tc<BITS, false, EPI_GENERAL, 5, true>(tmap, p, s);
+        }
+    }
     if (pm == 4) return launch_conv<BITS, 4>(epi, tmap, p, s);
     if (pm == 3) return launch_conv<BITS, 3>(epi, tmap, p, s);
     if (pm == 2) return launch_conv<BITS, 2>(epi, tmap, p, s);
@@ -1439,9 +1485,16 @@ int dispatch_tc(int bits, int epi, int pm, const TcMaps &tmap, const TcParams &p
 // single K steps, 2 forces double steps wherever they are possible.
 int g_forced_ks = 0;
 int g_pair_mode = 0;    // dsq_set_cta_pairs: 0 automatic, 1 never, 2 wherever possible
-int pick_pm(const TcParams &p, int bits)
+int pick_pm(const TcParams &p, int bits, bool im2col)
 {
     if (bits == 3 || p.ksteps < 2 || g_forced_ks == 1) return 1;
+    // whole-K rounds: a small convolution whose B tile can stay resident
+    if (im2col && g_forced_ks == 0 && p.ksteps >= 3 && p.ksteps <= Pipe<5>::KS &&
+        2 * p.BN <= Pipe<5>::A_COL0) {
+        TcParams q = p;
+        choose_b_mode(&q, bits, 5);
+        if (q.rounds == 1 && q.b_res) return 5;
+    }
     // CTA pairs: 256-wide N tiles and at least two 128-row tiles to put together
     if (p.BN == 256 && p.M > BM && g_pair_mode != 1) return 4;
     if (p.BN > 128) return p.ksteps >= 4 ? 3 : 1;
@@ -1504,8 +1557,8 @@ int dsq_gemm(const void *A_codes, const void *B_codes, int64_t M, int64_t N, int
     p.BN = pick_bn(p.m_tiles, (int)N, bits);
     if (bits == 2 && p.BN < 64) p.BN = 64;
     p.n_tiles = (int)((N + p.BN - 1) / p.BN);
-    const int pm = pick_pm(p, bits);
-    const int ks = pm == 1 ? 1 : 2;
+    const int pm = pick_pm(p, bits, false);
+    const int ks = pipe_info(pm).ks;
     if (pm == 4) p.m_tiles = (int)((M + 2 * BM - 1) / (2 * BM));
     choose_b_mode(&p, bits, pm);
     p.act = (const uint8_t *)A_codes;
@@ -1571,8 +1624,9 @@ int dsq_conv2d(const void *act_codes, const dsq_nhwc_t *shape, const dsq_quant_t
     p.m_tiles = (int)((M + BM - 1) / BM);
     p.BN = pick_bn(p.m_tiles, conv->Cout, bits);
     p.n_tiles = (conv->Cout + p.BN - 1) / p.BN;
-    const int pm = pick_pm(p, bits);
-    const int ks = pm == 1 ? 1 : 2;
+    const bool plain_rows = conv->KH == 1 && conv->stride == 1 && conv->pad == 0;
+    const int pm = pick_pm(p, bits, !plain_rows);
+    const int ks = pipe_info(pm).ks;
     if (pm == 4) p.m_tiles = (int)((M + 2 * BM - 1) / (2 * BM));
     choose_b_mode(&p, bits, pm);
     p.act = (const uint8_t *)act_codes;
@@ -1591,13 +1645,13 @@ int dsq_conv2d(const void *act_codes, const dsq_nhwc_t *shape, const dsq_quant_t
     }
     p.ws = (int *)workspace;
     TcMaps tmap;
+    // (whole-K rounds fetch B one K step per box)
     st = make_rows_tmap(&tmap.b, w_packed, row_bytes, (uint64_t)conv->Cout, row_bytes,
-                        ks * 16 * bits, pm == 4 ? p.BN / 2 : p.BN);
+                        (pm == 5 ? 1 : ks) * 16 * bits, pm == 4 ? p.BN / 2 : p.BN);
     if (st) return st;
     tmap.a = tmap.b;
     // a 1x1 stride-1 unpadded convolution reads the pixel rows as they lie
-    st = setup_a_tma(&p, &tmap.a, act_codes, M, bits, ks,
-                     conv->KH == 1 && conv->stride == 1 && conv->pad == 0, shape, conv->KH);
+    st = setup_a_tma(&p, &tmap.a, act_codes, M, bits, ks, plain_rows, shape, conv->KH);
     if (st) return st;
     // largest |2*acc + S_a| below 2^22: the epilogue may convert integers to
     // float through the 1.5 * 2^23 bias trick, which is exact there
