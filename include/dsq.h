@@ -278,6 +278,13 @@ int dsq_set_round_k_steps(int ks);
  * on it. */
 int dsq_set_cta_pairs(int mode);
 
+/* Fourth tuning hook: how dsq_gemm writes its int32 / fp32 outputs.  mode 0:
+ * automatic (each epilogue warp stages its 32 x 32 block in shared memory and
+ * one TMA store writes it, whenever N is a multiple of 4 and the staging tiles
+ * fit next to the operand rings), 1: always direct vector stores from the
+ * epilogue warps.  Results do not depend on it. */
+int dsq_set_gemm_store(int mode);
+
 /* ---- misc --------------------------------------------------------------- */
 const char *dsq_status_string(int status);
 int dsq_version(void);

@@ -170,6 +170,33 @@ __device__ __forceinline__ void tma_load_im2col_4d(uint32_t dst, const CUtensorM
         : "memory");
 }
 
+// 2-D tiled store, shared -> global, tracked by the issuing thread's bulk async
+// group.  Elements of the box outside the tensor are not written.  x * element
+// size must be a multiple of 16 bytes; neither coordinate may be negative.
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap *m, uint32_t src, int x, int y)
+{
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];" ::"l"(m),
+                 "r"(x), "r"(y), "r"(src)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_commit_group()
+{
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+// Waits until the bulk groups of this thread, except the newest N, have finished
+// READING their shared-memory source (the buffer may then be rewritten).
+template <int N>
+__device__ __forceinline__ void bulk_wait_group_read()
+{
+    asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void sts_128(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d)
+{
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c),
+                 "r"(d)
+                 : "memory");
+}
+
 // ---- tensor memory ---------------------------------------------------------
 // Executed by one full warp.  ncols: power of two, 32..512.  CG = 2: the
 // same warp of both CTAs of a pair executes it, and both get the same columns.

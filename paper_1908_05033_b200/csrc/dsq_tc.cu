@@ -124,6 +124,9 @@ struct TcParams {
     // join = 1: on the CTA's last tile the A and B warps join the epilogue (needs
     // a scale / bias staging slot for each of the 20 warps in shared memory)
     int join;
+    // stage = 1 (GEMM): the epilogue warps hand their 32 x 32 output blocks to TMA
+    // through a shared-memory staging tile instead of storing them themselves
+    int stage;
     int smem_bytes;                   // dynamic shared memory given to the launch
     // A gather geometry (a GEMM is a 1x1 convolution over an M x 1 image)
     const uint8_t *act;
@@ -267,7 +270,13 @@ constexpr int MAX_A_SLOTS = 6;
 constexpr int MAX_B_STAGES = 16;
 
 constexpr int JOIN_CNT = 5;               // warps per lane quarter in a joined epilogue
-__host__ __device__ inline int epi_slots(int join, int epw) { return join ? 4 * JOIN_CNT : 4 * epw; }
+// 256-byte slots behind the rings: scale / bias staging of the epilogue warps,
+// or (stage = 1, GEMM) one 4 KB output staging tile per epilogue warp, 1024-byte
+// aligned, from which TMA stores the int32 / fp32 rows
+__host__ __device__ inline int epi_slots(int join, int epw, int stage = 0)
+{
+    return stage ? 4 * epw * 16 + 4 : join ? 4 * JOIN_CNT : 4 * epw;
+}
 
 __host__ __device__ inline SmemLayout smem_layout(int BN, int bits, int s_p, int b_stages, int ks,
                                                 int a_slots, int epi_slots)
@@ -290,7 +299,9 @@ __host__ __device__ inline SmemLayout smem_layout(int BN, int bits, int s_p, int
 template <int BITS, bool A_SIGNED, int EPI, int PM, bool A_TMA>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
-              const __grid_constant__ CUtensorMap tmap_a, const TcParams p)
+              const __grid_constant__ CUtensorMap tmap_a,
+              const __grid_constant__ CUtensorMap tmap_c,
+              const __grid_constant__ CUtensorMap tmap_d, const TcParams p)
 {
     constexpr bool B_SIGNED = !A_SIGNED;
     constexpr int CH = Chunks<BITS>::CH;
@@ -311,7 +322,7 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
     const int BN = p.BN;
     const int BNL = BN / CG;                  // B rows this CTA expands
     const SmemLayout L =
-        smem_layout(BNL, BITS, p.s_p, p.b_stages, KS, GROUPS * A_RING, epi_slots(p.join, p.epw));
+        smem_layout(BNL, BITS, p.s_p, p.b_stages, KS, GROUPS * A_RING, epi_slots(p.join, p.epw, p.stage));
     // the layout must fit behind the 1024-byte aligned base (the host adds
     // slack only while it stays within the 227 KB limit); same answer in every
     // thread of every CTA, taken before any barrier exists
@@ -910,6 +921,42 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
                 }
                 tmem_ld_wait();
                 const int n0 = n_tile * BN + c0;
+                if (EPI == EPI_GEMM && p.stage) {
+                    // the warp's 32 rows x 32 columns go through a 128-byte-swizzled
+                    // staging tile to one TMA store (rows / columns past the matrix
+                    // are clipped by the store): the LSU sees 8 conflict-free shared
+                    // stores per lane instead of 32-byte pieces of 32 different lines
+                    const uint32_t stg =
+                        ((smem_u32(smem + L.epi) + 1023u) & ~1023u) +
+                        (uint32_t)(my_idx * 4 + quarter) * 4096u + (uint32_t)lane * 128u;
+                    const int y0 = m_tile * BMT + row_base + quarter * 32;
+#pragma unroll
+                    for (int c = 0; c < 32; ++c) r[c] = (uint32_t)((int)r[c] >> p.shift);
+#pragma unroll 1
+                    for (int o = 0; o < 2; ++o) {
+                        if (o == 0 ? p.C_i32 == nullptr : p.D_f32 == nullptr) continue;
+                        // the previous store has finished reading the tile
+                        if (lane == 0) bulk_wait_group_read<0>();
+                        __syncwarp();
+#pragma unroll
+                        for (int v = 0; v < 8; ++v) {
+                            uint32_t w[4];
+#pragma unroll
+                            for (int u = 0; u < 4; ++u)
+                                w[u] = o == 0 ? r[4 * v + u]
+                                              : __float_as_uint(
+                                                    __fmul_rn((float)(int)r[4 * v + u], rs));
+                            sts_128(stg + (uint32_t)((v ^ (lane & 7)) << 4), w[0], w[1], w[2], w[3]);
+                        }
+                        fence_proxy_async_smem();
+                        __syncwarp();
+                        if (lane == 0) {
+                            tma_store_2d(o == 0 ? &tmap_c : &tmap_d, stg, n0, y0);
+                            bulk_commit_group();
+                        }
+                    }
+                    continue;
+                }
                 if (!row_ok) continue;
 #pragma unroll
                 for (int c = 0; c < 32; ++c) r[c] = (uint32_t)((int)r[c] >> p.shift);
@@ -1117,6 +1164,8 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
     }
 
     // ---------------- teardown ---------------------------------------------
+    // (staged output tiles must have been read before the shared memory goes)
+    if (EPI == EPI_GEMM && p.stage && lane == 0) bulk_wait_group_read<0>();
     tc_fence_before_sync();
     __syncthreads();
     // a CTA of a pair stays until its peer has stopped signalling its barriers
@@ -1214,7 +1263,7 @@ EncodeTiledFn get_encode_fn()
 }
 
 // 2-D byte map over packed rows: inner dimension = row bytes, outer = rows.
-struct TcMaps { CUtensorMap b, a; };
+struct TcMaps { CUtensorMap b, a, c, d; };   // operands; GEMM outputs (int32 C, fp32 D)
 
 int make_rows_tmap(CUtensorMap *map, const void *base, uint64_t row_bytes, uint64_t rows,
                    uint64_t pitch, uint32_t box_bytes, uint32_t box_rows,
@@ -1230,6 +1279,22 @@ int make_rows_tmap(CUtensorMap *map, const void *base, uint64_t row_bytes, uint6
                     strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                     swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? DSQ_OK : DSQ_ERR_CUDA;
+}
+
+// Row-major M x N matrix of 4-byte elements, written in boxes of 32 x 32 from a
+// 128-byte-swizzled shared tile.
+int make_out_tmap(CUtensorMap *map, void *base, CUtensorMapDataType dtype, int64_t M, int64_t N)
+{
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return DSQ_ERR_CUDA;
+    cuuint64_t dims[2] = {(cuuint64_t)N, (cuuint64_t)M};
+    cuuint64_t strides[1] = {(cuuint64_t)N * 4};
+    cuuint32_t box[2] = {32, 32};
+    cuuint32_t estr[2] = {1, 1};
+    const CUresult r = fn(map, dtype, 2, base, dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                          CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? DSQ_OK : DSQ_ERR_CUDA;
 }
 
@@ -1389,7 +1454,7 @@ int launch_tc(const TcMaps &tmap, const TcParams &p, cudaStream_t s)
     constexpr bool PAIR = Pipe<PM>::PAIR;
     const SmemLayout L = smem_layout(PAIR ? p.BN / 2 : p.BN, BITS, p.s_p, p.b_stages,
                                      Pipe<PM>::KS, Pipe<PM>::GROUPS * Pipe<PM>::A_RING,
-                                     epi_slots(p.join, p.epw));
+                                     epi_slots(p.join, p.epw, p.stage));
     if (L.total > 227u * 1024u) return DSQ_ERR_UNSUPPORTED;
     int smem_bytes = (int)L.total + 1024;            // slack for the 1024-byte alignment
     if (smem_bytes > 227 * 1024) smem_bytes = 227 * 1024;
@@ -1421,14 +1486,14 @@ int launch_tc(const TcMaps &tmap, const TcParams &p, cudaStream_t s)
         attr[0].val.clusterDim.z = 1;
         cfg.attrs = attr;
         cfg.numAttrs = 1;
-        if (cudaLaunchKernelEx(&cfg, dsq_tc_kernel<BITS, A_SIGNED, EPI, PM, A_TMA>, tmap.b, tmap.a, q) !=
+        if (cudaLaunchKernelEx(&cfg, dsq_tc_kernel<BITS, A_SIGNED, EPI, PM, A_TMA>, tmap.b, tmap.a, tmap.c, tmap.d, q) !=
             cudaSuccess) {
             cudaGetLastError();
             return DSQ_ERR_CUDA;
         }
         return dsq_launch_status();
     }
-    dsq_tc_kernel<BITS, A_SIGNED, EPI, PM, A_TMA><<<grid, NUM_THREADS, smem_bytes, s>>>(tmap.b, tmap.a, q);
+    dsq_tc_kernel<BITS, A_SIGNED, EPI, PM, A_TMA><<<grid, NUM_THREADS, smem_bytes, s>>>(tmap.b, tmap.a, tmap.c, tmap.d, q);
     return dsq_launch_status();
 }
 
@@ -1485,6 +1550,7 @@ int dispatch_tc(int bits, int epi, int pm, const TcMaps &tmap, const TcParams &p
 // single K steps, 2 forces double steps wherever they are possible.
 int g_forced_ks = 0;
 int g_pair_mode = 0;    // dsq_set_cta_pairs: 0 automatic, 1 never, 2 wherever possible
+int g_stage_mode = 0;   // dsq_set_gemm_store: 0 automatic (TMA stores where possible), 1 direct stores
 int pick_pm(const TcParams &p, int bits, bool im2col)
 {
     if (bits == 3 || p.ksteps < 2 || g_forced_ks == 1) return 1;
@@ -1521,6 +1587,13 @@ int dsq_set_cta_pairs(int mode)
 {
     if (mode < 0 || mode > 2) return DSQ_ERR_SHAPE;
     g_pair_mode = mode;
+    return DSQ_OK;
+}
+
+int dsq_set_gemm_store(int mode)
+{
+    if (mode != 0 && mode != 1) return DSQ_ERR_SHAPE;
+    g_stage_mode = mode;
     return DSQ_OK;
 }
 
@@ -1579,6 +1652,27 @@ int dsq_gemm(const void *A_codes, const void *B_codes, int64_t M, int64_t N, int
     tmap.a = tmap.b;
     st = setup_a_tma(&p, &tmap.a, A_codes, M, bits, ks, true, nullptr, 1);
     if (st) return st;
+    tmap.c = tmap.b;
+    tmap.d = tmap.b;
+    // outputs through TMA stores when their rows are 16-byte multiples and the
+    // staging tiles fit in shared memory
+    if (g_stage_mode != 1 && N % 4 == 0) {
+        const PipeInfo pi = pipe_info(pm);
+        const SmemLayout Ls = smem_layout(pi.pair ? p.BN / 2 : p.BN, bits, p.s_p, p.b_stages, pi.ks,
+                                          pi.a_slots, epi_slots(0, p.epw, 1));
+        if (Ls.total + 1024 <= 227u * 1024u) {
+            p.stage = 1;
+            p.join = 0;
+            if (C_i32) {
+                st = make_out_tmap(&tmap.c, C_i32, CU_TENSOR_MAP_DATA_TYPE_INT32, M, N);
+                if (st) return st;
+            }
+            if (D_f32) {
+                st = make_out_tmap(&tmap.d, D_f32, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, M, N);
+                if (st) return st;
+            }
+        }
+    }
     return dispatch_tc(bits, EPI_GEMM, pm, tmap, p, (cudaStream_t)stream);
 }
 

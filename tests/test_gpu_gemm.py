@@ -28,7 +28,8 @@ def run(dsq, A, B, rs, bits):
 
 
 SIZES = [(1, 1, 1), (128, 32, 128), (128, 256, 128), (130, 70, 200),
-         (300, 257, 1000), (129, 513, 129), (64, 48, 4096), (515, 130, 771)]
+         (300, 257, 1000), (129, 513, 129), (64, 48, 4096), (515, 130, 771),
+         (130, 72, 200), (300, 260, 1000), (257, 516, 300)]
 
 
 @pytest.mark.parametrize("bits", [2, 3, 4])
@@ -38,6 +39,23 @@ def test_gemm_small_and_ragged(dsq, bits, size):
     A, B, rs = dsq_inputs.gemm_case(M, Nn, K, bits)
     C = native.gemm(A, B)
     Cg, Dg = run(dsq, A, B, rs, bits)
+    assert np.array_equal(C, Cg)
+    assert np.array_equal(native.gemm_dequant(C, rs), Dg)
+
+
+@pytest.mark.parametrize("bits", [2, 4])
+@pytest.mark.parametrize("size", [(130, 72, 200), (300, 260, 1000), (512, 512, 512)])
+def test_gemm_direct_stores(dsq, bits, size):
+    """Same results when the epilogue warps store the outputs themselves
+    instead of handing staged tiles to TMA."""
+    M, Nn, K = size
+    A, B, rs = dsq_inputs.gemm_case(M, Nn, K, bits)
+    C = native.gemm(A, B)
+    dsq.dsq_set_gemm_store(1)
+    try:
+        Cg, Dg = run(dsq, A, B, rs, bits)
+    finally:
+        dsq.dsq_set_gemm_store(0)
     assert np.array_equal(C, Cg)
     assert np.array_equal(native.gemm_dequant(C, rs), Dg)
 
