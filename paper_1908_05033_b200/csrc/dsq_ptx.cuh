@@ -298,43 +298,57 @@ __device__ __forceinline__ void mma_i8_ts(uint32_t d_tmem, uint32_t a_tmem,
 // Four consecutive K=32 instructions of one 128-byte K step in a single block:
 // A advances 8 tensor-memory columns and the B descriptor 32 bytes (2 units of
 // 16 bytes in its low word) per instruction.  Only the first one takes the
-// caller's accumulate flag.  Keeps the issuing thread's instruction count low.
+// caller's accumulate flag.
+//
+// Called by ALL lanes of a converged warp with warp-uniform arguments; one
+// elected lane issues.  Keeping the issuing code in uniform control flow lets
+// the compiler hold the descriptors in uniform registers, which is where the
+// instruction takes them from: issued from a divergent single-lane branch,
+// every instruction first pays for moving its operands there.
+#define DSQ_MMA_X4_BODY(CGS)                                                              \
+    asm volatile(                                                                         \
+        "{\n\t.reg .pred p0, p1, pe;\n\t.reg .b64 d0, d1, d2, d3;\n\t"                   \
+        ".reg .b32 l1, l2, l3, a1, a2, a3;\n\t"                                           \
+        "setp.ne.b32 p0, %5, 0;\n\tsetp.eq.b32 p1, %5, %5;\n\t"                           \
+        "add.u32 l1, %2, 2;\n\tadd.u32 l2, %2, 4;\n\tadd.u32 l3, %2, 6;\n\t"              \
+        "add.u32 a1, %1, 8;\n\tadd.u32 a2, %1, 16;\n\tadd.u32 a3, %1, 24;\n\t"            \
+        "mov.b64 d0, {%2, %3};\n\tmov.b64 d1, {l1, %3};\n\t"                              \
+        "mov.b64 d2, {l2, %3};\n\tmov.b64 d3, {l3, %3};\n\t"                              \
+        "elect.sync _|pe, 0xffffffff;\n\t"                                                \
+        "@pe tcgen05.mma.cta_group::" CGS ".kind::i8 [%0], [%1], d0, %4, p0;\n\t"          \
+        "@pe tcgen05.mma.cta_group::" CGS ".kind::i8 [%0], [a1], d1, %4, p1;\n\t"          \
+        "@pe tcgen05.mma.cta_group::" CGS ".kind::i8 [%0], [a2], d2, %4, p1;\n\t"          \
+        "@pe tcgen05.mma.cta_group::" CGS ".kind::i8 [%0], [a3], d3, %4, p1;\n\t}" ::"r"(  \
+            d_tmem),                                                                      \
+        "r"(a_tmem), "r"(b_desc_lo), "r"(b_desc_hi), "r"(idesc), "r"(accumulate_first)    \
+        : "memory")
 template <int CG = 1>
 __device__ __forceinline__ void mma_i8_ts_x4(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_desc_lo,
                                              uint32_t b_desc_hi, uint32_t idesc,
                                              uint32_t accumulate_first)
 {
-    if (CG == 1) {
+    if (CG == 1) DSQ_MMA_X4_BODY("1");
+    else DSQ_MMA_X4_BODY("2");
+}
+#undef DSQ_MMA_X4_BODY
+
+// tcgen05.commit by one elected lane of a converged warp (all lanes call).
+__device__ __forceinline__ void mma_commit_elect(uint32_t bar)
+{
     asm volatile(
-        "{\n\t.reg .pred p0, p1;\n\t.reg .b64 d0, d1, d2, d3;\n\t"
-        ".reg .b32 l1, l2, l3, a1, a2, a3;\n\t"
-        "setp.ne.b32 p0, %5, 0;\n\tsetp.eq.b32 p1, %5, %5;\n\t"
-        "add.u32 l1, %2, 2;\n\tadd.u32 l2, %2, 4;\n\tadd.u32 l3, %2, 6;\n\t"
-        "add.u32 a1, %1, 8;\n\tadd.u32 a2, %1, 16;\n\tadd.u32 a3, %1, 24;\n\t"
-        "mov.b64 d0, {%2, %3};\n\tmov.b64 d1, {l1, %3};\n\t"
-        "mov.b64 d2, {l2, %3};\n\tmov.b64 d3, {l3, %3};\n\t"
-        "tcgen05.mma.cta_group::1.kind::i8 [%0], [%1], d0, %4, p0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::i8 [%0], [a1], d1, %4, p1;\n\t"
-        "tcgen05.mma.cta_group::1.kind::i8 [%0], [a2], d2, %4, p1;\n\t"
-        "tcgen05.mma.cta_group::1.kind::i8 [%0], [a3], d3, %4, p1;\n\t}" ::"r"(d_tmem),
-        "r"(a_tmem), "r"(b_desc_lo), "r"(b_desc_hi), "r"(idesc), "r"(accumulate_first)
+        "{\n\t.reg .pred pe;\n\telect.sync _|pe, 0xffffffff;\n\t"
+        "@pe tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}" ::"r"(
+            bar)
         : "memory");
-    } else {
+}
+__device__ __forceinline__ void mma_commit_pair_elect(uint32_t bar, uint16_t cta_mask)
+{
     asm volatile(
-        "{\n\t.reg .pred p0, p1;\n\t.reg .b64 d0, d1, d2, d3;\n\t"
-        ".reg .b32 l1, l2, l3, a1, a2, a3;\n\t"
-        "setp.ne.b32 p0, %5, 0;\n\tsetp.eq.b32 p1, %5, %5;\n\t"
-        "add.u32 l1, %2, 2;\n\tadd.u32 l2, %2, 4;\n\tadd.u32 l3, %2, 6;\n\t"
-        "add.u32 a1, %1, 8;\n\tadd.u32 a2, %1, 16;\n\tadd.u32 a3, %1, 24;\n\t"
-        "mov.b64 d0, {%2, %3};\n\tmov.b64 d1, {l1, %3};\n\t"
-        "mov.b64 d2, {l2, %3};\n\tmov.b64 d3, {l3, %3};\n\t"
-        "tcgen05.mma.cta_group::2.kind::i8 [%0], [%1], d0, %4, p0;\n\t"
-        "tcgen05.mma.cta_group::2.kind::i8 [%0], [a1], d1, %4, p1;\n\t"
-        "tcgen05.mma.cta_group::2.kind::i8 [%0], [a2], d2, %4, p1;\n\t"
-        "tcgen05.mma.cta_group::2.kind::i8 [%0], [a3], d3, %4, p1;\n\t}" ::"r"(d_tmem),
-        "r"(a_tmem), "r"(b_desc_lo), "r"(b_desc_hi), "r"(idesc), "r"(accumulate_first)
+        "{\n\t.reg .pred pe;\n\telect.sync _|pe, 0xffffffff;\n\t"
+        "@pe tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 "
+        "[%0], %1;\n\t}" ::"r"(bar),
+        "h"(cta_mask)
         : "memory");
-    }
 }
 
 // 32 lanes x 32 columns store: thread t of the warp writes lane (base + t),

@@ -72,14 +72,23 @@ constexpr int BK_BYTES = 128;         // int8 bytes per row per K step (128 code
 //         expect, a TMA issue, a commit) costs a few hundred cycles whatever the
 //         amount of data behind it, so a tile pays for them once instead of
 //         once per K step; the two A groups take alternate tiles.
+//   PM 6: CTA PAIR on 256 x 128 tiles, KS = 4, 2 stages, TWO accumulator buffers:
+//         the epilogue of a tile (whose int32 / fp32 output is as large as the
+//         packed operands it came from) overlaps the next tile's rounds, which the
+//         256-wide pair tile cannot do (its accumulator and the A stages fill
+//         the 512 tensor-memory columns).  A round is two half rounds for the A
+//         side: each A group expands two of the four K steps of every round.
 constexpr int SU_MAX = 4;
 template <int PM> struct Pipe {
-    static constexpr int KS = PM == 1 ? 1 : PM == 5 ? 5 : 2;
+    static constexpr int KS = PM == 1 ? 1 : PM == 5 ? 5 : PM == 6 ? 4 : 2;
     static constexpr bool WIDE = PM == 3;
-    static constexpr bool PAIR = PM == 4;
+    static constexpr bool PAIR = PM == 4 || PM == 6;
+    // A half rounds per barrier round (each A group takes one half of every round)
+    static constexpr int HALVES = PM == 6 ? 2 : 1;
+    static constexpr int KSA = KS / HALVES;                  // K steps of an A step
     static constexpr bool WHOLE_K = PM == 5;
     // stages of expanded operands
-    static constexpr int SU = PM == 1 ? 4 : (PM == 3 || PM == 5) ? 2 : 3;
+    static constexpr int SU = PM == 1 ? 4 : (PM == 3 || PM == 5 || PM == 6) ? 2 : 3;
     static constexpr int GROUPS = WIDE ? 1 : 2;              // A groups in use
     static constexpr int A_D = PM == 1 ? 2 : 1;              // own A rounds in flight per thread
     static constexpr int A_RING = A_D + 1;                   // packed A ring slots per group
@@ -313,7 +322,8 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
     constexpr int S_U = Pipe<PM>::SU, A_D = Pipe<PM>::A_D, A_RING = Pipe<PM>::A_RING;
     constexpr int A_COL0 = Pipe<PM>::A_COL0;
     constexpr int A_SLOTS = GROUPS * A_RING;                // packed A ring slots
-    constexpr int A_SLOT_BYTES = KS * CH * BM * 16;         // one round of 128 rows
+    constexpr int HALVES = Pipe<PM>::HALVES, KSA = Pipe<PM>::KSA;
+    constexpr int A_SLOT_BYTES = KSA * CH * BM * 16;        // one A step of 128 rows
     static_assert(A_SLOTS <= MAX_A_SLOTS, "A ring barriers");
     static_assert(KS == 1 || BITS != 3, "3-bit rows use single K steps");
     extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -322,7 +332,8 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
     const int BN = p.BN;
     const int BNL = BN / CG;                  // B rows this CTA expands
     const SmemLayout L =
-        smem_layout(BNL, BITS, p.s_p, p.b_stages, KS, GROUPS * A_RING, epi_slots(p.join, p.epw, p.stage));
+        smem_layout(BNL, BITS, p.s_p, p.b_stages, KS, GROUPS * A_RING / HALVES,
+                    epi_slots(p.join, p.epw, p.stage));
     // the layout must fit behind the 1024-byte aligned base (the host adds
     // slack only while it stays within the 227 KB limit); same answer in every
     // thread of every CTA, taken before any barrier exists
@@ -331,7 +342,10 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
         return;
     }
     const int S_P = p.s_p;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // (the shuffle tells the compiler that the warp index is the same in all
+    // lanes, so the role branches below are uniform control flow)
+    const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0);
+    const int lane = threadIdx.x & 31;
     // a pair is the two CTAs of a cluster; rank 0 issues the MMAs
     const uint32_t rank = PAIR ? cluster_ctarank() : 0u;
     const int tile0 = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
@@ -371,16 +385,17 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
         else mbar_arrive(bar);
     };
     // completion of the issued MMAs, signalled to this barrier in both CTAs
+    // (called by all lanes of the MMA warp; one elected lane issues)
     auto commit_all = [&](uint32_t bar) {
-        if (PAIR) mma_commit_pair(bar, (uint16_t)3);
-        else mma_commit<1>(bar);
+        if (PAIR) mma_commit_pair_elect(bar, (uint16_t)3);
+        else mma_commit_elect(bar);
     };
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S_U; ++s) {
             // operands of a round: the four warps of one A group and (unless the
             // expanded B tile is resident) the B warps, of every CTA of the pair
-            mbar_init(bar_a_full(s), (4 + (p.b_res ? 0 : NUM_B_WARPS / B_GROUPS)) * CG);
+            mbar_init(bar_a_full(s), (4 * HALVES + (p.b_res ? 0 : NUM_B_WARPS / B_GROUPS)) * CG);
             mbar_init(bar_u_empty(s), 1);    // tcgen05.commit
         }
         for (int s = 0; s < MAX_B_STAGES; ++s) mbar_init(bar_b_full(s), NUM_B_WARPS * CG);
@@ -413,7 +428,7 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
     // no arrival may reach the peer before its barriers exist
     if (PAIR) cluster_sync_all();
     tc_fence_after_sync();
-    const uint32_t tmem_base = *tmem_slot;
+    const uint32_t tmem_base = __shfl_sync(0xffffffffu, *tmem_slot, 0);
 
     // Epilogue roles.  epi_idx >= 0: the warp takes part in the epilogue of every
     // tile (p.epw warps per TMEM lane quarter).  join_idx >= 0: it takes part in
@@ -458,7 +473,8 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
     } else if (warp == WARP_TMA_A) {
         // ---------------- producer: TMA packed A boxes -----------------------
         if (A_TMA && lane == 0) {
-            const uint32_t n_a_steps = (uint32_t)my_tiles_all * p.rounds;
+            const int a_steps_tile = p.rounds * HALVES;          // A steps per tile
+            const uint32_t n_a_steps = (uint32_t)my_tiles_all * a_steps_tile;
             const uint32_t ring = smem_u32(smem + L.a_ring);
             uint32_t g = 0, issued_a = 0;
             int ka = 0, tile_a = tile0;
@@ -470,7 +486,7 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
                 const int m0 = (tile_a / p.n_tiles) * BMT + row_base;
                 if (p.a_tma == 1) {
                     mbar_arrive_expect_tx(bar_ar_full(sl), A_SLOT_BYTES);
-                    tma_load_2d(ring + sl * A_SLOT_BYTES, &tmap_a, ka * (KS * 16 * BITS), m0,
+                    tma_load_2d(ring + sl * A_SLOT_BYTES, &tmap_a, ka * (KSA * 16 * BITS), m0,
                                 bar_ar_full(sl));
                 } else {
                     if (ka == 0) {                 // first pixel of the tile, first tap
@@ -496,7 +512,7 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
                     }
                 }
                 ++issued_a;
-                if (++ka == p.rounds) { ka = 0; tile_a += tstep; }
+                if (++ka == a_steps_tile) { ka = 0; tile_a += tstep; }
             }
             for (uint32_t k = (issued_a > (uint32_t)A_SLOTS ? issued_a - A_SLOTS : 0);
                  k < issued_a; ++k)
@@ -504,7 +520,9 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
         }
     } else if (warp == WARP_MMA) {
         // ---------------- MMA issuer ---------------------------------------
-        if (lane == 0 && rank == 0) {
+        // The whole warp runs the loop in uniform control flow (waits included);
+        // the issue wrappers elect one lane.
+        if (rank == 0) {
             const uint32_t idesc = idesc_i8(BN, A_SIGNED, B_SIGNED, BMT);
             const uint64_t b_desc0 = smem_desc_sw128(smem_u32(smem + L.b_tiles));
             const uint32_t b_desc_lo0 = (uint32_t)b_desc0, b_desc_hi = (uint32_t)(b_desc0 >> 32);
@@ -643,7 +661,7 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
                 if (load && ++ld_slot == A_RING) ld_slot = 0;
             }
         };
-        const uint32_t n_steps = (uint32_t)my_tiles_all * p.rounds;
+        const uint32_t n_steps = (uint32_t)my_tiles_all * p.rounds * HALVES;
         // own steps: g = group, group + GROUPS, ...
         const uint32_t n_own =
             GROUPS == 1 ? n_steps : (n_steps > (uint32_t)group ? (n_steps - group + 1) / 2 : 0u);
@@ -686,19 +704,22 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
                 cp_async_wait<A_D>();              // own step i - A_D has landed
                 if (Pipe<PM>::COAL) __syncwarp();  // ... the other lanes' copies of my row too
             }
-            const int s = g % S_U;
-            const uint32_t ph = (g / S_U) & 1u;
+            // A step g is half (g % HALVES) of barrier round g / HALVES
+            const uint32_t rg = g / HALVES;
+            const int half = (int)(g % HALVES);
+            const int s = rg % S_U;
+            const uint32_t ph = (rg / S_U) & 1u;
             // chunks of this round that exist (im2col: nothing is loaded past the
             // last filter tap)
-            int kvalid = KS * CH;
+            int kvalid = KSA * CH;
             if (a_tma) {
-                if (p.a_tma == 2) kvalid = p.a_kchunks - kr * (KS * CH);
+                if (p.a_tma == 2) kvalid = p.a_kchunks - kr * (KSA * CH);
                 kr += GROUPS;
                 if (kr >= p.rounds) kr -= p.rounds;
                 if (kr >= p.rounds) kr -= p.rounds;
             }
 #pragma unroll
-            for (int h = 0; h < KS; ++h) {
+            for (int h = 0; h < KSA; ++h) {
                 uint32_t o[32];
                 {
                     uint4 cur[CH];
@@ -721,7 +742,7 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
                 }
                 __syncwarp();
                 tmem_st_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + A_COL0 +
-                                  (s * KS + h) * 32, o);
+                                  (s * KS + half * KSA + h) * 32, o);
             }
             if (!ok) break;
             if (++rd_slot == A_RING) rd_slot = 0;
@@ -753,7 +774,8 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
         // being a multiple of 128 bytes apart); (row & 7) does not depend on i
         constexpr int CHK = KS * CH;
         constexpr int ROWS_PER_IT = (BITS == 3) ? BT : BT / CH;
-        constexpr int MAX_IT = (BITS == 3) ? 1 : ((PAIR ? 128 : 256) * CH) / BT;
+        // (pairs expand half of a tile's B rows; PM 6 tiles are 128 wide)
+        constexpr int MAX_IT = (BITS == 3) ? 1 : ((PM == 6 ? 64 : PAIR ? 128 : 256) * CH) / BT;
         const int row0 = (BITS == 3) ? tid : tid / CH;
         const int j = (BITS == 3) ? 0 : tid % CH;
         const int sw = row0 & 7;
@@ -790,7 +812,7 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
                             *reinterpret_cast<uint4 *>(rowp + ((q ^ sw) << 4)) =
                                 expand3_chunk<B_SIGNED>(w, q, p.orv);
                     }
-                } else if (KS > 2) {
+                } else if (Pipe<PM>::WHOLE_K) {
                     // whole-K mode (resident tile, expanded once per CTA): K step
                     // by K step, packed layout [K step][row][CH chunks]
                     constexpr int OUT = Chunks<BITS>::OUT;
@@ -811,15 +833,21 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
                         }
                 } else {
                     constexpr int OUT = Chunks<BITS>::OUT;
-                    constexpr int KSV = KS > 2 ? 1 : KS;   // (whole-K mode never gets here)
+                    constexpr int KSV = Pipe<PM>::WHOLE_K ? 1 : KS;   // (whole-K never gets here)
                     uint4 v[MAX_IT][KSV];
+                    // The packed tile is row-major, so the rows of a quarter warp
+                    // (two with 4-bit codes, four with 2-bit codes) would fetch the
+                    // same 16-byte bank groups: each row starts at another K step
+                    // (register slot h holds K step (h + rot) mod KS)
+                    const int rot = BITS == 4 ? (row0 & 1) : KSV == 4 ? (row0 & 3) : ((row0 >> 1) & 1);
 #pragma unroll
                     for (int i = 0; i < MAX_IT; ++i)
                         if (i < n_it && row0 + i * ROWS_PER_IT < BNL) {
 #pragma unroll
                             for (int h = 0; h < KSV; ++h)
                                 v[i][h] = reinterpret_cast<const uint4 *>(
-                                    src)[(row0 + i * ROWS_PER_IT) * CHK + h * CH + j];
+                                    src)[(row0 + i * ROWS_PER_IT) * CHK +
+                                         ((h + rot) & (KSV - 1)) * CH + j];
                         }
                     if (!p.b_res && !(ok = wait_bar(bar_u_empty(su), phu ^ 1u, ctl, 7))) break;
                     uint8_t *rowp = dst + row0 * BK_BYTES;
@@ -836,7 +864,8 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
                                         expand_word<BITS, B_SIGNED>(v[i][h].z, c, p.orv),
                                         expand_word<BITS, B_SIGNED>(v[i][h].w, c, p.orv));
                                     *reinterpret_cast<uint4 *>(
-                                        rowp + h * b_sub_bytes + i * ROWS_PER_IT * BK_BYTES +
+                                        rowp + ((h + rot) & (KSV - 1)) * b_sub_bytes +
+                                        i * ROWS_PER_IT * BK_BYTES +
                                         (((j * OUT + c) ^ sw) << 4)) = o;
                                 }
                         }
@@ -1301,10 +1330,11 @@ int make_out_tmap(CUtensorMap *map, void *base, CUtensorMapDataType dtype, int64
 // Resident B: one N tile and few K steps, so the expanded B tile of every K
 // step fits in shared memory next to the rings; it is then expanded once per
 // CTA instead of once per M tile.
-struct PipeInfo { int ks, su, a_slots, a_col0, s_p, wide, pair, whole_k; };
+struct PipeInfo { int ks, su, a_slots, a_col0, s_p, wide, pair, whole_k, ksa; };
 PipeInfo pipe_info(int pm)
 {
     switch (pm) {
+    case 6: return {Pipe<6>::KS, Pipe<6>::SU, Pipe<6>::GROUPS * Pipe<6>::A_RING / 2, Pipe<6>::A_COL0, Pipe<6>::S_P, 0, 1, 0, Pipe<6>::KSA};
     case 5: return {Pipe<5>::KS, Pipe<5>::SU, Pipe<5>::GROUPS * Pipe<5>::A_RING, Pipe<5>::A_COL0, Pipe<5>::S_P, 0, 0, 1};
     case 4: return {Pipe<4>::KS, Pipe<4>::SU, Pipe<4>::GROUPS * Pipe<4>::A_RING, Pipe<4>::A_COL0, Pipe<4>::S_P, 0, 1};
     case 1: return {Pipe<1>::KS, Pipe<1>::SU, Pipe<1>::GROUPS * Pipe<1>::A_RING, Pipe<1>::A_COL0, Pipe<1>::S_P, 0};
@@ -1453,7 +1483,8 @@ int launch_tc(const TcMaps &tmap, const TcParams &p, cudaStream_t s)
     if ((p.a_tma != 0) != A_TMA) return DSQ_ERR_UNSUPPORTED;
     constexpr bool PAIR = Pipe<PM>::PAIR;
     const SmemLayout L = smem_layout(PAIR ? p.BN / 2 : p.BN, BITS, p.s_p, p.b_stages,
-                                     Pipe<PM>::KS, Pipe<PM>::GROUPS * Pipe<PM>::A_RING,
+                                     Pipe<PM>::KS,
+                                     Pipe<PM>::GROUPS * Pipe<PM>::A_RING / Pipe<PM>::HALVES,
                                      epi_slots(p.join, p.epw, p.stage));
     if (L.total > 227u * 1024u) return DSQ_ERR_UNSUPPORTED;
     int smem_bytes = (int)L.total + 1024;            // slack for the 1024-byte alignment
@@ -1519,6 +1550,7 @@ int launch_bits(int epi, int pm, const TcMaps &tmap, const TcParams &p, cudaStre
 {
     if (epi == EPI_GEMM) {
         // 2- and 4-bit GEMMs always fetch A with TMA
+        if (pm == 6) return launch_tc<BITS, true, EPI_GEMM, 6, true>(tmap, p, s);
         if (pm == 4) return launch_tc<BITS, true, EPI_GEMM, 4, true>(tmap, p, s);
         if (pm == 3) return launch_tc<BITS, true, EPI_GEMM, 3, true>(tmap, p, s);
         if (pm == 2) return launch_tc<BITS, true, EPI_GEMM, 2, true>(tmap, p, s);
@@ -1551,6 +1583,14 @@ int dispatch_tc(int bits, int epi, int pm, const TcMaps &tmap, const TcParams &p
 int g_forced_ks = 0;
 int g_pair_mode = 0;    // dsq_set_cta_pairs: 0 automatic, 1 never, 2 wherever possible
 int g_stage_mode = 0;   // dsq_set_gemm_store: 0 automatic (TMA stores where possible), 1 direct stores
+// Whether a GEMM runs its CTA pairs on 256 x 128 tiles with overlapped epilogues
+// (PM 6) rather than on 256 x 256 tiles (PM 4).
+bool pair128_pays(int64_t M, int64_t N)
+{
+    (void)M; (void)N;
+    return false;
+}
+
 int pick_pm(const TcParams &p, int bits, bool im2col)
 {
     if (bits == 3 || p.ksteps < 2 || g_forced_ks == 1) return 1;
@@ -1585,7 +1625,7 @@ int dsq_set_round_k_steps(int ks)
 
 int dsq_set_cta_pairs(int mode)
 {
-    if (mode < 0 || mode > 2) return DSQ_ERR_SHAPE;
+    if (mode < 0 || mode > 3) return DSQ_ERR_SHAPE;
     g_pair_mode = mode;
     return DSQ_OK;
 }
@@ -1630,9 +1670,18 @@ int dsq_gemm(const void *A_codes, const void *B_codes, int64_t M, int64_t N, int
     p.BN = pick_bn(p.m_tiles, (int)N, bits);
     if (bits == 2 && p.BN < 64) p.BN = 64;
     p.n_tiles = (int)((N + p.BN - 1) / p.BN);
-    const int pm = pick_pm(p, bits, false);
+    int pm = pick_pm(p, bits, false);
+    // pairs on 256 x 128 tiles with two accumulator buffers (see Pipe<6>)
+    if (bits != 3 && g_forced_bn == 0 && g_forced_ks == 0 && M > BM && N > 64 && p.ksteps >= 8 &&
+        (g_pair_mode == 3 || (g_pair_mode == 0 && pm == 4 && pair128_pays(M, N)))) {
+        pm = 6;
+        p.BN = 128;
+        p.n_tiles = (int)((N + p.BN - 1) / p.BN);
+    }
     const int ks = pipe_info(pm).ks;
-    if (pm == 4) p.m_tiles = (int)((M + 2 * BM - 1) / (2 * BM));
+    const int ksa = pipe_info(pm).ksa ? pipe_info(pm).ksa : ks;
+    const bool pair = pipe_info(pm).pair != 0;
+    if (pair) p.m_tiles = (int)((M + 2 * BM - 1) / (2 * BM));
     choose_b_mode(&p, bits, pm);
     p.act = (const uint8_t *)A_codes;
     p.H = 1; p.W = (int)M; p.Ho = 1; p.Wo = (int)M;
@@ -1647,10 +1696,10 @@ int dsq_gemm(const void *A_codes, const void *B_codes, int64_t M, int64_t N, int
     p.ws = (int *)workspace;
     TcMaps tmap;
     int st = make_rows_tmap(&tmap.b, B_codes, pitch, (uint64_t)N, pitch, ks * 16 * bits,
-                            pm == 4 ? p.BN / 2 : p.BN);
+                            pair ? p.BN / 2 : p.BN);
     if (st) return st;
     tmap.a = tmap.b;
-    st = setup_a_tma(&p, &tmap.a, A_codes, M, bits, ks, true, nullptr, 1);
+    st = setup_a_tma(&p, &tmap.a, A_codes, M, bits, ksa, true, nullptr, 1);
     if (st) return st;
     tmap.c = tmap.b;
     tmap.d = tmap.b;

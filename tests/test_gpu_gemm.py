@@ -60,6 +60,24 @@ def test_gemm_direct_stores(dsq, bits, size):
     assert np.array_equal(native.gemm_dequant(C, rs), Dg)
 
 
+@pytest.mark.parametrize("bits", [2, 4])
+@pytest.mark.parametrize("size", [(512, 512, 1024), (300, 260, 1100), (1024, 640, 2048),
+                                  (129, 72, 4096)])
+def test_gemm_pairs_on_128_wide_tiles(dsq, bits, size):
+    """CTA pairs on 256 x 128 tiles with two accumulator buffers (forced through
+    the tuning hook; the automatic choice may pick another tiling)."""
+    M, Nn, K = size
+    A, B, rs = dsq_inputs.gemm_case(M, Nn, K, bits)
+    C = native.gemm(A, B)
+    dsq.dsq_set_cta_pairs(3)
+    try:
+        Cg, Dg = run(dsq, A, B, rs, bits)
+    finally:
+        dsq.dsq_set_cta_pairs(0)
+    assert np.array_equal(C, Cg)
+    assert np.array_equal(native.gemm_dequant(C, rs), Dg)
+
+
 @pytest.mark.parametrize("bits", [2, 3, 4])
 def test_gemm_extreme_codes(dsq, bits):
     # every product at its most negative: K * (-2^(b-1)) * (2^b - 1)
