@@ -9,16 +9,29 @@
 //
 //   B: TMA (cp.async.bulk.tensor.2d) packed tile -> shared ring ->
 //      unpack warps -> int8 tile in the K-major 128B-swizzled layout
-//   A: one thread per tile row gathers the row's packed 16-byte chunks
-//      straight from global memory (implicit im2col, zero fill outside the
-//      image), expands them in registers and stores them to TENSOR MEMORY
-//      (tcgen05.st): the A operand never touches shared memory, whose
-//      bandwidth is what bounds this kernel
-//   one thread issues tcgen05.mma.kind::i8 (128 x BN x 32 per instruction,
-//      A from tensor memory, B from shared memory), accumulating int32 in
-//      tensor memory (two accumulator buffers when BN <= 192)
+//   A: TMA brings the packed rows of a tile into a second shared ring: plain
+//      2-D boxes for a GEMM or a 1x1 stride-1 convolution, im2col boxes
+//      (cp.async.bulk.tensor.4d...im2col: 128 consecutive output pixels x one
+//      run of one filter tap, zero fill outside the image) for every other
+//      convolution.  One thread per tile row reads its row's 16-byte chunks,
+//      expands them in registers and stores them to TENSOR MEMORY
+//      (tcgen05.st): the expanded A operand never touches shared memory,
+//      whose bandwidth is what bounds this kernel.  (3-bit GEMM rows are
+//      gathered with cp.async instead.)
+//   one warp issues tcgen05.mma.kind::i8 (128 x BN x 32 per instruction, or
+//      256 x BN x 32 for a CTA pair; A from tensor memory, B from shared
+//      memory), accumulating int32 in tensor memory (two accumulator buffers
+//      where they fit beside the A stages)
 //   epilogue warps read tensor memory (tcgen05.ld), apply the dequantise /
-//      requantise epilogue and write codes / fp32 / int32.
+//      requantise epilogue and write codes / fp32 / int32 (GEMM outputs go
+//      through swizzled staging tiles and TMA stores); on a CTA's last tile
+//      the A and B warps join them.
+//
+// Each role's loop is a chain of hand-offs (barrier wait, expect, TMA or MMA
+// issue, commit); one hand-off costs a few hundred cycles while the unpack
+// warps keep the shared-memory pipeline busy, whatever amount of data is
+// behind it.  Hence: rounds of several K steps, A and B boxes issued by
+// threads of two different warps, MMA issue in uniform control flow.
 //
 // Signed codes are expanded into the TOP b bits of the byte (value * 2^(8-b)):
 // this costs no sign-extension arithmetic, and the exact factor is shifted out
@@ -1604,12 +1617,10 @@ int pick_pm(const TcParams &p, int bits, bool im2col)
     // CTA pairs: 256-wide N tiles and at least two 128-row tiles to put together
     if (p.BN == 256 && p.M > BM && g_pair_mode != 1) return 4;
     if (p.BN > 128) return p.ksteps >= 4 ? 3 : 1;
-    if (g_forced_ks == 2) return 2;
-    // when the expanded B tile can stay resident with single K steps, the
-    // rounds are cheap already and single steps measured slightly faster
-    TcParams q = p;
-    choose_b_mode(&q, bits, 1);
-    return q.b_res ? 1 : 2;
+    // two K steps per round: a round costs about the same whatever it carries
+    // (measured faster than single steps even where those would keep the
+    // expanded B tile resident)
+    return 2;
 }
 
 }  // namespace
