@@ -285,6 +285,16 @@ int dsq_set_cta_pairs(int mode);
  * epilogue warps.  Results do not depend on it. */
 int dsq_set_gemm_store(int mode);
 
+/* Fifth hook: programmatic dependent launch of the tensor-core kernels
+ * (default on).  dsq_conv2d / dsq_gemm launch their kernel with the
+ * programmatic stream-serialisation attribute: its set-up (barriers, tensor
+ * memory, descriptor prefetch) may run while the previous kernel of the
+ * stream is finishing, and it waits for that kernel to complete
+ * (griddepcontrol.wait) before it reads or writes any global data, so stream
+ * order is kept.  0 switches to plain launches.  Results do not depend on
+ * it. */
+int dsq_set_dependent_launch(int on);
+
 /* ---- misc --------------------------------------------------------------- */
 const char *dsq_status_string(int status);
 int dsq_version(void);

@@ -78,6 +78,7 @@ _SIGNATURES = {
     "dsq_set_round_k_steps": (_int, [_int]),
     "dsq_set_cta_pairs": (_int, [_int]),
     "dsq_set_gemm_store": (_int, [_int]),
+    "dsq_set_dependent_launch": (_int, [_int]),
     "dsq_status_string": (C.c_char_p, [_int]),
     "dsq_version": (_int, []),
 }
@@ -330,6 +331,10 @@ def dsq_set_cta_pairs(mode):
 
 def dsq_set_gemm_store(mode):
     _check(lib.dsq_set_gemm_store(mode), "dsq_set_gemm_store")
+
+
+def dsq_set_dependent_launch(on):
+    _check(lib.dsq_set_dependent_launch(on), "dsq_set_dependent_launch")
 
 
 def dsq_set_tile_n(bn):

@@ -54,6 +54,21 @@ __device__ __forceinline__ uint64_t global_timer_ns()
     return t;
 }
 
+// ---- programmatic dependent launch --------------------------------------------
+// launch_dependents: the grids queued behind this one with the programmatic
+// serialisation attribute may start being scheduled once every CTA of this
+// grid has executed it (or exited).  wait: blocks until all grids this one
+// depends on have completed and their memory is visible; a no-op for a grid
+// launched without the attribute.
+__device__ __forceinline__ void grid_launch_dependents()
+{
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+__device__ __forceinline__ void grid_dependency_wait()
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 // ---- thread-block clusters (CTA pairs) ---------------------------------------
 __device__ __forceinline__ uint32_t cluster_ctarank()
 {

@@ -442,6 +442,12 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
     if (PAIR) cluster_sync_all();
     tc_fence_after_sync();
     const uint32_t tmem_base = __shfl_sync(0xffffffffu, *tmem_slot, 0);
+    // Programmatic dependent launch: everything above (barriers, tensor memory,
+    // descriptor prefetch) touched no global data, so it may run while the
+    // kernel before this one is still finishing; nothing below starts before
+    // that kernel has completed.  The kernel behind this one may set up likewise.
+    grid_launch_dependents();
+    grid_dependency_wait();
 
     // Epilogue roles.  epi_idx >= 0: the warp takes part in the epilogue of every
     // tile (p.epw warps per TMEM lane quarter).  join_idx >= 0: it takes part in
@@ -1471,6 +1477,7 @@ int setup_a_tma(TcParams *p, CUtensorMap *map, const void *A, int64_t rows, int 
 }
 
 int g_forced_bn = 0;   // dsq_set_tile_n
+int g_pdl = 1;         // dsq_set_dependent_launch
 
 int pick_bn(int m_tiles, int ncols, int bits)
 {
@@ -1515,29 +1522,35 @@ int launch_tc(const TcMaps &tmap, const TcParams &p, cudaStream_t s)
     if (p.BN * p.n_acc > Pipe<PM>::A_COL0) return DSQ_ERR_UNSUPPORTED;
     TcParams q = p;
     q.smem_bytes = smem_bytes;
+    // one cluster of two CTAs (the two SMs of a TPC) per tile in flight
+    if (PAIR && grid > 74) grid = 74;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(PAIR ? 2 * grid : grid);
+    cfg.blockDim = dim3(NUM_THREADS);
+    cfg.dynamicSmemBytes = (size_t)smem_bytes;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[2];
+    int na = 0;
     if (PAIR) {
-        // one cluster of two CTAs (the two SMs of a TPC) per tile in flight
-        if (grid > 74) grid = 74;
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(2 * grid);
-        cfg.blockDim = dim3(NUM_THREADS);
-        cfg.dynamicSmemBytes = (size_t)smem_bytes;
-        cfg.stream = s;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeClusterDimension;
-        attr[0].val.clusterDim.x = 2;
-        attr[0].val.clusterDim.y = 1;
-        attr[0].val.clusterDim.z = 1;
-        cfg.attrs = attr;
-        cfg.numAttrs = 1;
-        if (cudaLaunchKernelEx(&cfg, dsq_tc_kernel<BITS, A_SIGNED, EPI, PM, A_TMA>, tmap.b, tmap.a, tmap.c, tmap.d, q) !=
-            cudaSuccess) {
-            cudaGetLastError();
-            return DSQ_ERR_CUDA;
-        }
-        return dsq_launch_status();
+        attr[na].id = cudaLaunchAttributeClusterDimension;
+        attr[na].val.clusterDim.x = 2;
+        attr[na].val.clusterDim.y = 1;
+        attr[na].val.clusterDim.z = 1;
+        ++na;
     }
-    dsq_tc_kernel<BITS, A_SIGNED, EPI, PM, A_TMA><<<grid, NUM_THREADS, smem_bytes, s>>>(tmap.b, tmap.a, tmap.c, tmap.d, q);
+    if (g_pdl) {
+        // the kernel waits for its predecessors itself (griddepcontrol.wait)
+        attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[na].val.programmaticStreamSerializationAllowed = 1;
+        ++na;
+    }
+    cfg.attrs = attr;
+    cfg.numAttrs = na;
+    if (cudaLaunchKernelEx(&cfg, dsq_tc_kernel<BITS, A_SIGNED, EPI, PM, A_TMA>, tmap.b, tmap.a,
+                           tmap.c, tmap.d, q) != cudaSuccess) {
+        cudaGetLastError();
+        return DSQ_ERR_CUDA;
+    }
     return dsq_launch_status();
 }
 
@@ -1638,6 +1651,13 @@ int dsq_set_cta_pairs(int mode)
 {
     if (mode < 0 || mode > 3) return DSQ_ERR_SHAPE;
     g_pair_mode = mode;
+    return DSQ_OK;
+}
+
+int dsq_set_dependent_launch(int on)
+{
+    if (on != 0 && on != 1) return DSQ_ERR_SHAPE;
+    g_pdl = on;
     return DSQ_OK;
 }
 

@@ -56,6 +56,45 @@ def test_tiny_stack_every_layer(dsq, bits, w_offset):
     compare_stack(st, 9, st.batch, w_offset)
 
 
+def test_tiny_stack_plain_launches(dsq):
+    """Same codes with programmatic dependent launch switched off."""
+    st = dsq_inputs.tiny_stack(bits=4)
+    dsq.dsq_set_dependent_launch(0)
+    try:
+        compare_stack(st, 9, st.batch, 0.5, debug=False)
+    finally:
+        dsq.dsq_set_dependent_launch(1)
+
+
+def test_resnet18_stack_graph_replay_matches_eager(dsq):
+    """The captured call sequence (dependent launches become programmatic graph
+    edges) reproduces the eager pass bit for bit, replay after replay."""
+    from paper_1908_05033_b200.stack import GpuStack
+    st = dsq_inputs.resnet18_stack(batch=4)
+    x = T(dsq_inputs.stack_input(st, batch=4, workload_id=3))
+    params = dsq_inputs.stack_params(st, workload_id=3)
+    g = GpuStack(st, params, batch=4)
+    eager = g.forward(x).clone()
+    names = list(st.tensor_shapes())
+    want = {n: g.codes[n].clone() for n in names}
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        gr = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(gr, stream=side):
+            g.forward(x)
+    torch.cuda.synchronize()
+    for _ in range(3):
+        for n in names:
+            g.codes[n].fill_(0xFF)
+        gr.replay()
+        torch.cuda.synchronize()
+        g.check()
+        for n in names:
+            assert torch.equal(g.codes[n], want[n]), n
+    assert torch.equal(g.codes[st.out], eager)
+
+
 def test_resnet18_stack_batch1_every_layer(dsq):
     st = dsq_inputs.resnet18_stack()
     _, ref = compare_stack(st, 3, 1)
