@@ -165,7 +165,15 @@ struct TcParams {
     //      pitch, so a box never straddles two taps); K columns past the last
     //      tap are not loaded, the A threads put zeros there (a_kchunks = 16-byte
     //      chunks of a row that exist)
-    int a_tma, a_lc, a_nsub, a_kchunks;
+    //   3: whole image rows (3x3, stride 1, pad 1 over 64 channels, whole-K
+    //      rounds): the tile's output pixels lie in a few consecutive image rows
+    //      and all their taps in those rows plus one above and one below.  a_nr
+    //      rows of the (N*H) x (W*P bytes) matrix are fetched once per tile as ONE
+    //      box, and every A thread picks its pixel's 3 x 3P bytes out of them,
+    //      zeroing the taps outside the image: a third of the im2col bytes, in
+    //      rows of up to 2 KB instead of one pixel's P bytes (the TMA unit spends
+    //      a few cycles per row whatever its length).  a_bw = W*P.
+    int a_tma, a_lc, a_nsub, a_kchunks, a_nr, a_bw;
     // epilogue
     int mode, shift, out_pitch, small_acc;
     DsqEpi e;
@@ -318,7 +326,10 @@ __host__ __device__ inline SmemLayout smem_layout(int BN, int bits, int s_p, int
     return L;
 }
 
-template <int BITS, bool A_SIGNED, int EPI, int PM, bool A_TMA>
+// A_TMA: 0 = A gathered with cp.async, 1 = TMA boxes (2-D or im2col), 3 = whole
+// image rows (TcParams::a_tma); a template parameter so that the A threads' loop
+// carries one fetch path (the kernel is sensitive to its code size)
+template <int BITS, bool A_SIGNED, int EPI, int PM, int A_TMA>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
               const __grid_constant__ CUtensorMap tmap_a,
@@ -503,7 +514,13 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
                 const int sl = (int)(g % A_SLOTS);
                 if (!wait_bar(bar_ar_empty(sl), ((g / A_SLOTS) & 1u) ^ 1u, ctl, 11)) break;
                 const int m0 = (tile_a / p.n_tiles) * BMT + row_base;
-                if (p.a_tma == 1) {
+                if (A_TMA == 3) {
+                    // rows R0-1 .. R0-2+a_nr of the row matrix (R = n*H + h); rows
+                    // outside it are filled with zeros (and masked by the readers)
+                    mbar_arrive_expect_tx(bar_ar_full(sl), (uint32_t)(p.a_nr * p.a_bw));
+                    tma_load_2d(ring + sl * A_SLOT_BYTES, &tmap_a, 0, m0 / p.W - 1,
+                                bar_ar_full(sl));
+                } else if (p.a_tma == 1) {
                     mbar_arrive_expect_tx(bar_ar_full(sl), A_SLOT_BYTES);
                     tma_load_2d(ring + sl * A_SLOT_BYTES, &tmap_a, ka * (KSA * 16 * BITS), m0,
                                 bar_ar_full(sl));
@@ -694,7 +711,7 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
             pend_s = -1;
         };
         // TMA mode: slot = 128 rows of KS*CH chunks, chunk index XOR-swizzled
-        constexpr bool a_tma = A_TMA;
+        constexpr bool a_tma = A_TMA != 0;
         // chunk jj of the round lies in box jj >> a_lc, at chunk (jj ^ swizzle) of
         // this thread's row of that box
         const int lc = p.a_lc;
@@ -731,6 +748,25 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
             // chunks of this round that exist (im2col: nothing is loaded past the
             // last filter tap)
             int kvalid = KSA * CH;
+            // rows mode: where this thread's pixel lies in the staged image rows
+            constexpr int CPP = BITS / 2;              // 16-byte chunks per pixel (64 channels)
+            constexpr bool rows_mode = Pipe<PM>::WHOLE_K && BITS != 3 && A_TMA == 3;
+            uint32_t rows_base = 0, rowmask = 0, colmask = 0, sw16 = 0;
+            if (Pipe<PM>::WHOLE_K && rows_mode) {
+                const int tile = tile0 + (int)g * tstep;       // one round per tile
+                const int m0 = (tile / p.n_tiles) * BMT + row_base;
+                const int m = m0 + row;
+                const int R = m / p.W, wo = m - R * p.W, ho = R % p.H;
+                // bit kh / kw: that row / column of the 3x3 window is inside the image
+                rowmask = m < p.M ? (uint32_t)((ho > 0) | 2 | ((ho < p.H - 1) << 2)) : 0u;
+                colmask = (uint32_t)((wo > 0) | 2 | ((wo < p.W - 1) << 2));
+                rows_base = smem_u32(smem + L.a_ring) + aslot * SLOT_BYTES +
+                            (uint32_t)((R - m0 / p.W) * p.a_bw + (wo - 1) * p.P);
+                // two chunks per pixel: adjacent lanes are 32 bytes apart, so lanes
+                // 4..7 of a quarter warp fetch each pair of chunks in the other
+                // order (and swap afterwards): conflict-free 128-bit loads
+                sw16 = CPP == 2 ? (uint32_t)((lane >> 2) & 1) << 4 : 0u;
+            }
             if (a_tma) {
                 if (p.a_tma == 2) kvalid = p.a_kchunks - kr * (KSA * CH);
                 kr += GROUPS;
@@ -744,13 +780,33 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
                     uint4 cur[CH];
 #pragma unroll
                     for (int j = 0; j < CH; ++j) {
-                        if (a_tma) {
+                        if (Pipe<PM>::WHOLE_K && BITS != 3 && rows_mode) {
+                            // chunk jj of the K row: window row jj / (3 CPP), then
+                            // 3 CPP consecutive chunks.  Always loaded (the address
+                            // stays inside shared memory), zeroed when outside
+                            const int kk = h * CH + j;
+                            const int kh = kk / (3 * CPP), q = kk % (3 * CPP);
+                            const uint32_t keep =
+                                ((rowmask >> kh) & (colmask >> (q / CPP)) & 1u) ? 0xFFFFFFFFu : 0u;
+                            uint4 v = lds_128(rows_base + (uint32_t)(kh * p.a_bw) +
+                                              ((uint32_t)(q * 16) ^ sw16));
+                            v.x &= keep; v.y &= keep; v.z &= keep; v.w &= keep;
+                            cur[j] = v;
+                        } else if (a_tma) {
                             cur[j] = (h * CH + j < kvalid)
                                          ? lds_128(tma_chunk(h * CH + j) + aslot * SLOT_BYTES)
                                          : make_uint4(0u, 0u, 0u, 0u);
                         } else {
                             cur[j] = lds_128(cell0 + rd_slot * SLOT_BYTES +
                                              (h * CH + j) * (BM * 16));
+                        }
+                    }
+                    if (rows_mode && CPP == 2 && sw16) {
+#pragma unroll
+                        for (int j = 0; j + 1 < CH; j += 2) {
+                            const uint4 t = cur[j];
+                            cur[j] = cur[j + 1];
+                            cur[j + 1] = t;
                         }
                     }
                     expand_row_regs<BITS, A_SIGNED>(cur, p.orv, o);
@@ -1437,14 +1493,41 @@ CUtensorMapSwizzle swizzle_for_span(int bytes)
 // box per round.  Any other convolution: im2col boxes over the NHWC tensor,
 // `sub` the largest such power of two that divides the pixel pitch.
 int setup_a_tma(TcParams *p, CUtensorMap *map, const void *A, int64_t rows, int bits, int ks,
-                bool plain_rows, const dsq_nhwc_t *shape, int ksize)
+                bool plain_rows, const dsq_nhwc_t *shape, int ksize, bool whole_k)
 {
     p->a_tma = 0;
     p->a_lc = 0;
     p->a_nsub = 1;
     p->a_kchunks = 0;
+    p->a_nr = p->a_bw = 0;
     const int round_bytes = ks * bits * 16;
     if (bits == 3) return DSQ_OK;
+    // whole image rows (TcParams::a_tma == 3): 3x3, stride 1, pad 1, 64 channels
+    if (whole_k && !plain_rows && ksize == 3 && p->stride == 1 && p->pad == 1 &&
+        p->P == 8 * bits) {
+        const int64_t row_bytes = (int64_t)shape->W * p->P;
+        const int nr = (BM - 1 + shape->W - 1) / shape->W + 3;
+        if (row_bytes <= 2048 && row_bytes % 16 == 0 && nr <= 256 &&
+            nr * row_bytes <= (int64_t)round_bytes * BM) {
+            EncodeTiledFn fn = get_encode_fn();
+            if (!fn) return DSQ_ERR_CUDA;
+            // 8-byte elements, so that a box may span a whole row of up to 2 KB
+            cuuint64_t dims[2] = {(cuuint64_t)(row_bytes / 8),
+                                  (cuuint64_t)shape->N * (cuuint64_t)shape->H};
+            cuuint64_t strides[1] = {(cuuint64_t)row_bytes};
+            cuuint32_t box[2] = {(cuuint32_t)(row_bytes / 8), (cuuint32_t)nr};
+            cuuint32_t estr[2] = {1, 1};
+            const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT64, 2, const_cast<void *>(A),
+                                  dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                  CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+            if (r != CUDA_SUCCESS) return DSQ_ERR_CUDA;
+            p->a_tma = 3;
+            p->a_nr = nr;
+            p->a_bw = (int)row_bytes;
+            return DSQ_OK;
+        }
+    }
     if (plain_rows) {
         const int st = make_rows_tmap(map, A, (uint64_t)p->P, (uint64_t)rows, (uint64_t)p->P,
                                       (uint32_t)round_bytes, BM, swizzle_for_span(round_bytes));
@@ -1497,10 +1580,10 @@ int pick_bn(int m_tiles, int ncols, int bits)
     return best;
 }
 
-template <int BITS, bool A_SIGNED, int EPI, int PM, bool A_TMA>
+template <int BITS, bool A_SIGNED, int EPI, int PM, int A_TMA>
 int launch_tc(const TcMaps &tmap, const TcParams &p, cudaStream_t s)
 {
-    if ((p.a_tma != 0) != A_TMA) return DSQ_ERR_UNSUPPORTED;
+    if ((p.a_tma == 3 ? 3 : p.a_tma != 0) != A_TMA) return DSQ_ERR_UNSUPPORTED;
     constexpr bool PAIR = Pipe<PM>::PAIR;
     const SmemLayout L = smem_layout(PAIR ? p.BN / 2 : p.BN, BITS, p.s_p, p.b_stages,
                                      Pipe<PM>::KS,
@@ -1559,15 +1642,15 @@ int launch_conv(int epi, const TcMaps &tmap, const TcParams &p, cudaStream_t s)
 {
     if (p.a_tma) {
         switch (epi) {
-        case EPI_CODES: return launch_tc<BITS, false, EPI_CODES, PM, true>(tmap, p, s);
-        case EPI_CODES_RES: return launch_tc<BITS, false, EPI_CODES_RES, PM, true>(tmap, p, s);
-        default: return launch_tc<BITS, false, EPI_GENERAL, PM, true>(tmap, p, s);
+        case EPI_CODES: return launch_tc<BITS, false, EPI_CODES, PM, 1>(tmap, p, s);
+        case EPI_CODES_RES: return launch_tc<BITS, false, EPI_CODES_RES, PM, 1>(tmap, p, s);
+        default: return launch_tc<BITS, false, EPI_GENERAL, PM, 1>(tmap, p, s);
         }
     }
     switch (epi) {
-    case EPI_CODES: return launch_tc<BITS, false, EPI_CODES, PM, false>(tmap, p, s);
-    case EPI_CODES_RES: return launch_tc<BITS, false, EPI_CODES_RES, PM, false>(tmap, p, s);
-    default: return launch_tc<BITS, false, EPI_GENERAL, PM, false>(tmap, p, s);
+    case EPI_CODES: return launch_tc<BITS, false, EPI_CODES, PM, 0>(tmap, p, s);
+    case EPI_CODES_RES: return launch_tc<BITS, false, EPI_CODES_RES, PM, 0>(tmap, p, s);
+    default: return launch_tc<BITS, false, EPI_GENERAL, PM, 0>(tmap, p, s);
     }
 }
 
@@ -1576,17 +1659,24 @@ int launch_bits(int epi, int pm, const TcMaps &tmap, const TcParams &p, cudaStre
 {
     if (epi == EPI_GEMM) {
         // 2- and 4-bit GEMMs always fetch A with TMA
-        if (pm == 6) return launch_tc<BITS, true, EPI_GEMM, 6, true>(tmap, p, s);
-        if (pm == 4) return launch_tc<BITS, true, EPI_GEMM, 4, true>(tmap, p, s);
-        if (pm == 3) return launch_tc<BITS, true, EPI_GEMM, 3, true>(tmap, p, s);
-        if (pm == 2) return launch_tc<BITS, true, EPI_GEMM, 2, true>(tmap, p, s);
-        return launch_tc<BITS, true, EPI_GEMM, 1, true>(tmap, p, s);
+        if (pm == 6) return launch_tc<BITS, true, EPI_GEMM, 6, 1>(tmap, p, s);
+        if (pm == 4) return launch_tc<BITS, true, EPI_GEMM, 4, 1>(tmap, p, s);
+        if (pm == 3) return launch_tc<BITS, true, EPI_GEMM, 3, 1>(tmap, p, s);
+        if (pm == 2) return launch_tc<BITS, true, EPI_GEMM, 2, 1>(tmap, p, s);
+        return launch_tc<BITS, true, EPI_GEMM, 1, 1>(tmap, p, s);
+    }
+    if (pm == 5 && p.a_tma == 3) {
+        switch (epi) {
+        case EPI_CODES: return launch_tc<BITS, false, EPI_CODES, 5, 3>(tmap, p, s);
+        case EPI_CODES_RES: return launch_tc<BITS, false, EPI_CODES_RES, 5, 3>(tmap, p, s);
+        default: return launch_tc<BITS, false, EPI_GENERAL, 5, 3>(tmap, p, s);
+        }
     }
     if (pm == 5) {
         switch (epi) {
-        case EPI_CODES: return launch_tc<BITS, false, EPI_CODES, 5, true>(tmap, p, s);
-        case EPI_CODES_RES: return launch_tc<BITS, false, EPI_CODES_RES, 5, true>(tmap, p, s);
-        default: return launch_tc<BITS, false, EPI_GENERAL, 5, true>(tmap, p, s);
+        case EPI_CODES: return launch_tc<BITS, false, EPI_CODES, 5, 1>(tmap, p, s);
+        case EPI_CODES_RES: return launch_tc<BITS, false, EPI_CODES_RES, 5, 1>(tmap, p, s);
+        default: return launch_tc<BITS, false, EPI_GENERAL, 5, 1>(tmap, p, s);
         }
     }
     if (pm == 4) return launch_conv<BITS, 4>(epi, tmap, p, s);
@@ -1600,7 +1690,7 @@ int dispatch_tc(int bits, int epi, int pm, const TcMaps &tmap, const TcParams &p
 {
     if (bits == 4) return launch_bits<4>(epi, pm, tmap, p, s);
     if (bits == 2) return launch_bits<2>(epi, pm, tmap, p, s);
-    if (bits == 3 && epi == EPI_GEMM) return launch_tc<3, true, EPI_GEMM, 1, false>(tmap, p, s);
+    if (bits == 3 && epi == EPI_GEMM) return launch_tc<3, true, EPI_GEMM, 1, 0>(tmap, p, s);
     return DSQ_ERR_UNSUPPORTED;
 }
 
@@ -1730,7 +1820,7 @@ int dsq_gemm(const void *A_codes, const void *B_codes, int64_t M, int64_t N, int
                             pair ? p.BN / 2 : p.BN);
     if (st) return st;
     tmap.a = tmap.b;
-    st = setup_a_tma(&p, &tmap.a, A_codes, M, bits, ksa, true, nullptr, 1);
+    st = setup_a_tma(&p, &tmap.a, A_codes, M, bits, ksa, true, nullptr, 1, false);
     if (st) return st;
     tmap.c = tmap.b;
     tmap.d = tmap.b;
@@ -1825,7 +1915,7 @@ int dsq_conv2d(const void *act_codes, const dsq_nhwc_t *shape, const dsq_quant_t
     if (st) return st;
     tmap.a = tmap.b;
     // a 1x1 stride-1 unpadded convolution reads the pixel rows as they lie
-    st = setup_a_tma(&p, &tmap.a, act_codes, M, bits, ks, plain_rows, shape, conv->KH);
+    st = setup_a_tma(&p, &tmap.a, act_codes, M, bits, ks, plain_rows, shape, conv->KH, pm == 5);
     if (st) return st;
     // largest |2*acc + S_a| below 2^22: the epilogue may convert integers to
     // float through the 1.5 * 2^23 bias trick, which is exact there
