@@ -1012,66 +1012,6 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
                 }
             };
             fetch_cols(my_idx * 32);
-            if (EPI == EPI_GEMM && p.stage) {
-                // The warp's 32 rows x 32 columns go through a 128-byte-swizzled
-                // staging tile to one TMA store (rows / columns past the matrix are
-                // clipped by the store): the LSU sees 8 conflict-free shared stores
-                // per lane instead of 32-byte pieces of 32 different lines.  The
-                // tensor-memory load of the next block is issued as soon as this
-                // block's registers have gone to the staging tile.
-                const uint32_t stg = ((smem_u32(smem + L.epi) + 1023u) & ~1023u) +
-                                     (uint32_t)(my_idx * 4 + quarter) * 4096u;
-                const uint32_t stg_row = stg + (uint32_t)lane * 128u;
-                const int y0 = m_tile * BMT + row_base + quarter * 32;
-                uint32_t r[32];
-                int c0 = my_idx * 32;
-                if (c0 < BN) {
-                    __syncwarp();
-                    tmem_ld_32x32(taddr + c0, r);
-                }
-#pragma unroll 1
-                for (; c0 < BN; c0 += 32 * epi_cnt) {
-                    const int n0 = n_tile * BN + c0;
-                    const int c_next = c0 + 32 * epi_cnt;
-                    __syncwarp();                  // (lane 0 comes back from its store)
-                    tmem_ld_wait();
-#pragma unroll
-                    for (int c = 0; c < 32; ++c) r[c] = (uint32_t)((int)r[c] >> p.shift);
-                    if (p.C_i32) {
-                        if (lane == 0) bulk_wait_group_read<0>();   // staging tile free again
-                        __syncwarp();
-#pragma unroll
-                        for (int v = 0; v < 8; ++v)
-                            sts_128(stg_row + (uint32_t)((v ^ (lane & 7)) << 4), r[4 * v],
-                                    r[4 * v + 1], r[4 * v + 2], r[4 * v + 3]);
-                        if (!p.D_f32 && c_next < BN) tmem_ld_32x32(taddr + c_next, r);
-                        fence_proxy_async_smem();
-                        __syncwarp();
-                        if (lane == 0) {
-                            tma_store_2d(&tmap_c, stg, n0, y0);
-                            bulk_commit_group();
-                        }
-                    }
-                    if (p.D_f32) {
-                        if (lane == 0) bulk_wait_group_read<0>();
-                        __syncwarp();
-#pragma unroll
-                        for (int v = 0; v < 8; ++v)
-                            sts_128(stg_row + (uint32_t)((v ^ (lane & 7)) << 4),
-                                    __float_as_uint(__fmul_rn((float)(int)r[4 * v], rs)),
-                                    __float_as_uint(__fmul_rn((float)(int)r[4 * v + 1], rs)),
-                                    __float_as_uint(__fmul_rn((float)(int)r[4 * v + 2], rs)),
-                                    __float_as_uint(__fmul_rn((float)(int)r[4 * v + 3], rs)));
-                        if (c_next < BN) tmem_ld_32x32(taddr + c_next, r);
-                        fence_proxy_async_smem();
-                        __syncwarp();
-                        if (lane == 0) {
-                            tma_store_2d(&tmap_d, stg, n0, y0);
-                            bulk_commit_group();
-                        }
-                    }
-                }
-            } else
 #pragma unroll 1
             for (int c0 = my_idx * 32; c0 < BN; c0 += 32 * epi_cnt) {
                 uint32_t r[32];
@@ -1085,6 +1025,42 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
                 }
                 tmem_ld_wait();
                 const int n0 = n_tile * BN + c0;
+                if (EPI == EPI_GEMM && p.stage) {
+                    // the warp's 32 rows x 32 columns go through a 128-byte-swizzled
+                    // staging tile to one TMA store (rows / columns past the matrix
+                    // are clipped by the store): the LSU sees 8 conflict-free shared
+                    // stores per lane instead of 32-byte pieces of 32 different lines
+                    const uint32_t stg =
+                        ((smem_u32(smem + L.epi) + 1023u) & ~1023u) +
+                        (uint32_t)(my_idx * 4 + quarter) * 4096u + (uint32_t)lane * 128u;
+                    const int y0 = m_tile * BMT + row_base + quarter * 32;
+#pragma unroll
+                    for (int c = 0; c < 32; ++c) r[c] = (uint32_t)((int)r[c] >> p.shift);
+#pragma unroll 1
+                    for (int o = 0; o < 2; ++o) {
+                        if (o == 0 ? p.C_i32 == nullptr : p.D_f32 == nullptr) continue;
+                        // the previous store has finished reading the tile
+                        if (lane == 0) bulk_wait_group_read<0>();
+                        __syncwarp();
+#pragma unroll
+                        for (int v = 0; v < 8; ++v) {
+                            uint32_t w[4];
+#pragma unroll
+                            for (int u = 0; u < 4; ++u)
+                                w[u] = o == 0 ? r[4 * v + u]
+                                              : __float_as_uint(
+                                                    __fmul_rn((float)(int)r[4 * v + u], rs));
+                            sts_128(stg + (uint32_t)((v ^ (lane & 7)) << 4), w[0], w[1], w[2], w[3]);
+                        }
+                        fence_proxy_async_smem();
+                        __syncwarp();
+                        if (lane == 0) {
+                            tma_store_2d(o == 0 ? &tmap_c : &tmap_d, stg, n0, y0);
+                            bulk_commit_group();
+                        }
+                    }
+                    continue;
+                }
                 if (!row_ok) continue;
 #pragma unroll
                 for (int c = 0; c < 32; ++c) r[c] = (uint32_t)((int)r[c] >> p.shift);
