@@ -122,3 +122,22 @@ def test_gemm_full_size_sampled(dsq, bits, size):
     # determinism: a second run gives identical bits
     Cg2, _ = run(dsq, A, B, rs, bits)
     assert np.array_equal(Cg, Cg2)
+
+
+def test_gemm_repeated_launches_identical(dsq):
+    """Many tiles per CTA, both outputs, launch after launch: every run gives
+    the bits of the first (a race between the epilogue and the next tile's
+    MMAs, or between a staged store and the next block, shows up here)."""
+    size, bits = 8192, 4
+    A, B, rs = dsq_inputs.gemm_case(size, size, size, bits)
+    ws = dsq.new_workspace()
+    Ap, Bp = dsq.dsq_pack_codes(T(A), bits), dsq.dsq_pack_codes(T(B), bits)
+    rst = T(rs)
+    C0, D0 = dsq.dsq_gemm(Ap, Bp, size, size, size, bits, ws, row_scale=rst)
+    C0, D0 = C0.clone(), D0.clone()
+    for _ in range(16):
+        C, D = dsq.dsq_gemm(Ap, Bp, size, size, size, bits, ws, row_scale=rst)
+        assert torch.equal(C, C0) and torch.equal(D, D0)
+    assert dsq.dsq_workspace_status(ws) == 0
+    rows = np.arange(0, size, 517)
+    assert np.array_equal(native.gemm(A[rows], B), N(C0)[rows])
