@@ -118,6 +118,17 @@ def test_conv_geometries(dsq, geom, bits, w_off):
 
 
 @pytest.mark.parametrize("bits", [2, 4])
+@pytest.mark.parametrize("geom", [(6, 60, 60), (4, 70, 70), (1, 150, 150), (3, 97, 83)])
+def test_conv_whole_k_rounds(dsq, geom, bits):
+    """3x3 over 64 channels on more tiles than SMs: one round per tile, the A
+    rows staged as whole image rows (rows of at most 2 KB) or as im2col boxes
+    (wider images); image widths that do not divide the 128-pixel tile, a
+    ragged last tile, every element against the oracle."""
+    n, h, w = geom
+    conv_case(dsq, n, h, w, 64, 64, 3, 1, 1, bits, 0.5, residual=(n == 6), seed=n + h)
+
+
+@pytest.mark.parametrize("bits", [2, 4])
 def test_conv_residual_and_per_channel(dsq, bits):
     conv_case(dsq, 2, 14, 14, 64, 64, 3, 1, 1, bits, 0.5, residual=True)
     conv_case(dsq, 1, 10, 10, 48, 200, 1, 1, 0, bits, 0.5, residual=True,
