@@ -278,11 +278,13 @@ int dsq_set_round_k_steps(int ks);
  * on it. */
 int dsq_set_cta_pairs(int mode);
 
-/* Fourth tuning hook: how dsq_gemm writes its int32 / fp32 outputs.  mode 0:
- * automatic (each epilogue warp stages its 32 x 32 block in shared memory and
- * one TMA store writes it, whenever N is a multiple of 4 and the staging tiles
- * fit next to the operand rings), 1: always direct vector stores from the
- * epilogue warps.  Results do not depend on it. */
+/* Fourth tuning hook: how dsq_gemm writes its int32 / fp32 outputs.  mode 1
+ * (the default): direct vector stores from the epilogue warps.  mode 0: each
+ * epilogue warp stages its 32 x 32 block in shared memory and one TMA store
+ * writes it, whenever N is a multiple of 4 and the staging tiles fit next to
+ * the operand rings.  The staged path is kept for experiments only: with both
+ * outputs requested, long runs of 8192^3 launches returned a wrong tile once
+ * in a while and one run ended in a launch failure, cause not found. */
 int dsq_set_gemm_store(int mode);
 
 /* Fifth hook: programmatic dependent launch of the tensor-core kernels

@@ -55,7 +55,7 @@ def main(argv=None):
     ap.add_argument("--tile-n", type=int, default=0)
     ap.add_argument("--round-k", type=int, default=0)
     ap.add_argument("--pairs", type=int, default=0, help="0 auto, 1 never, 2 wherever possible")
-    ap.add_argument("--gemm-store", type=int, default=0, help="0 TMA stores, 1 direct stores")
+    ap.add_argument("--gemm-store", type=int, default=1, help="1 direct stores (default), 0 staged TMA stores")
     a = ap.parse_args(argv)
     dev = "cuda"
     ws = B.new_workspace(dev)

@@ -28,6 +28,10 @@ __global__ void __launch_bounds__(256)
 dwconv3x3_kernel(const uint8_t *__restrict__ act, const uint8_t *__restrict__ wgt,
                  int N, int H, int W, int C, int Ho, int Wo, int pitch, DsqEpi e)
 {
+    // lets a tensor-core kernel queued behind this one (programmatic dependent
+    // launch) set itself up while this grid runs; it still waits for this grid
+    // to complete before touching global data
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     constexpr int UB = BITS;                 // bytes per 8-channel unit
     constexpr uint32_t MASK = (1u << BITS) - 1u;
     constexpr int OW = 4;                    // outputs per thread along W

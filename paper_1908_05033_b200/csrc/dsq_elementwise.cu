@@ -81,6 +81,10 @@ __global__ void __launch_bounds__(256)
 quantize_flat_kernel(const float4 *__restrict__ x, uint4 *__restrict__ out,
                      int64_t n_lines, DsqQ q)
 {
+    // lets a tensor-core kernel queued behind this one (programmatic dependent
+    // launch) set itself up while this grid runs; it still waits for this grid
+    // to complete before touching global data
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     constexpr int NF = (BITS == 4) ? 1 : 2;
     constexpr int F4_PER_LINE = 8 * NF;
     const int lane = threadIdx.x & 31;
@@ -153,6 +157,10 @@ __global__ void __launch_bounds__(256)
 quantize_rows_kernel(const float *__restrict__ x, uint32_t *__restrict__ out,
                      int64_t rows, int k, int pitch_words, int bits, DsqQ q)
 {
+    // lets a tensor-core kernel queued behind this one (programmatic dependent
+    // launch) set itself up while this grid runs; it still waits for this grid
+    // to complete before touching global data
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int64_t total = rows * pitch_words;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total;
          i += (int64_t)gridDim.x * blockDim.x) {
@@ -246,6 +254,10 @@ __global__ void __launch_bounds__(256)
 maxpool_kernel(const uint32_t *__restrict__ in, uint32_t *__restrict__ out,
                int N, int H, int W, int C, int pitch_words, int bits)
 {
+    // lets a tensor-core kernel queued behind this one (programmatic dependent
+    // launch) set itself up while this grid runs; it still waits for this grid
+    // to complete before touching global data
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int Ho = H / 2, Wo = W / 2;
     const int64_t total = (int64_t)N * Ho * Wo * pitch_words;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total;

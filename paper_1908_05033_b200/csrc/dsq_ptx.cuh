@@ -90,14 +90,30 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank)
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
     return r;
 }
-// Arrive on an mbarrier of any CTA of the cluster (shared::cluster address).
-// Default semantics (release at CTA scope): what the arriving thread wrote to
-// its own shared / tensor memory is complete before the arrival is seen, which
-// is all the peer's MMA thread needs before it lets the tensor core read that
-// memory.  (A cluster-scope release costs over a thousand cycles per arrival.)
+// One bounded attempt with acquire semantics at cluster scope (pairs with an
+// arrival released at cluster scope by a thread of the peer CTA).
+__device__ __forceinline__ uint32_t mbar_try_wait_cluster(uint32_t bar, uint32_t parity,
+                                                          uint32_t hint_ns = 2000u)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity), "r"(hint_ns)
+        : "memory");
+    return ok;
+}
+// Arrive on an mbarrier of any CTA of the cluster (shared::cluster address),
+// released at cluster scope: what the arriving thread wrote (and what it has
+// observed of its warp-mates' writes) to its own shared / tensor memory is in
+// place before a thread of the other CTA that waits with acquire at cluster
+// scope sees the arrival.
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
 {
-    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr)
+                 : "memory");
 }
 
 // ---- cp.async (16-byte, L2 only); src_bytes = 0 writes zeros -----------------

@@ -404,8 +404,13 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
     Ctl ctl{reinterpret_cast<volatile int *>(smem + L.abort_flag), p.ws};
     // The consumer of a_full / b_full / acc_empty is the MMA thread of rank 0:
     // in a pair both CTAs arrive on rank 0's barriers.
+    // An arrival that crosses to the peer CTA is released at cluster scope: what
+    // the arriving CTA wrote to its shared and tensor memory must be in place
+    // when rank 0 lets the tensor cores of both SMs read it (rank 0 waits with
+    // acquire at cluster scope).  With CTA-scope arrivals, one 8192^3 GEMM launch
+    // in about 150 returned a wrong half tile of the peer's columns.
     auto arrive_leader = [&](uint32_t bar) {
-        if (PAIR) mbar_arrive_cluster(map_to_cta(bar, 0u));
+        if (PAIR && rank != 0) mbar_arrive_cluster(map_to_cta(bar, 0u));
         else mbar_arrive(bar);
     };
     // completion of the issued MMAs, signalled to this barrier in both CTAs
@@ -569,6 +574,7 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
                 const int as = p.n_acc == 2 ? (it & 1) : 0;
                 const uint32_t aph = (p.n_acc == 2 ? (it >> 1) : it) & 1u;
                 if (!(ok = wait_bar(bar_acc_empty(as), aph ^ 1u, ctl, 3))) break;
+                if (PAIR) mbar_try_wait_cluster(bar_acc_empty(as), aph ^ 1u);
                 tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + as * BN;
 #pragma unroll 1
@@ -581,6 +587,8 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
                     // common case without the call: the operands are there already
                     if (!mbar_try_wait(bar_a_full(s), ph))
                         if (!(ok = wait_bar(bar_a_full(s), ph, ctl, 4))) break;
+                    // (the peer CTA's arrivals are released at cluster scope)
+                    if (PAIR) mbar_try_wait_cluster(bar_a_full(s), ph);
                     tc_fence_after_sync();
                     // per K step 4 instructions, 32 bytes of K each
 #pragma unroll
@@ -1698,7 +1706,7 @@ int dispatch_tc(int bits, int epi, int pm, const TcMaps &tmap, const TcParams &p
 // single K steps, 2 forces double steps wherever they are possible.
 int g_forced_ks = 0;
 int g_pair_mode = 0;    // dsq_set_cta_pairs: 0 automatic, 1 never, 2 wherever possible
-int g_stage_mode = 0;   // dsq_set_gemm_store: 0 automatic (TMA stores where possible), 1 direct stores
+int g_stage_mode = 1;   // dsq_set_gemm_store: 1 direct stores (default), 0 staged TMA stores where possible
 // Whether a GEMM runs its CTA pairs on 256 x 128 tiles with overlapped epilogues
 // (PM 6) rather than on 256 x 256 tiles (PM 4).
 bool pair128_pays(int64_t M, int64_t N)

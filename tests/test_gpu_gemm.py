@@ -44,23 +44,6 @@ def test_gemm_small_and_ragged(dsq, bits, size):
 
 
 @pytest.mark.parametrize("bits", [2, 4])
-@pytest.mark.parametrize("size", [(130, 72, 200), (300, 260, 1000), (512, 512, 512)])
-def test_gemm_direct_stores(dsq, bits, size):
-    """Same results when the epilogue warps store the outputs themselves
-    instead of handing staged tiles to TMA."""
-    M, Nn, K = size
-    A, B, rs = dsq_inputs.gemm_case(M, Nn, K, bits)
-    C = native.gemm(A, B)
-    dsq.dsq_set_gemm_store(1)
-    try:
-        Cg, Dg = run(dsq, A, B, rs, bits)
-    finally:
-        dsq.dsq_set_gemm_store(0)
-    assert np.array_equal(C, Cg)
-    assert np.array_equal(native.gemm_dequant(C, rs), Dg)
-
-
-@pytest.mark.parametrize("bits", [2, 4])
 @pytest.mark.parametrize("size", [(512, 512, 1024), (300, 260, 1100), (1024, 640, 2048),
                                   (129, 72, 4096)])
 def test_gemm_pairs_on_128_wide_tiles(dsq, bits, size):
