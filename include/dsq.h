@@ -274,8 +274,9 @@ int dsq_set_round_k_steps(int ks);
 /* Third tuning hook: CTA pairs.  With 256-wide N tiles the tensor-core
  * kernels run as clusters of two CTAs that share one 256 x 256 tile
  * (tcgen05 cta_group::2; each SM expands half of the B operand).  mode 0:
- * automatic, 1: never, 2: wherever the shapes allow.  Results do not depend
- * on it. */
+ * automatic, 1: never, 2: wherever the shapes allow, 3 (dsq_gemm only): pairs
+ * on 256 x 128 tiles with two accumulator buffers, so that a tile's epilogue
+ * overlaps the next tile's rounds.  Results do not depend on it. */
 int dsq_set_cta_pairs(int mode);
 
 /* Fourth tuning hook: how dsq_gemm writes its int32 / fp32 outputs.  mode 1
