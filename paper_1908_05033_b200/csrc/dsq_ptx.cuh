@@ -110,6 +110,17 @@ __device__ __forceinline__ uint32_t mbar_try_wait_cluster(uint32_t bar, uint32_t
 // observed of its warp-mates' writes) to its own shared / tensor memory is in
 // place before a thread of the other CTA that waits with acquire at cluster
 // scope sees the arrival.
+// Same without the cluster-scope release (for arrivals that publish nothing the
+// peer SM reads).
+__device__ __forceinline__ void mbar_arrive_cluster_relaxed(uint32_t cluster_addr)
+{
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// Arrival on this CTA's own barrier, released at cluster scope.
+__device__ __forceinline__ void mbar_arrive_release_cluster(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.release.cluster.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
 {
     asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr)

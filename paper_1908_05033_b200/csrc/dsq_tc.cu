@@ -404,11 +404,14 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
     Ctl ctl{reinterpret_cast<volatile int *>(smem + L.abort_flag), p.ws};
     // The consumer of a_full / b_full / acc_empty is the MMA thread of rank 0:
     // in a pair both CTAs arrive on rank 0's barriers.
-    // An arrival that crosses to the peer CTA is released at cluster scope: what
-    // the arriving CTA wrote to its shared and tensor memory must be in place
-    // when rank 0 lets the tensor cores of both SMs read it (rank 0 waits with
-    // acquire at cluster scope).  With CTA-scope arrivals, one 8192^3 GEMM launch
-    // in about 150 returned a wrong half tile of the peer's columns.
+    // Memory ordering in a pair.  The expanded B halves in shared memory are read
+    // by the tensor cores of BOTH SMs, so the B warps of both CTAs release their
+    // arrivals at cluster scope and rank 0's MMA warp waits with acquire at
+    // cluster scope.  (With CTA-scope arrivals, one 8192^3 GEMM launch in about
+    // 150 returned a wrong block of 128 columns.)  The A operand sits in each
+    // SM's own tensor memory and is read by that SM's tensor core only: its
+    // arrivals need no cluster-scope release.  The epilogue warps' arrivals
+    // (accumulator handed back) cross with a cluster-scope release as well.
     auto arrive_leader = [&](uint32_t bar) {
         if (PAIR && rank != 0) mbar_arrive_cluster(map_to_cta(bar, 0u));
         else mbar_arrive(bar);
@@ -715,7 +718,12 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
             tmem_st_wait();
             tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) arrive_leader(bar_a_full(pend_s));
+            // (the A operand sits in this SM's tensor memory and only this SM's
+            // tensor core reads it: no cluster-scope release needed)
+            if (lane == 0) {
+                if (PAIR && rank != 0) mbar_arrive_cluster_relaxed(map_to_cta(bar_a_full(pend_s), 0u));
+                else mbar_arrive(bar_a_full(pend_s));
+            }
             pend_s = -1;
         };
         // TMA mode: slot = 128 rows of KS*CH chunks, chunk index XOR-swizzled
@@ -957,7 +965,9 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
                 fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0) {
-                    arrive_leader(p.b_res ? bar_b_full(su) : bar_a_full(su));
+                    // (a pair's B halves are read by the tensor cores of BOTH SMs)
+                    if (PAIR && rank == 0) mbar_arrive_release_cluster(bar_a_full(su));
+                    else arrive_leader(p.b_res ? bar_b_full(su) : bar_a_full(su));
                     mbar_arrive(bar_p_empty(sp));
                 }
             }
