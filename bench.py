@@ -39,7 +39,7 @@ import dsq_inputs  # noqa: E402
 # DRAM traffic of the dominant kernel (dsq_tc_kernel) per launch in this
 # workload, from one ncu capture (profiles/bench_launch_list.txt); valid only
 # for the kernel sources it was taken on (checked by hash)
-TRAFFIC = {"bytes_per_launch": 4728515, "sources_sha256": "7c194a4922733605aea74d4ff7aaf23c858202ab186e62b0f147320a40d3f543"}
+TRAFFIC = {"bytes_per_launch": 4728441, "sources_sha256": "89bc47d406d28b71028414db5fd3c069869ee66c86bb207ba91c8f00d996b40f"}
 
 WORKLOAD = "resnet18-shaped stack, 4-bit W/A, batch 64, 56x56x64 stem output, 19 convs"
 METRIC = "4-bit ResNet-18 conv-stack throughput (effective low-bit conv TOPS alongside)"
