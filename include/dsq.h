@@ -181,7 +181,10 @@ int dsq_conv2d(const void *act_codes, const dsq_nhwc_t *shape,
                float *y_f32, void *y_codes, int32_t *acc_out,
                void *workspace, size_t ws_bytes, void *stream);
 
-/* Depthwise 3x3 convolution on CUDA cores (not a dense contraction):
+/* Depthwise 3x3 convolution on CUDA cores (not a dense contraction; the
+ * depthwise layers of the MobileNetV2 rows of the paper's Table 7, each a
+ * quantised convolution in the sense of Algorithm 1 steps 1-5 with one filter
+ * per channel):
  * acc[n][ho][wo][c] = sum over the 3x3 taps of q_a * c_w, then the same
  * epilogue with per-channel S_a.  Same arguments as dsq_conv2d;
  * conv->groups = Cin = Cout = shape->C, KH = KW = 3, pad = 1, bits in {2,4}.
@@ -191,7 +194,10 @@ int dsq_dwconv2d(const void *act_codes, const dsq_nhwc_t *shape,
                  const dsq_conv_t *conv, const dsq_epilogue_t *ep,
                  float *y_f32, void *y_codes, int32_t *acc_out, void *stream);
 
-/* Plain low-bit GEMM on the tensor cores: C[m][n] = sum_k A[m][k] * B[n][k].
+/* Plain low-bit GEMM on the tensor cores: C[m][n] = sum_k A[m][k] * B[n][k]
+ * (paper Sec. 3.5: a quantised convolution is lowered to a GEMM over codes
+ * whose multiply-accumulates are the core operation; Algorithm 1 step 5 on
+ * codes, without the convolution's gather).
  *   A_codes   packed rows [M][K] of SIGNED codes
  *   B_codes   packed rows [N][K] of UNSIGNED codes
  *   C_i32     nullable: int32 [M][N]
@@ -234,8 +240,10 @@ int dsq_gemm_static_ws(const void *A_codes, const void *B_codes, int64_t M,
                        const float *row_scale, float *D_f32,
                        int wait_and_check, void *stream);
 
-/* 2x2 stride-2 max-pool on packed unsigned codes (exact on codes because the
- * quantiser is monotone).  H and W must be even. */
+/* 2x2 stride-2 max-pool on packed unsigned codes.  Exact on codes: the hard
+ * quantiser of Eq. 2 is monotone non-decreasing, so the maximum of the codes
+ * is the code of the maximum (pooling then Algorithm 1 steps 1, 3 equals
+ * steps 1, 3 then pooling).  H and W must be even. */
 int dsq_maxpool2x2(const void *codes_in, const dsq_nhwc_t *shape, int bits,
                    void *codes_out, size_t bytes, void *stream);
 
@@ -259,44 +267,6 @@ int dsq_unpack(const void *packed, int64_t rows, int64_t k, int bits,
  * to *macs_out (host).  Gives the denominator "measured INT8 peak". */
 int dsq_probe_i8_mma_rate(int iters, float *ms_out, double *macs_out,
                           void *workspace, size_t ws_bytes, void *stream);
-
-/* Tuning hook for the tensor-core kernels: force the tile width along N
- * (output channels) to 32, 64, 128, 192 or 256 for all later dsq_conv2d /
- * dsq_gemm calls of this process; 0 restores the automatic choice.  Results
- * do not depend on it. */
-int dsq_set_tile_n(int bn);
-
-/* Second tuning hook: K steps (of 128 codes) per pipeline round of the
- * tensor-core kernels, 1 or 2; 0 restores the automatic choice (2 whenever
- * the N tile is at most 128 wide).  Results do not depend on it. */
-int dsq_set_round_k_steps(int ks);
-
-/* Third tuning hook: CTA pairs.  With 256-wide N tiles the tensor-core
- * kernels run as clusters of two CTAs that share one 256 x 256 tile
- * (tcgen05 cta_group::2; each SM expands half of the B operand).  mode 0:
- * automatic, 1: never, 2: wherever the shapes allow, 3 (dsq_gemm only): pairs
- * on 256 x 128 tiles with two accumulator buffers, so that a tile's epilogue
- * overlaps the next tile's rounds.  Results do not depend on it. */
-int dsq_set_cta_pairs(int mode);
-
-/* Fourth tuning hook: how dsq_gemm writes its int32 / fp32 outputs.  mode 1
- * (the default): direct vector stores from the epilogue warps.  mode 0: each
- * epilogue warp stages its 32 x 32 block in shared memory and one TMA store
- * writes it, whenever N is a multiple of 4 and the staging tiles fit next to
- * the operand rings.  The staged path is kept for experiments only: with both
- * outputs requested, long runs of 8192^3 launches returned a wrong tile once
- * in a while and one run ended in a launch failure, cause not found. */
-int dsq_set_gemm_store(int mode);
-
-/* Fifth hook: programmatic dependent launch of the tensor-core kernels
- * (default on).  dsq_conv2d / dsq_gemm launch their kernel with the
- * programmatic stream-serialisation attribute: its set-up (barriers, tensor
- * memory, descriptor prefetch) may run while the previous kernel of the
- * stream is finishing, and it waits for that kernel to complete
- * (griddepcontrol.wait) before it reads or writes any global data, so stream
- * order is kept.  0 switches to plain launches.  Results do not depend on
- * it. */
-int dsq_set_dependent_launch(int on);
 
 /* ---- misc --------------------------------------------------------------- */
 const char *dsq_status_string(int status);

@@ -74,19 +74,24 @@ _SIGNATURES = {
     "dsq_unpack": (_int, [_vp, _i64, _i64, _int, _int, _vp, _vp]),
     "dsq_probe_i8_mma_rate": (_int, [_int, C.POINTER(C.c_float),
                                      C.POINTER(C.c_double), _vp, _sz, _vp]),
-    "dsq_set_tile_n": (_int, [_int]),
-    "dsq_set_round_k_steps": (_int, [_int]),
-    "dsq_set_cta_pairs": (_int, [_int]),
-    "dsq_set_gemm_store": (_int, [_int]),
-    "dsq_set_dependent_launch": (_int, [_int]),
     "dsq_status_string": (C.c_char_p, [_int]),
     "dsq_version": (_int, []),
 }
-for _name, (_res, _args) in _SIGNATURES.items():
+# tuning / test hooks (csrc/dsq_hooks.h; not part of include/dsq.h)
+_HOOKS = {
+    "dsq_set_tile_n": (_int, [_int]),
+    "dsq_set_round_k_steps": (_int, [_int]),
+    "dsq_set_cta_pairs": (_int, [_int]),
+    "dsq_set_dependent_launch": (_int, [_int]),
+    "dsq_set_wait_limit_ns": (_int, [C.c_longlong]),
+    "dsq_set_test_skip_b_round": (_int, [_int]),
+}
+for _name, (_res, _args) in list(_SIGNATURES.items()) + list(_HOOKS.items()):
     _f = getattr(lib, _name)       # AttributeError if a symbol is missing
     _f.restype, _f.argtypes = _res, _args
 
 EXPORTED_SYMBOLS = tuple(_SIGNATURES)
+HOOK_SYMBOLS = tuple(_HOOKS)
 
 
 class DsqError(RuntimeError):
@@ -329,8 +334,14 @@ def dsq_set_cta_pairs(mode):
     _check(lib.dsq_set_cta_pairs(mode), "dsq_set_cta_pairs")
 
 
-def dsq_set_gemm_store(mode):
-    _check(lib.dsq_set_gemm_store(mode), "dsq_set_gemm_store")
+def dsq_set_wait_limit_ns(ns):
+    """Test hook: limit of the kernels' barrier waits (0 = default 2 s)."""
+    _check(lib.dsq_set_wait_limit_ns(int(ns)), "dsq_set_wait_limit_ns")
+
+
+def dsq_set_test_skip_b_round(r):
+    """Test hook: the B producer leaves out round r (-1 = off)."""
+    _check(lib.dsq_set_test_skip_b_round(int(r)), "dsq_set_test_skip_b_round")
 
 
 def dsq_set_dependent_launch(on):
@@ -366,4 +377,5 @@ def dsq_probe_i8_mma_rate(iters, ws):
 
 
 __all__ = [n for n in dir() if n.startswith("dsq_")] + [
-    "lib", "DsqError", "EXPORTED_SYMBOLS", "new_workspace", "check_workspace"]
+    "lib", "DsqError", "EXPORTED_SYMBOLS", "HOOK_SYMBOLS", "new_workspace",
+    "check_workspace"]

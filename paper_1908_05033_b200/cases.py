@@ -55,7 +55,6 @@ def main(argv=None):
     ap.add_argument("--tile-n", type=int, default=0)
     ap.add_argument("--round-k", type=int, default=0)
     ap.add_argument("--pairs", type=int, default=0, help="0 auto, 1 never, 2 wherever possible")
-    ap.add_argument("--gemm-store", type=int, default=1, help="1 direct stores (default), 0 staged TMA stores")
     a = ap.parse_args(argv)
     dev = "cuda"
     ws = B.new_workspace(dev)
@@ -66,7 +65,6 @@ def main(argv=None):
     B.dsq_set_tile_n(a.tile_n)
     B.dsq_set_round_k_steps(a.round_k)
     B.dsq_set_cta_pairs(a.pairs)
-    B.dsq_set_gemm_store(a.gemm_store)
     out = {"case": a.case, "bits": bits, "tile_n": a.tile_n}
     if a.case == "gemm":
         n = a.size

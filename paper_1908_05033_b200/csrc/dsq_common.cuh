@@ -5,6 +5,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "../../include/dsq.h"
 
 #define DSQ_VERSION 100
@@ -12,11 +14,9 @@
 // Workspace layout (device memory owned by the caller).
 //   word 0 : status (0 = ok, else a dsq_status code written by a kernel)
 //   word 1 : detail of the first failure (which wait ran out)
-//   word 2 : dynamic tile counter of the tensor-core kernels
 #define DSQ_WS_BYTES 256
 #define DSQ_WS_STATUS 0
 #define DSQ_WS_DETAIL 1
-#define DSQ_WS_TILE 2
 
 #define DSQ_CUDA_TRY(expr)                          \
     do {                                            \
@@ -38,6 +38,24 @@ static inline int dsq_check_quant(const dsq_quant_t *q)
     if (!dsq_finite(q->lo) || !dsq_finite(q->hi) || !(q->hi > q->lo))
         return DSQ_ERR_RANGE;
     return DSQ_OK;
+}
+
+// Number of SMs of the current device (looked up once per device; 0 if the
+// runtime cannot tell).  Grids are sized from it.
+#define DSQ_MAX_DEVICES 64
+inline int dsq_sm_count()
+{
+    static std::atomic<int> cached[DSQ_MAX_DEVICES];
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0) return 0;
+    if (dev < DSQ_MAX_DEVICES) {
+        const int c = cached[dev].load(std::memory_order_relaxed);
+        if (c > 0) return c;
+    }
+    int sms = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+    if (dev < DSQ_MAX_DEVICES) cached[dev].store(sms, std::memory_order_relaxed);
+    return sms;
 }
 
 static inline int dsq_launch_status()

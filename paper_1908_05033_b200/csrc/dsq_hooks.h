@@ -1,0 +1,49 @@
+/*
+ * dsq_hooks.h - process-wide tuning and test hooks of the tensor-core kernels.
+ * Not part of the public interface (include/dsq.h): profiling tools and the
+ * test-suite use them to force a tiling or a pipeline, or to make a bounded
+ * wait run out.  Each hook sets one atomic integer that later dsq_conv2d /
+ * dsq_gemm calls read; results never depend on the tuning hooks.
+ */
+#ifndef DSQ_HOOKS_H_
+#define DSQ_HOOKS_H_
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Force the tile width along N (output channels): 32, 64, 128, 192 or 256;
+ * 0 restores the automatic choice. */
+int dsq_set_tile_n(int bn);
+
+/* K steps (of 128 codes) per pipeline round: 1 or 2; 0 = automatic. */
+int dsq_set_round_k_steps(int ks);
+
+/* CTA pairs (clusters of two CTAs on one 256 x 256 tile, tcgen05
+ * cta_group::2): 0 automatic, 1 never, 2 wherever the shapes allow. */
+int dsq_set_cta_pairs(int mode);
+
+/* Programmatic dependent launch of the tensor-core kernels (default 1): the
+ * kernel's set-up may overlap the tail of the previous kernel of the stream;
+ * it waits for that kernel (griddepcontrol.wait) before touching global
+ * memory.  0 = plain launches. */
+int dsq_set_dependent_launch(int on);
+
+/* Limit of every device-side barrier wait in nanoseconds (default 2 s; 0
+ * restores the default). */
+int dsq_set_wait_limit_ns(long long ns);
+
+/* Test hook: in every later launch the thread that issues the TMA copies of
+ * the packed B operand leaves out the copy of round `round` of its CTA
+ * (0 = the first) and issues nothing after it; -1 switches the hook off.
+ * The warps that wait for that copy then run into the wait limit: the kernel
+ * records DSQ_ERR_TIMEOUT in the workspace, every role leaves its loop,
+ * copies and MMAs already in flight are allowed to finish, tensor memory is
+ * freed and the kernel returns.  Nothing faults and nothing waits longer
+ * than the limit; the outputs of such a launch are undefined. */
+int dsq_set_test_skip_b_round(int round);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DSQ_HOOKS_H_ */

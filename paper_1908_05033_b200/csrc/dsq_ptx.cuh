@@ -105,22 +105,25 @@ __device__ __forceinline__ uint32_t mbar_try_wait_cluster(uint32_t bar, uint32_t
         : "memory");
     return ok;
 }
-// Arrive on an mbarrier of any CTA of the cluster (shared::cluster address),
-// released at cluster scope: what the arriving thread wrote (and what it has
-// observed of its warp-mates' writes) to its own shared / tensor memory is in
-// place before a thread of the other CTA that waits with acquire at cluster
-// scope sees the arrival.
-// Same without the cluster-scope release (for arrivals that publish nothing the
-// peer SM reads).
-__device__ __forceinline__ void mbar_arrive_cluster_relaxed(uint32_t cluster_addr)
+// Arrive on an mbarrier of any CTA of the cluster (shared::cluster address)
+// with the default semantics of mbarrier.arrive (release at CTA scope).  For
+// arrivals that publish no memory the waiting CTA reads: the signal itself is
+// an atomic update of the barrier object in its home shared memory and is
+// seen by the waiter whatever the scope.
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr)
 {
     asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
-// Arrival on this CTA's own barrier, released at cluster scope.
+// Arrival on this CTA's own barrier, released at cluster scope: what the
+// arriving thread wrote (and what it has observed of its warp-mates' writes)
+// to shared memory is in place before a thread that waits with acquire at
+// cluster scope sees the arrival - and therefore before the tensor core of
+// the peer SM, started by that thread, reads it.
 __device__ __forceinline__ void mbar_arrive_release_cluster(uint32_t bar)
 {
     asm volatile("mbarrier.arrive.release.cluster.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
+// Same on a barrier of any CTA of the cluster (shared::cluster address).
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
 {
     asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr)
@@ -210,33 +213,6 @@ __device__ __forceinline__ void tma_load_im2col_4d(uint32_t dst, const CUtensorM
         " [%0], [%1, {%2, %3, %4, %5}], [%6], {%7, %8};" ::"r"(dst),
         "l"(m), "r"(c), "r"(w), "r"(h), "r"(n), "r"(bar), "h"(off_w), "h"(off_h)
         : "memory");
-}
-
-// 2-D tiled store, shared -> global, tracked by the issuing thread's bulk async
-// group.  Elements of the box outside the tensor are not written.  x * element
-// size must be a multiple of 16 bytes; neither coordinate may be negative.
-__device__ __forceinline__ void tma_store_2d(const CUtensorMap *m, uint32_t src, int x, int y)
-{
-    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];" ::"l"(m),
-                 "r"(x), "r"(y), "r"(src)
-                 : "memory");
-}
-__device__ __forceinline__ void bulk_commit_group()
-{
-    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-}
-// Waits until the bulk groups of this thread, except the newest N, have finished
-// READING their shared-memory source (the buffer may then be rewritten).
-template <int N>
-__device__ __forceinline__ void bulk_wait_group_read()
-{
-    asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
-}
-__device__ __forceinline__ void sts_128(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d)
-{
-    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c),
-                 "r"(d)
-                 : "memory");
 }
 
 // ---- tensor memory ---------------------------------------------------------

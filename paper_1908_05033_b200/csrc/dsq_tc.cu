@@ -23,9 +23,8 @@
 //      memory), accumulating int32 in tensor memory (two accumulator buffers
 //      where they fit beside the A stages)
 //   epilogue warps read tensor memory (tcgen05.ld), apply the dequantise /
-//      requantise epilogue and write codes / fp32 / int32 (GEMM outputs go
-//      through swizzled staging tiles and TMA stores); on a CTA's last tile
-//      the A and B warps join them.
+//      requantise epilogue and write codes / fp32 / int32 with vector stores;
+//      on a CTA's last tile the A and B warps join them.
 //
 // Each role's loop is a chain of hand-offs (barrier wait, expect, TMA or MMA
 // issue, commit); one hand-off costs a few hundred cycles while the unpack
@@ -49,6 +48,7 @@
 #include <cuda.h>
 
 #include "dsq_epilogue.cuh"
+#include "dsq_hooks.h"
 #include "dsq_ptx.cuh"
 
 using namespace dsq_ptx;
@@ -85,23 +85,14 @@ constexpr int BK_BYTES = 128;         // int8 bytes per row per K step (128 code
 //         expect, a TMA issue, a commit) costs a few hundred cycles whatever the
 //         amount of data behind it, so a tile pays for them once instead of
 //         once per K step; the two A groups take alternate tiles.
-//   PM 6: CTA PAIR on 256 x 128 tiles, KS = 4, 2 stages, TWO accumulator buffers:
-//         the epilogue of a tile (whose int32 / fp32 output is as large as the
-//         packed operands it came from) overlaps the next tile's rounds, which the
-//         256-wide pair tile cannot do (its accumulator and the A stages fill
-//         the 512 tensor-memory columns).  A round is two half rounds for the A
-//         side: each A group expands two of the four K steps of every round.
 constexpr int SU_MAX = 4;
 template <int PM> struct Pipe {
-    static constexpr int KS = PM == 1 ? 1 : PM == 5 ? 5 : PM == 6 ? 4 : 2;
+    static constexpr int KS = PM == 1 ? 1 : PM == 5 ? 5 : 2;
     static constexpr bool WIDE = PM == 3;
-    static constexpr bool PAIR = PM == 4 || PM == 6;
-    // A half rounds per barrier round (each A group takes one half of every round)
-    static constexpr int HALVES = PM == 6 ? 2 : 1;
-    static constexpr int KSA = KS / HALVES;                  // K steps of an A step
+    static constexpr bool PAIR = PM == 4;
     static constexpr bool WHOLE_K = PM == 5;
     // stages of expanded operands
-    static constexpr int SU = PM == 1 ? 4 : (PM == 3 || PM == 5 || PM == 6) ? 2 : 3;
+    static constexpr int SU = PM == 1 ? 4 : (PM == 3 || PM == 5) ? 2 : 3;
     static constexpr int GROUPS = WIDE ? 1 : 2;              // A groups in use
     static constexpr int A_D = PM == 1 ? 2 : 1;              // own A rounds in flight per thread
     static constexpr int A_RING = A_D + 1;                   // packed A ring slots per group
@@ -129,7 +120,9 @@ static_assert(WARP_A0 + NUM_A_WARPS == WARP_B0 && WARP_B0 + NUM_B_WARPS == WARP_
                   WARP_E0 + NUM_E_WARPS == WARP_TMA_A && WARP_TMA_A + 1 == NUM_WARPS,
               "warp roles");
 constexpr int NUM_THREADS = NUM_WARPS * 32;
-constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;   // a wait gives up after 2 s
+constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;   // default: a wait gives up after 2 s
+// once a CTA has given up, copies and MMAs already in flight get this long to land
+constexpr unsigned long long DRAIN_LIMIT_NS = 20000000ull;
 
 enum { MODE_CONV = 0, MODE_GEMM = 1 };
 // epilogue variants (template parameter): GEMM; convolution writing codes
@@ -146,10 +139,13 @@ struct TcParams {
     // join = 1: on the CTA's last tile the A and B warps join the epilogue (needs
     // a scale / bias staging slot for each of the 20 warps in shared memory)
     int join;
-    // stage = 1 (GEMM): the epilogue warps hand their 32 x 32 output blocks to TMA
-    // through a shared-memory staging tile instead of storing them themselves
-    int stage;
     int smem_bytes;                   // dynamic shared memory given to the launch
+    // every wait on a barrier gives up after this many nanoseconds
+    unsigned long long wait_ns;
+    // test hook (dsq_set_test_skip_b_round): the B producer leaves out the copy
+    // of this round (counted over the CTA's rounds; -1 = none) and stops, so
+    // that the wait on it runs out
+    int skip_b_round;
     // A gather geometry (a GEMM is a 1x1 convolution over an M x 1 image)
     const uint8_t *act;
     int H, W, Ho, Wo, stride, pad, KW, taps, P;
@@ -190,25 +186,59 @@ struct TcParams {
 struct Ctl {
     volatile int *abort_flag;   // shared memory
     int *ws;
+    unsigned long long limit_ns;
 };
 
-// Not inlined on purpose: the kernel has a dozen wait sites and its code must
-// stay small enough for the instruction caches.
-__device__ __noinline__ bool wait_bar(uint32_t bar, uint32_t parity, const Ctl &c, int tag)
+// Slow path of a wait.  Not inlined on purpose: the kernel has a dozen wait
+// sites and its code must stay small enough for the instruction caches.
+// CLUSTER: acquire at cluster scope (the barrier also collects arrivals that
+// threads of the peer CTA released at cluster scope).
+template <bool CLUSTER>
+__device__ __noinline__ bool wait_bar_slow(uint32_t bar, uint32_t parity, const Ctl &c, int tag)
 {
-    if (mbar_try_wait(bar, parity)) return true;
     const uint64_t t0 = global_timer_ns();
     for (uint32_t it = 1;; ++it) {
-        if (mbar_try_wait(bar, parity)) return true;
+        if (CLUSTER ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity)) return true;
         if ((it & 63u) == 0u) {
             if (*c.abort_flag) return false;
-            if (global_timer_ns() - t0 > WAIT_LIMIT_NS) break;
+            if (global_timer_ns() - t0 > c.limit_ns) break;
         }
     }
     if (atomicCAS(c.ws + DSQ_WS_STATUS, 0, (int)DSQ_ERR_TIMEOUT) == 0)
         c.ws[DSQ_WS_DETAIL] = tag;
     *c.abort_flag = 1;
     return false;
+}
+
+// Bounded wait of ONE thread (the TMA producer threads).
+__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, const Ctl &c, int tag)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    return wait_bar_slow<false>(bar, parity, c, tag);
+}
+
+// Bounded wait of a whole converged warp.  All 32 lanes get the same answer:
+// the code behind a wait holds warp-wide instructions (tcgen05.ld / st,
+// __syncwarp), so the lanes must not part ways when one of them sees the phase
+// complete and another the abort flag.
+template <bool CLUSTER = false>
+__device__ __forceinline__ bool wait_bar_warp(uint32_t bar, uint32_t parity, const Ctl &c, int tag)
+{
+    bool ok = CLUSTER ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity);
+    if (!ok) ok = wait_bar_slow<CLUSTER>(bar, parity, c, tag);
+    return __all_sync(0xffffffffu, ok);
+}
+
+// Wait used while leaving after a failure: ignores the abort flag (what is in
+// flight must still land before shared or tensor memory is given up), bounded
+// by DRAIN_LIMIT_NS.
+__device__ __noinline__ void wait_bar_drain(uint32_t bar, uint32_t parity)
+{
+    const uint64_t t0 = global_timer_ns();
+    for (uint32_t it = 1;; ++it) {
+        if (mbar_try_wait(bar, parity)) return;
+        if ((it & 15u) == 0u && global_timer_ns() - t0 > DRAIN_LIMIT_NS) return;
+    }
 }
 
 // ---------------------------------------------------------------------------
@@ -300,12 +330,10 @@ constexpr int MAX_A_SLOTS = 6;
 constexpr int MAX_B_STAGES = 16;
 
 constexpr int JOIN_CNT = 5;               // warps per lane quarter in a joined epilogue
-// 256-byte slots behind the rings: scale / bias staging of the epilogue warps,
-// or (stage = 1, GEMM) one 4 KB output staging tile per epilogue warp, 1024-byte
-// aligned, from which TMA stores the int32 / fp32 rows
-__host__ __device__ inline int epi_slots(int join, int epw, int stage = 0)
+// 256-byte slots behind the rings: scale / bias staging of the epilogue warps
+__host__ __device__ inline int epi_slots(int join, int epw)
 {
-    return stage ? 4 * epw * 16 + 4 : join ? 4 * JOIN_CNT : 4 * epw;
+    return join ? 4 * JOIN_CNT : 4 * epw;
 }
 
 __host__ __device__ inline SmemLayout smem_layout(int BN, int bits, int s_p, int b_stages, int ks,
@@ -319,7 +347,7 @@ __host__ __device__ inline SmemLayout smem_layout(int BN, int bits, int s_p, int
     // per-warp scale / bias staging (any warp may take part in an epilogue)
     L.epi = o;      o += epi_slots * 64 * 4;
     o = (o + 127u) & ~127u;
-    L.bars = o;     o += 8 * (2 * SU_MAX + MAX_B_STAGES + 2 * MAX_S_P + 4 + 2 * MAX_A_SLOTS + 1);
+    L.bars = o;     o += 8 * (2 * SU_MAX + MAX_B_STAGES + 2 * MAX_S_P + 4 + 2 * MAX_A_SLOTS + 2);
     L.tmem_slot = o; o += 8;
     L.abort_flag = o; o += 8;
     L.total = o;
@@ -332,9 +360,7 @@ __host__ __device__ inline SmemLayout smem_layout(int BN, int bits, int s_p, int
 template <int BITS, bool A_SIGNED, int EPI, int PM, int A_TMA>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
-              const __grid_constant__ CUtensorMap tmap_a,
-              const __grid_constant__ CUtensorMap tmap_c,
-              const __grid_constant__ CUtensorMap tmap_d, const TcParams p)
+              const __grid_constant__ CUtensorMap tmap_a, const TcParams p)
 {
     constexpr bool B_SIGNED = !A_SIGNED;
     constexpr int CH = Chunks<BITS>::CH;
@@ -346,8 +372,7 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
     constexpr int S_U = Pipe<PM>::SU, A_D = Pipe<PM>::A_D, A_RING = Pipe<PM>::A_RING;
     constexpr int A_COL0 = Pipe<PM>::A_COL0;
     constexpr int A_SLOTS = GROUPS * A_RING;                // packed A ring slots
-    constexpr int HALVES = Pipe<PM>::HALVES, KSA = Pipe<PM>::KSA;
-    constexpr int A_SLOT_BYTES = KSA * CH * BM * 16;        // one A step of 128 rows
+    constexpr int A_SLOT_BYTES = KS * CH * BM * 16;         // one round of 128 rows
     static_assert(A_SLOTS <= MAX_A_SLOTS, "A ring barriers");
     static_assert(KS == 1 || BITS != 3, "3-bit rows use single K steps");
     extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -356,12 +381,15 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
     const int BN = p.BN;
     const int BNL = BN / CG;                  // B rows this CTA expands
     const SmemLayout L =
-        smem_layout(BNL, BITS, p.s_p, p.b_stages, KS, GROUPS * A_RING / HALVES,
-                    epi_slots(p.join, p.epw, p.stage));
+        smem_layout(BNL, BITS, p.s_p, p.b_stages, KS, GROUPS * A_RING,
+                    epi_slots(p.join, p.epw));
     // the layout must fit behind the 1024-byte aligned base (the host adds
     // slack only while it stays within the 227 KB limit); same answer in every
     // thread of every CTA, taken before any barrier exists
     if ((uint32_t)(smem - smem_raw) + L.total > (uint32_t)p.smem_bytes) {
+        // (global memory, the workspace included, is touched only once the
+        // kernels before this one have completed)
+        grid_dependency_wait();
         if (threadIdx.x == 0) atomicCAS(p.ws + DSQ_WS_STATUS, 0, (int)DSQ_ERR_UNSUPPORTED);
         return;
     }
@@ -400,18 +428,22 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
     };
     // completes once, when the accumulators of this CTA's last tile are final
     const uint32_t bar_last_full = bars + 8u * (BAR_P + 2 * MAX_S_P + 4 + 2 * MAX_A_SLOTS);
+    // used once, by an MMA warp that gives up: completion of what it had issued
+    const uint32_t bar_drain = bar_last_full + 8u;
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + L.tmem_slot);
-    Ctl ctl{reinterpret_cast<volatile int *>(smem + L.abort_flag), p.ws};
+    Ctl ctl{reinterpret_cast<volatile int *>(smem + L.abort_flag), p.ws, p.wait_ns};
     // The consumer of a_full / b_full / acc_empty is the MMA thread of rank 0:
     // in a pair both CTAs arrive on rank 0's barriers.
     // Memory ordering in a pair.  The expanded B halves in shared memory are read
     // by the tensor cores of BOTH SMs, so the B warps of both CTAs release their
-    // arrivals at cluster scope and rank 0's MMA warp waits with acquire at
-    // cluster scope.  (With CTA-scope arrivals, one 8192^3 GEMM launch in about
-    // 150 returned a wrong block of 128 columns.)  The A operand sits in each
-    // SM's own tensor memory and is read by that SM's tensor core only: its
-    // arrivals need no cluster-scope release.  The epilogue warps' arrivals
-    // (accumulator handed back) cross with a cluster-scope release as well.
+    // arrivals at cluster scope and rank 0's MMA warp spins on the barrier with
+    // acquire at cluster scope (wait_bar_warp<true>).  (With CTA-scope arrivals,
+    // one 8192^3 GEMM launch in about 150 returned a wrong block of 128
+    // columns.)  The A operand sits in each SM's own tensor memory, is complete
+    // there before its arrival (tcgen05.wait::st) and is read by that SM's
+    // tensor core only: those arrivals publish no memory and keep the default
+    // scope.  The epilogue warps' arrivals (accumulator handed back) cross with
+    // a cluster-scope release as well.
     auto arrive_leader = [&](uint32_t bar) {
         if (PAIR && rank != 0) mbar_arrive_cluster(map_to_cta(bar, 0u));
         else mbar_arrive(bar);
@@ -427,7 +459,7 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
         for (int s = 0; s < S_U; ++s) {
             // operands of a round: the four warps of one A group and (unless the
             // expanded B tile is resident) the B warps, of every CTA of the pair
-            mbar_init(bar_a_full(s), (4 * HALVES + (p.b_res ? 0 : NUM_B_WARPS / B_GROUPS)) * CG);
+            mbar_init(bar_a_full(s), (4 + (p.b_res ? 0 : NUM_B_WARPS / B_GROUPS)) * CG);
             mbar_init(bar_u_empty(s), 1);    // tcgen05.commit
         }
         for (int s = 0; s < MAX_B_STAGES; ++s) mbar_init(bar_b_full(s), NUM_B_WARPS * CG);
@@ -444,6 +476,7 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
             mbar_init(bar_acc_empty(s), 4 * p.epw * CG);
         }
         mbar_init(bar_last_full, 1);         // tcgen05.commit
+        mbar_init(bar_drain, 1);             // tcgen05.commit
         *ctl.abort_flag = 0;
         mbar_init_fence();
     }
@@ -487,6 +520,7 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
 #pragma unroll 1
             for (; g < n_b_steps; ++g) {
                 if (!wait_bar(bar_p_empty(s), ph ^ 1u, ctl, 1)) break;
+                if ((int)g == p.skip_b_round) break;
                 mbar_arrive_expect_tx(bar_p_full(s), b_packed_bytes);
                 if (Pipe<PM>::WHOLE_K) {
                     // a box is at most 256 bytes wide: one box per K step, stored
@@ -506,12 +540,12 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
             }
             // let outstanding copies land before the CTA can exit
             for (uint32_t k = (issued_b > (uint32_t)S_P ? issued_b - S_P : 0); k < issued_b; ++k)
-                wait_bar(bar_p_full(k % S_P), (k / S_P) & 1u, ctl, 2);
+                wait_bar_drain(bar_p_full(k % S_P), (k / S_P) & 1u);
         }
     } else if (warp == WARP_TMA_A) {
         // ---------------- producer: TMA packed A boxes -----------------------
         if (A_TMA && lane == 0) {
-            const int a_steps_tile = p.rounds * HALVES;          // A steps per tile
+            const int a_steps_tile = p.rounds;                   // A steps per tile
             const uint32_t n_a_steps = (uint32_t)my_tiles_all * a_steps_tile;
             const uint32_t ring = smem_u32(smem + L.a_ring);
             uint32_t g = 0, issued_a = 0;
@@ -530,7 +564,7 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
                                 bar_ar_full(sl));
                 } else if (p.a_tma == 1) {
                     mbar_arrive_expect_tx(bar_ar_full(sl), A_SLOT_BYTES);
-                    tma_load_2d(ring + sl * A_SLOT_BYTES, &tmap_a, ka * (KSA * 16 * BITS), m0,
+                    tma_load_2d(ring + sl * A_SLOT_BYTES, &tmap_a, ka * (KS * 16 * BITS), m0,
                                 bar_ar_full(sl));
                 } else {
                     if (ka == 0) {                 // first pixel of the tile, first tap
@@ -560,7 +594,7 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
             }
             for (uint32_t k = (issued_a > (uint32_t)A_SLOTS ? issued_a - A_SLOTS : 0);
                  k < issued_a; ++k)
-                wait_bar(bar_ar_full(k % A_SLOTS), (k / A_SLOTS) & 1u, ctl, 2);
+                wait_bar_drain(bar_ar_full(k % A_SLOTS), (k / A_SLOTS) & 1u);
         }
     } else if (warp == WARP_MMA) {
         // ---------------- MMA issuer ---------------------------------------
@@ -576,8 +610,8 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
             for (int tile = tile0; ok && tile < total_tiles; tile += tstep, ++it) {
                 const int as = p.n_acc == 2 ? (it & 1) : 0;
                 const uint32_t aph = (p.n_acc == 2 ? (it >> 1) : it) & 1u;
-                if (!(ok = wait_bar(bar_acc_empty(as), aph ^ 1u, ctl, 3))) break;
-                if (PAIR) mbar_try_wait_cluster(bar_acc_empty(as), aph ^ 1u);
+                // (in a pair the peer CTA's arrivals were released at cluster scope)
+                if (!(ok = wait_bar_warp<PAIR>(bar_acc_empty(as), aph ^ 1u, ctl, 3))) break;
                 tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + as * BN;
 #pragma unroll 1
@@ -586,12 +620,8 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
                     const uint32_t ph = (g / S_U) & 1u;
                     const int bs = p.b_res ? ks : s;
                     if (p.b_res && it == 0)
-                        if (!(ok = wait_bar(bar_b_full(bs), 0u, ctl, 10))) break;
-                    // common case without the call: the operands are there already
-                    if (!mbar_try_wait(bar_a_full(s), ph))
-                        if (!(ok = wait_bar(bar_a_full(s), ph, ctl, 4))) break;
-                    // (the peer CTA's arrivals are released at cluster scope)
-                    if (PAIR) mbar_try_wait_cluster(bar_a_full(s), ph);
+                        if (!(ok = wait_bar_warp<PAIR>(bar_b_full(bs), 0u, ctl, 10))) break;
+                    if (!(ok = wait_bar_warp<PAIR>(bar_a_full(s), ph, ctl, 4))) break;
                     tc_fence_after_sync();
                     // per K step 4 instructions, 32 bytes of K each
 #pragma unroll
@@ -605,6 +635,13 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
                     commit_all(bar_acc_full(as));
                     if (tile + tstep >= total_tiles) commit_all(bar_last_full);
                 }
+            }
+            if (!ok) {
+                // giving up: instructions already issued may still be reading the
+                // operands and writing the accumulators; they must have finished
+                // before shared and tensor memory are given up
+                commit_all(bar_drain);
+                wait_bar_drain(bar_drain, 0u);
             }
         }
     } else if (warp < WARP_B0) {
@@ -708,7 +745,7 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
                 if (load && ++ld_slot == A_RING) ld_slot = 0;
             }
         };
-        const uint32_t n_steps = (uint32_t)my_tiles_all * p.rounds * HALVES;
+        const uint32_t n_steps = (uint32_t)my_tiles_all * p.rounds;
         // own steps: g = group, group + GROUPS, ...
         const uint32_t n_own =
             GROUPS == 1 ? n_steps : (n_steps > (uint32_t)group ? (n_steps - group + 1) / 2 : 0u);
@@ -718,10 +755,15 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
             tmem_st_wait();
             tc_fence_before_sync();
             __syncwarp();
-            // (the A operand sits in this SM's tensor memory and only this SM's
-            // tensor core reads it: no cluster-scope release needed)
+            // The A operand sits in this SM's tensor memory and only this SM's
+            // tensor core reads it.  tcgen05.wait::st above returns once the
+            // stores have COMPLETED (the data is in tensor memory; completion
+            // of a tcgen05 operation carries no scope), and
+            // tcgen05.fence::before_thread_sync orders it before the arrival:
+            // the crossing arrival publishes no memory of its own, so it needs
+            // no cluster-scope release.
             if (lane == 0) {
-                if (PAIR && rank != 0) mbar_arrive_cluster_relaxed(map_to_cta(bar_a_full(pend_s), 0u));
+                if (PAIR && rank != 0) mbar_arrive_remote(map_to_cta(bar_a_full(pend_s), 0u));
                 else mbar_arrive(bar_a_full(pend_s));
             }
             pend_s = -1;
@@ -751,19 +793,16 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
             const uint32_t g = GROUPS * (i - A_D) + group;
             const int aslot = (int)(g % A_SLOTS);
             if (a_tma) {
-                if (!(ok = wait_bar(bar_ar_full(aslot), (g / A_SLOTS) & 1u, ctl, 12))) break;
+                if (!(ok = wait_bar_warp(bar_ar_full(aslot), (g / A_SLOTS) & 1u, ctl, 12))) break;
             } else {
                 cp_async_wait<A_D>();              // own step i - A_D has landed
                 if (Pipe<PM>::COAL) __syncwarp();  // ... the other lanes' copies of my row too
             }
-            // A step g is half (g % HALVES) of barrier round g / HALVES
-            const uint32_t rg = g / HALVES;
-            const int half = (int)(g % HALVES);
-            const int s = rg % S_U;
-            const uint32_t ph = (rg / S_U) & 1u;
+            const int s = g % S_U;
+            const uint32_t ph = (g / S_U) & 1u;
             // chunks of this round that exist (im2col: nothing is loaded past the
             // last filter tap)
-            int kvalid = KSA * CH;
+            int kvalid = KS * CH;
             // rows mode: where this thread's pixel lies in the staged image rows
             constexpr int CPP = BITS / 2;              // 16-byte chunks per pixel (64 channels)
             constexpr bool rows_mode = Pipe<PM>::WHOLE_K && BITS != 3 && A_TMA == 3;
@@ -784,13 +823,13 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
                 sw16 = CPP == 2 ? (uint32_t)((lane >> 2) & 1) << 4 : 0u;
             }
             if (a_tma) {
-                if (p.a_tma == 2) kvalid = p.a_kchunks - kr * (KSA * CH);
+                if (p.a_tma == 2) kvalid = p.a_kchunks - kr * (KS * CH);
                 kr += GROUPS;
                 if (kr >= p.rounds) kr -= p.rounds;
                 if (kr >= p.rounds) kr -= p.rounds;
             }
 #pragma unroll
-            for (int h = 0; h < KSA; ++h) {
+            for (int h = 0; h < KS; ++h) {
                 uint32_t o[32];
                 {
                     uint4 cur[CH];
@@ -828,12 +867,12 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
                     expand_row_regs<BITS, A_SIGNED>(cur, p.orv, o);
                 }
                 if (h == 0) {
-                    if (!(ok = wait_bar(bar_u_empty(s), ph ^ 1u, ctl, 5))) break;
+                    if (!(ok = wait_bar_warp(bar_u_empty(s), ph ^ 1u, ctl, 5))) break;
                     tc_fence_after_sync();
                 }
                 __syncwarp();
                 tmem_st_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + A_COL0 +
-                                  (s * KS + half * KSA + h) * 32, o);
+                                  (s * KS + h) * 32, o);
             }
             if (!ok) break;
             if (++rd_slot == A_RING) rd_slot = 0;
@@ -865,8 +904,8 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
         // being a multiple of 128 bytes apart); (row & 7) does not depend on i
         constexpr int CHK = KS * CH;
         constexpr int ROWS_PER_IT = (BITS == 3) ? BT : BT / CH;
-        // (pairs expand half of a tile's B rows; PM 6 tiles are 128 wide)
-        constexpr int MAX_IT = (BITS == 3) ? 1 : ((PM == 6 ? 64 : PAIR ? 128 : 256) * CH) / BT;
+        // (pairs expand half of a tile's B rows)
+        constexpr int MAX_IT = (BITS == 3) ? 1 : ((PAIR ? 128 : 256) * CH) / BT;
         const int row0 = (BITS == 3) ? tid : tid / CH;
         const int j = (BITS == 3) ? 0 : tid % CH;
         const int sw = row0 & 7;
@@ -881,7 +920,7 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
                 if (sp >= S_P) { sp -= S_P; php ^= 1u; }
                 const int su = p.b_res ? (int)g : (int)(g % S_U);
                 const uint32_t phu = (g / S_U) & 1u;
-                if (!(ok = wait_bar(bar_p_full(sp), php, ctl, 6))) break;
+                if (!(ok = wait_bar_warp(bar_p_full(sp), php, ctl, 6))) break;
                 const uint8_t *src = smem + L.b_packed + sp * b_packed_bytes;
                 uint8_t *dst = smem + L.b_tiles + su * b_tile_bytes;
                 if (BITS == 3) {
@@ -895,7 +934,7 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
                             w[4 * l + 2] = v.z; w[4 * l + 3] = v.w;
                         }
                     }
-                    if (!p.b_res && !(ok = wait_bar(bar_u_empty(su), phu ^ 1u, ctl, 7))) break;
+                    if (!p.b_res && !(ok = wait_bar_warp(bar_u_empty(su), phu ^ 1u, ctl, 7))) break;
                     if (row0 < BNL) {
                         uint8_t *rowp = dst + row0 * BK_BYTES;
 #pragma unroll
@@ -940,7 +979,7 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
                                     src)[(row0 + i * ROWS_PER_IT) * CHK +
                                          ((h + rot) & (KSV - 1)) * CH + j];
                         }
-                    if (!p.b_res && !(ok = wait_bar(bar_u_empty(su), phu ^ 1u, ctl, 7))) break;
+                    if (!p.b_res && !(ok = wait_bar_warp(bar_u_empty(su), phu ^ 1u, ctl, 7))) break;
                     uint8_t *rowp = dst + row0 * BK_BYTES;
 #pragma unroll
                     for (int i = 0; i < MAX_IT; ++i) {
@@ -1007,8 +1046,8 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
             const bool row_ok = m < p.M;
             // helpers have not followed the accumulator barriers' phases: they wait
             // on the single-use barrier of the last tile
-            if (!(ok = epi_idx >= 0 ? wait_bar(bar_acc_full(as), aph, ctl, 8)
-                                    : wait_bar(bar_last_full, 0u, ctl, 13)))
+            if (!(ok = epi_idx >= 0 ? wait_bar_warp(bar_acc_full(as), aph, ctl, 8)
+                                    : wait_bar_warp(bar_last_full, 0u, ctl, 13)))
                 break;
             tc_fence_after_sync();
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + as * BN;
@@ -1043,42 +1082,6 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
                 }
                 tmem_ld_wait();
                 const int n0 = n_tile * BN + c0;
-                if (EPI == EPI_GEMM && p.stage) {
-                    // the warp's 32 rows x 32 columns go through a 128-byte-swizzled
-                    // staging tile to one TMA store (rows / columns past the matrix
-                    // are clipped by the store): the LSU sees 8 conflict-free shared
-                    // stores per lane instead of 32-byte pieces of 32 different lines
-                    const uint32_t stg =
-                        ((smem_u32(smem + L.epi) + 1023u) & ~1023u) +
-                        (uint32_t)(my_idx * 4 + quarter) * 4096u + (uint32_t)lane * 128u;
-                    const int y0 = m_tile * BMT + row_base + quarter * 32;
-#pragma unroll
-                    for (int c = 0; c < 32; ++c) r[c] = (uint32_t)((int)r[c] >> p.shift);
-#pragma unroll 1
-                    for (int o = 0; o < 2; ++o) {
-                        if (o == 0 ? p.C_i32 == nullptr : p.D_f32 == nullptr) continue;
-                        // the previous store has finished reading the tile
-                        if (lane == 0) bulk_wait_group_read<0>();
-                        __syncwarp();
-#pragma unroll
-                        for (int v = 0; v < 8; ++v) {
-                            uint32_t w[4];
-#pragma unroll
-                            for (int u = 0; u < 4; ++u)
-                                w[u] = o == 0 ? r[4 * v + u]
-                                              : __float_as_uint(
-                                                    __fmul_rn((float)(int)r[4 * v + u], rs));
-                            sts_128(stg + (uint32_t)((v ^ (lane & 7)) << 4), w[0], w[1], w[2], w[3]);
-                        }
-                        fence_proxy_async_smem();
-                        __syncwarp();
-                        if (lane == 0) {
-                            tma_store_2d(o == 0 ? &tmap_c : &tmap_d, stg, n0, y0);
-                            bulk_commit_group();
-                        }
-                    }
-                    continue;
-                }
                 if (!row_ok) continue;
 #pragma unroll
                 for (int c = 0; c < 32; ++c) r[c] = (uint32_t)((int)r[c] >> p.shift);
@@ -1286,8 +1289,6 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
     }
 
     // ---------------- teardown ---------------------------------------------
-    // (staged output tiles must have been read before the shared memory goes)
-    if (EPI == EPI_GEMM && p.stage && lane == 0) bulk_wait_group_read<0>();
     tc_fence_before_sync();
     __syncthreads();
     // a CTA of a pair stays until its peer has stopped signalling its barriers
@@ -1332,7 +1333,7 @@ __global__ void __launch_bounds__(128, 1) mma_rate_kernel(int iters, int *ws)
     tc_fence_after_sync();
     const uint32_t tmem = tmem_slot;
     if (threadIdx.x == 0) {
-        Ctl ctl{&abort_flag, ws};
+        Ctl ctl{&abort_flag, ws, WAIT_LIMIT_NS};
         const uint32_t idesc = idesc_i8(256, true, false);
         const uint64_t ad = smem_desc_sw128(smem_u32(smem));
         const uint64_t bd = smem_desc_sw128(smem_u32(smem + 128 * 128));
@@ -1385,7 +1386,7 @@ EncodeTiledFn get_encode_fn()
 }
 
 // 2-D byte map over packed rows: inner dimension = row bytes, outer = rows.
-struct TcMaps { CUtensorMap b, a, c, d; };   // operands; GEMM outputs (int32 C, fp32 D)
+struct TcMaps { CUtensorMap b, a; };   // the two operands
 
 int make_rows_tmap(CUtensorMap *map, const void *base, uint64_t row_bytes, uint64_t rows,
                    uint64_t pitch, uint32_t box_bytes, uint32_t box_rows,
@@ -1404,30 +1405,13 @@ int make_rows_tmap(CUtensorMap *map, const void *base, uint64_t row_bytes, uint6
     return r == CUDA_SUCCESS ? DSQ_OK : DSQ_ERR_CUDA;
 }
 
-// Row-major M x N matrix of 4-byte elements, written in boxes of 32 x 32 from a
-// 128-byte-swizzled shared tile.
-int make_out_tmap(CUtensorMap *map, void *base, CUtensorMapDataType dtype, int64_t M, int64_t N)
-{
-    EncodeTiledFn fn = get_encode_fn();
-    if (!fn) return DSQ_ERR_CUDA;
-    cuuint64_t dims[2] = {(cuuint64_t)N, (cuuint64_t)M};
-    cuuint64_t strides[1] = {(cuuint64_t)N * 4};
-    cuuint32_t box[2] = {32, 32};
-    cuuint32_t estr[2] = {1, 1};
-    const CUresult r = fn(map, dtype, 2, base, dims, strides, box, estr,
-                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                          CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return r == CUDA_SUCCESS ? DSQ_OK : DSQ_ERR_CUDA;
-}
-
 // Resident B: one N tile and few K steps, so the expanded B tile of every K
 // step fits in shared memory next to the rings; it is then expanded once per
 // CTA instead of once per M tile.
-struct PipeInfo { int ks, su, a_slots, a_col0, s_p, wide, pair, whole_k, ksa; };
+struct PipeInfo { int ks, su, a_slots, a_col0, s_p, wide, pair, whole_k; };
 PipeInfo pipe_info(int pm)
 {
     switch (pm) {
-    case 6: return {Pipe<6>::KS, Pipe<6>::SU, Pipe<6>::GROUPS * Pipe<6>::A_RING / 2, Pipe<6>::A_COL0, Pipe<6>::S_P, 0, 1, 0, Pipe<6>::KSA};
     case 5: return {Pipe<5>::KS, Pipe<5>::SU, Pipe<5>::GROUPS * Pipe<5>::A_RING, Pipe<5>::A_COL0, Pipe<5>::S_P, 0, 0, 1};
     case 4: return {Pipe<4>::KS, Pipe<4>::SU, Pipe<4>::GROUPS * Pipe<4>::A_RING, Pipe<4>::A_COL0, Pipe<4>::S_P, 0, 1};
     case 1: return {Pipe<1>::KS, Pipe<1>::SU, Pipe<1>::GROUPS * Pipe<1>::A_RING, Pipe<1>::A_COL0, Pipe<1>::S_P, 0};
@@ -1447,7 +1431,7 @@ void choose_b_mode(TcParams *p, int bits, int pm)
     p->b_res = 0;
     p->b_stages = pi.su;
     p->epw = pi.wide ? 2 : 1;
-    if (!pi.wide && !pi.pair && p->n_tiles == 1 && p->rounds <= MAX_B_STAGES && p->m_tiles > 148) {
+    if (!pi.wide && !pi.pair && p->n_tiles == 1 && p->rounds <= MAX_B_STAGES && p->m_tiles > dsq_sm_count()) {
         const SmemLayout L = smem_layout(p->BN, bits, p->s_p, p->rounds, pi.ks, pi.a_slots,
                                          epi_slots(1, 3));
         if (L.total + 1024 <= 227u * 1024u) {
@@ -1577,12 +1561,19 @@ int setup_a_tma(TcParams *p, CUtensorMap *map, const void *A, int64_t rows, int 
     return DSQ_OK;
 }
 
-int g_forced_bn = 0;   // dsq_set_tile_n
-int g_pdl = 1;         // dsq_set_dependent_launch
+// process-wide hooks (csrc/dsq_hooks.h)
+std::atomic<int> g_forced_bn{0};      // dsq_set_tile_n
+std::atomic<int> g_pdl{1};            // dsq_set_dependent_launch
+std::atomic<int> g_forced_ks{0};      // dsq_set_round_k_steps: 0 automatic, 1 single K steps, 2 double
+std::atomic<int> g_pair_mode{0};      // dsq_set_cta_pairs: 0 automatic, 1 never, 2 wherever possible
+std::atomic<unsigned long long> g_wait_ns{WAIT_LIMIT_NS};   // dsq_set_wait_limit_ns
+std::atomic<int> g_skip_b_round{-1};  // dsq_set_test_skip_b_round
 
 int pick_bn(int m_tiles, int ncols, int bits)
 {
-    if (g_forced_bn) return (bits == 2 && g_forced_bn < 64) ? 64 : g_forced_bn;
+    const int forced = g_forced_bn.load();
+    if (forced) return (bits == 2 && forced < 64) ? 64 : forced;
+    const int sms = dsq_sm_count() > 0 ? dsq_sm_count() : 148;
     const int cands[5] = {256, 192, 128, 64, 32};
     int best = 0;
     double best_cost = 1e30;
@@ -1591,7 +1582,7 @@ int pick_bn(int m_tiles, int ncols, int bits)
         if (bits == 2 && bn < 64) continue;
         const int n_tiles = (ncols + bn - 1) / bn;
         const int64_t tiles = (int64_t)m_tiles * n_tiles;
-        const int64_t waves = (tiles + 147) / 148;
+        const int64_t waves = (tiles + sms - 1) / sms;
         const double cost = (double)waves * (100.0 + bn);
         if (cost < best_cost) { best_cost = cost; best = bn; }
     }
@@ -1605,26 +1596,35 @@ int launch_tc(const TcMaps &tmap, const TcParams &p, cudaStream_t s)
     constexpr bool PAIR = Pipe<PM>::PAIR;
     const SmemLayout L = smem_layout(PAIR ? p.BN / 2 : p.BN, BITS, p.s_p, p.b_stages,
                                      Pipe<PM>::KS,
-                                     Pipe<PM>::GROUPS * Pipe<PM>::A_RING / Pipe<PM>::HALVES,
-                                     epi_slots(p.join, p.epw, p.stage));
+                                     Pipe<PM>::GROUPS * Pipe<PM>::A_RING,
+                                     epi_slots(p.join, p.epw));
     if (L.total > 227u * 1024u) return DSQ_ERR_UNSUPPORTED;
     int smem_bytes = (int)L.total + 1024;            // slack for the 1024-byte alignment
     if (smem_bytes > 227 * 1024) smem_bytes = 227 * 1024;
-    static bool configured = false;
-    if (!configured) {
+    // The opt-in to large dynamic shared memory is a per-device attribute of
+    // the function: one bit per device ordinal for this instantiation.
+    static std::atomic<unsigned long long> configured{0ull};
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0) return DSQ_ERR_CUDA;
+    const unsigned long long dev_bit = dev < 64 ? 1ull << dev : 0ull;
+    if (!(configured.load(std::memory_order_acquire) & dev_bit)) {
         if (cudaFuncSetAttribute(dsq_tc_kernel<BITS, A_SIGNED, EPI, PM, A_TMA>,
                                  cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  227 * 1024) != cudaSuccess)
             return DSQ_ERR_CUDA;
-        configured = true;
+        configured.fetch_or(dev_bit, std::memory_order_release);
     }
+    const int sms = dsq_sm_count();
+    if (sms <= 0) return DSQ_ERR_CUDA;
     int grid = p.m_tiles * p.n_tiles;
-    if (grid > 148) grid = 148;
+    if (grid > sms) grid = sms;
     if (p.BN * p.n_acc > Pipe<PM>::A_COL0) return DSQ_ERR_UNSUPPORTED;
     TcParams q = p;
     q.smem_bytes = smem_bytes;
+    q.wait_ns = g_wait_ns.load();
+    q.skip_b_round = g_skip_b_round.load();
     // one cluster of two CTAs (the two SMs of a TPC) per tile in flight
-    if (PAIR && grid > 74) grid = 74;
+    if (PAIR && grid > sms / 2) grid = sms / 2;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(PAIR ? 2 * grid : grid);
     cfg.blockDim = dim3(NUM_THREADS);
@@ -1639,7 +1639,7 @@ int launch_tc(const TcMaps &tmap, const TcParams &p, cudaStream_t s)
         attr[na].val.clusterDim.z = 1;
         ++na;
     }
-    if (g_pdl) {
+    if (g_pdl.load()) {
         // the kernel waits for its predecessors itself (griddepcontrol.wait)
         attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
         attr[na].val.programmaticStreamSerializationAllowed = 1;
@@ -1648,7 +1648,7 @@ int launch_tc(const TcMaps &tmap, const TcParams &p, cudaStream_t s)
     cfg.attrs = attr;
     cfg.numAttrs = na;
     if (cudaLaunchKernelEx(&cfg, dsq_tc_kernel<BITS, A_SIGNED, EPI, PM, A_TMA>, tmap.b, tmap.a,
-                           tmap.c, tmap.d, q) != cudaSuccess) {
+                           q) != cudaSuccess) {
         cudaGetLastError();
         return DSQ_ERR_CUDA;
     }
@@ -1677,7 +1677,6 @@ int launch_bits(int epi, int pm, const TcMaps &tmap, const TcParams &p, cudaStre
 {
     if (epi == EPI_GEMM) {
         // 2- and 4-bit GEMMs always fetch A with TMA
-        if (pm == 6) return launch_tc<BITS, true, EPI_GEMM, 6, 1>(tmap, p, s);
         if (pm == 4) return launch_tc<BITS, true, EPI_GEMM, 4, 1>(tmap, p, s);
         if (pm == 3) return launch_tc<BITS, true, EPI_GEMM, 3, 1>(tmap, p, s);
         if (pm == 2) return launch_tc<BITS, true, EPI_GEMM, 2, 1>(tmap, p, s);
@@ -1712,31 +1711,20 @@ int dispatch_tc(int bits, int epi, int pm, const TcMaps &tmap, const TcParams &p
     return DSQ_ERR_UNSUPPORTED;
 }
 
-// Pipeline mode for a problem (see Pipe<PM>); g_forced_ks: 0 automatic, 1 forces
-// single K steps, 2 forces double steps wherever they are possible.
-int g_forced_ks = 0;
-int g_pair_mode = 0;    // dsq_set_cta_pairs: 0 automatic, 1 never, 2 wherever possible
-int g_stage_mode = 1;   // dsq_set_gemm_store: 1 direct stores (default), 0 staged TMA stores where possible
-// Whether a GEMM runs its CTA pairs on 256 x 128 tiles with overlapped epilogues
-// (PM 6) rather than on 256 x 256 tiles (PM 4).
-bool pair128_pays(int64_t M, int64_t N)
-{
-    (void)M; (void)N;
-    return false;
-}
-
+// Pipeline mode for a problem (see Pipe<PM>).
 int pick_pm(const TcParams &p, int bits, bool im2col)
 {
-    if (bits == 3 || p.ksteps < 2 || g_forced_ks == 1) return 1;
+    const int forced_ks = g_forced_ks.load();
+    if (bits == 3 || p.ksteps < 2 || forced_ks == 1) return 1;
     // whole-K rounds: a small convolution whose B tile can stay resident
-    if (im2col && g_forced_ks == 0 && p.ksteps >= 3 && p.ksteps <= Pipe<5>::KS &&
+    if (im2col && forced_ks == 0 && p.ksteps >= 3 && p.ksteps <= Pipe<5>::KS &&
         2 * p.BN <= Pipe<5>::A_COL0) {
         TcParams q = p;
         choose_b_mode(&q, bits, 5);
         if (q.rounds == 1 && q.b_res) return 5;
     }
     // CTA pairs: 256-wide N tiles and at least two 128-row tiles to put together
-    if (p.BN == 256 && p.M > BM && g_pair_mode != 1) return 4;
+    if (p.BN == 256 && p.M > BM && g_pair_mode.load() != 1) return 4;
     if (p.BN > 128) return p.ksteps >= 4 ? 3 : 1;
     // two K steps per round: a round costs about the same whatever it carries
     // (measured faster than single steps even where those would keep the
@@ -1757,7 +1745,7 @@ int dsq_set_round_k_steps(int ks)
 
 int dsq_set_cta_pairs(int mode)
 {
-    if (mode < 0 || mode > 3) return DSQ_ERR_SHAPE;
+    if (mode < 0 || mode > 2) return DSQ_ERR_SHAPE;
     g_pair_mode = mode;
     return DSQ_OK;
 }
@@ -1769,10 +1757,16 @@ int dsq_set_dependent_launch(int on)
     return DSQ_OK;
 }
 
-int dsq_set_gemm_store(int mode)
+int dsq_set_test_skip_b_round(int round)
 {
-    if (mode != 0 && mode != 1) return DSQ_ERR_SHAPE;
-    g_stage_mode = mode;
+    g_skip_b_round = round < 0 ? -1 : round;
+    return DSQ_OK;
+}
+
+int dsq_set_wait_limit_ns(long long ns)
+{
+    if (ns < 0) return DSQ_ERR_SHAPE;
+    g_wait_ns = ns == 0 ? WAIT_LIMIT_NS : (unsigned long long)ns;
     return DSQ_OK;
 }
 
@@ -1784,20 +1778,32 @@ int dsq_set_tile_n(int bn)
     return DSQ_OK;
 }
 
-int dsq_gemm(const void *A_codes, const void *B_codes, int64_t M, int64_t N, int64_t K,
-             int bits, int32_t *C_i32, const float *row_scale, float *D_f32, void *workspace,
-             size_t ws_bytes, void *stream)
+// Argument checks of dsq_gemm (everything that can be seen from the host).
+static int gemm_check_args(const void *A_codes, const void *B_codes, int64_t M, int64_t N,
+                           int64_t K, int bits, const int32_t *C_i32, const float *row_scale,
+                           const float *D_f32)
 {
-    if (!A_codes || !B_codes || !workspace) return DSQ_ERR_NULL;
+    if (!A_codes || !B_codes) return DSQ_ERR_NULL;
     if (!C_i32 && !D_f32) return DSQ_ERR_NULL;
     if (D_f32 && !row_scale) return DSQ_ERR_NULL;
     if (bits < 2 || bits > 4) return DSQ_ERR_BITS;
     if (M <= 0 || N <= 0 || K <= 0 || M > (1 << 24) || N > (1 << 24) || K > (1 << 24))
         return DSQ_ERR_SHAPE;
     if ((double)K * 128.0 * (double)((1 << bits) - 1) > 2147483647.0) return DSQ_ERR_OVERFLOW;
-    if (!dsq_aligned16(A_codes) || !dsq_aligned16(B_codes) || !dsq_aligned16(workspace) ||
+    if (!dsq_aligned16(A_codes) || !dsq_aligned16(B_codes) ||
         (C_i32 && !dsq_aligned16(C_i32)) || (D_f32 && !dsq_aligned16(D_f32)))
         return DSQ_ERR_ALIGN;
+    return DSQ_OK;
+}
+
+int dsq_gemm(const void *A_codes, const void *B_codes, int64_t M, int64_t N, int64_t K,
+             int bits, int32_t *C_i32, const float *row_scale, float *D_f32, void *workspace,
+             size_t ws_bytes, void *stream)
+{
+    if (!workspace) return DSQ_ERR_NULL;
+    int st = gemm_check_args(A_codes, B_codes, M, N, K, bits, C_i32, row_scale, D_f32);
+    if (st) return st;
+    if (!dsq_aligned16(workspace)) return DSQ_ERR_ALIGN;
     if (ws_bytes < DSQ_WS_BYTES) return DSQ_ERR_SIZE;
 
     const size_t pitch = dsq_row_pitch(K, bits);
@@ -1809,16 +1815,8 @@ int dsq_gemm(const void *A_codes, const void *B_codes, int64_t M, int64_t N, int
     p.BN = pick_bn(p.m_tiles, (int)N, bits);
     if (bits == 2 && p.BN < 64) p.BN = 64;
     p.n_tiles = (int)((N + p.BN - 1) / p.BN);
-    int pm = pick_pm(p, bits, false);
-    // pairs on 256 x 128 tiles with two accumulator buffers (see Pipe<6>)
-    if (bits != 3 && g_forced_bn == 0 && g_forced_ks == 0 && M > BM && N > 64 && p.ksteps >= 8 &&
-        (g_pair_mode == 3 || (g_pair_mode == 0 && pm == 4 && pair128_pays(M, N)))) {
-        pm = 6;
-        p.BN = 128;
-        p.n_tiles = (int)((N + p.BN - 1) / p.BN);
-    }
+    const int pm = pick_pm(p, bits, false);
     const int ks = pipe_info(pm).ks;
-    const int ksa = pipe_info(pm).ksa ? pipe_info(pm).ksa : ks;
     const bool pair = pipe_info(pm).pair != 0;
     if (pair) p.m_tiles = (int)((M + 2 * BM - 1) / (2 * BM));
     choose_b_mode(&p, bits, pm);
@@ -1834,33 +1832,12 @@ int dsq_gemm(const void *A_codes, const void *B_codes, int64_t M, int64_t N, int
     p.D_f32 = D_f32;
     p.ws = (int *)workspace;
     TcMaps tmap;
-    int st = make_rows_tmap(&tmap.b, B_codes, pitch, (uint64_t)N, pitch, ks * 16 * bits,
-                            pair ? p.BN / 2 : p.BN);
+    st = make_rows_tmap(&tmap.b, B_codes, pitch, (uint64_t)N, pitch, ks * 16 * bits,
+                        pair ? p.BN / 2 : p.BN);
     if (st) return st;
     tmap.a = tmap.b;
-    st = setup_a_tma(&p, &tmap.a, A_codes, M, bits, ksa, true, nullptr, 1, false);
+    st = setup_a_tma(&p, &tmap.a, A_codes, M, bits, ks, true, nullptr, 1, false);
     if (st) return st;
-    tmap.c = tmap.b;
-    tmap.d = tmap.b;
-    // outputs through TMA stores when their rows are 16-byte multiples and the
-    // staging tiles fit in shared memory
-    if (g_stage_mode != 1 && N % 4 == 0) {
-        const PipeInfo pi = pipe_info(pm);
-        const SmemLayout Ls = smem_layout(pi.pair ? p.BN / 2 : p.BN, bits, p.s_p, p.b_stages, pi.ks,
-                                          pi.a_slots, epi_slots(0, p.epw, 1));
-        if (Ls.total + 1024 <= 227u * 1024u) {
-            p.stage = 1;
-            p.join = 0;
-            if (C_i32) {
-                st = make_out_tmap(&tmap.c, C_i32, CU_TENSOR_MAP_DATA_TYPE_INT32, M, N);
-                if (st) return st;
-            }
-            if (D_f32) {
-                st = make_out_tmap(&tmap.d, D_f32, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, M, N);
-                if (st) return st;
-            }
-        }
-    }
     return dispatch_tc(bits, EPI_GEMM, pm, tmap, p, (cudaStream_t)stream);
 }
 
@@ -1977,21 +1954,26 @@ int dsq_gemm_static_ws(const void *A_codes, const void *B_codes, int64_t M, int6
                        float *D_f32, int wait_and_check, void *stream)
 {
     static_assert(DSQ_STATIC_WS_BYTES >= DSQ_WS_BYTES, "static workspace too small");
+    // everything that can fail on the host fails here, before the symbol
+    // lookup and before anything is enqueued on the caller's stream
+    const int bad = gemm_check_args(A_codes, B_codes, M, N, K, bits, C_i32, row_scale, D_f32);
+    if (bad) return bad;
     if (M > DSQ_STATIC_WS_MAX_DIM || N > DSQ_STATIC_WS_MAX_DIM || K > DSQ_STATIC_WS_MAX_DIM)
         return DSQ_ERR_SIZE;
     // In host code `g_static_ws` is only a handle for the symbol, not a device
     // address.  The address on the current device is looked up once per device
     // (no allocation happens: the array is part of the loaded module).
-    static void *dev_ptr[64] = {};
+    static std::atomic<void *> dev_ptr[DSQ_MAX_DEVICES];
     int dev = -1;
     DSQ_CUDA_TRY(cudaGetDevice(&dev));
-    if (dev < 0 || dev >= 64) return DSQ_ERR_UNSUPPORTED;
-    if (!dev_ptr[dev]) {
+    if (dev < 0 || dev >= DSQ_MAX_DEVICES) return DSQ_ERR_UNSUPPORTED;
+    void *ws = dev_ptr[dev].load(std::memory_order_acquire);
+    if (!ws) {
         void *ptr = nullptr;
         if (cudaGetSymbolAddress(&ptr, g_static_ws) != cudaSuccess || !ptr) return DSQ_ERR_CUDA;
-        dev_ptr[dev] = ptr;
+        dev_ptr[dev].store(ptr, std::memory_order_release);
+        ws = ptr;
     }
-    void *ws = dev_ptr[dev];
     cudaStream_t s = (cudaStream_t)stream;
     // the array keeps what the previous call left: the status words start at 0
     DSQ_CUDA_TRY(cudaMemsetAsync(ws, 0, DSQ_STATIC_WS_BYTES, s));

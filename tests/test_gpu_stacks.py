@@ -146,3 +146,42 @@ def test_resnet18_full_batch_sampled_images(dsq):
     torch.cuda.synchronize()
     assert torch.equal(out1, g.codes[st.out])
     g.check()
+
+
+def _unpack_image(dsq, g, name, img):
+    H, W, Cc = g.shapes[name]
+    packed = g.codes[name][img:img + 1].reshape(H * W, -1).contiguous()
+    return N(dsq.dsq_unpack(packed, H * W, Cc, g.bits, False)).reshape(1, H, W, Cc)
+
+
+def _full_batch_sampled(dsq, st, wid, images):
+    """One forward pass at the batch and image size the benchmark times; the
+    oracle recomputes single images alone (images are independent) and every
+    code tensor of every layer must match for them."""
+    from paper_1908_05033_b200.stack import GpuStack
+    x = dsq_inputs.stack_input(st, workload_id=wid)
+    params = dsq_inputs.stack_params(st, workload_id=wid)
+    g = GpuStack(st, params)
+    assert g.batch == st.batch
+    g.forward(T(x))
+    g.check()
+    names = list(st.tensor_shapes())
+    for img in images:
+        ref = ostack.run_stack(st, x[img:img + 1], params, keep=names)
+        for name in names:
+            assert np.array_equal(_unpack_image(dsq, g, name, img), ref[name]), (img, name)
+    return g
+
+
+def test_mobilenetv2_full_batch_sampled_images(dsq):
+    """MobileNetV2-shaped stack at batch 64 on 112x112x32, as timed."""
+    st = dsq_inputs.mobilenetv2_stack()
+    assert st.batch == 64 and st.in_shape == (112, 112, 32)
+    _full_batch_sampled(dsq, st, 4, (0, 37, 63))
+
+
+def test_vgg16_full_size_sampled_images(dsq):
+    """VGG-16-shaped 2-bit stack at batch 32 on 224x224x64, as timed."""
+    st = dsq_inputs.vgg16_stack()
+    assert st.batch == 32 and st.in_shape == (224, 224, 64)
+    _full_batch_sampled(dsq, st, 5, (0, 21))

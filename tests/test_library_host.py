@@ -14,8 +14,8 @@ from paper_1908_05033_b200 import binding as B
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
-def declared_functions():
-    text = open(os.path.join(ROOT, "include", "dsq.h")).read()
+def declared_functions(path=("include", "dsq.h")):
+    text = open(os.path.join(ROOT, *path)).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
     return sorted(set(re.findall(r"\b(dsq_[a-z0-9_]+)\s*\(", text)))
 
@@ -28,6 +28,11 @@ def test_every_declared_symbol_is_exported_and_bound():
     for n in names:
         assert hasattr(dsq.lib, n), n
     assert set(names) == set(B.EXPORTED_SYMBOLS)
+    # the tuning / test hooks live in an internal header, not in include/dsq.h
+    hooks = declared_functions(("paper_1908_05033_b200", "csrc", "dsq_hooks.h"))
+    assert set(hooks) == set(B.HOOK_SYMBOLS) and not set(hooks) & set(names)
+    for n in hooks:
+        assert hasattr(dsq.lib, n), n
 
 
 def test_size_queries():
@@ -77,6 +82,12 @@ def test_validation_status_codes_without_a_gpu():
     assert lib.dsq_gemm(fake, fake, 128, 128, 128, 4, fake, None, fake, fake, 256, None) == -1
     # K so large that 2^7 * (2^b - 1) * K overflows int32
     assert lib.dsq_gemm(fake, fake, 128, 128, 1 << 21, 4, fake, None, None, fake, 256, None) == -7
+    # the no-workspace variant rejects bad arguments before it looks up its
+    # scratch or enqueues anything (so this works without a GPU)
+    assert lib.dsq_gemm_static_ws(None, fake, 128, 128, 128, 4, fake, None, None, 1, None) == -1
+    assert lib.dsq_gemm_static_ws(fake, fake, 128, 128, 128, 5, fake, None, None, 1, None) == -3
+    assert lib.dsq_gemm_static_ws(fake, fake, 128, 128, 128, 4, odd, None, None, 1, None) == -2
+    assert lib.dsq_gemm_static_ws(fake, fake, 65537, 16, 16, 4, fake, None, None, 1, None) == -5
 
     # conv: unsupported geometry, lo != 0 with padding, 3-bit, bad w_offset
     scale = C.c_void_p(0x2000)

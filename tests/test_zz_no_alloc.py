@@ -14,6 +14,7 @@ import torch
 
 pytestmark = pytest.mark.gpu
 
+from oracle import native
 import dsq_inputs
 from gpu_util import T, N
 
@@ -43,8 +44,30 @@ def test_static_workspace_gemm_matches_dsq_gemm_twice_in_a_row():
         # the tolerance the GEMM parity tests use
         assert torch.equal(C_out, C_ref)
         assert torch.equal(D_out, D_ref)
+        # ... and the oracle's (the same sizes are among the GEMM parity cases)
+        C_cpu = native.gemm(A, B)
+        assert np.array_equal(N(C_out), C_cpu)
+        assert np.array_equal(N(D_out), native.gemm_dequant(C_cpu, rs))
+        # enqueue-only form: returns at once, the caller synchronises
+        C_out.fill_(-1)
+        st = lib.dsq_gemm_static_ws(
+            C.c_void_p(Ap.data_ptr()), C.c_void_p(Bp.data_ptr()), M, Nn, K, bits,
+            C.c_void_p(C_out.data_ptr()), None, None, 0, stream)
+        assert st == 0
+        torch.cuda.synchronize()
+        assert torch.equal(C_out, C_ref)
     # the documented limit is enforced before anything is launched
     st = lib.dsq_gemm_static_ws(C.c_void_p(Ap.data_ptr()), C.c_void_p(Bp.data_ptr()),
                                 65537, 16, 16, 4, C.c_void_p(C_out.data_ptr()), None, None,
                                 1, stream)
     assert st == -5
+    # a rejected call leaves the stream and the outputs untouched
+    C_out.fill_(7)
+    st = lib.dsq_gemm_static_ws(None, C.c_void_p(Bp.data_ptr()), M, Nn, K, bits,
+                                C.c_void_p(C_out.data_ptr()), None, None, 1, stream)
+    assert st == -1
+    st = lib.dsq_gemm_static_ws(C.c_void_p(Ap.data_ptr()), C.c_void_p(Bp.data_ptr()), M, Nn, K,
+                                5, C.c_void_p(C_out.data_ptr()), None, None, 1, stream)
+    assert st == -3
+    torch.cuda.synchronize()
+    assert bool((C_out == 7).all())
