@@ -64,9 +64,11 @@ class GpuStack:
         self.debug = {}
 
     def forward(self, x):
-        """x: fp32 NHWC CUDA tensor.  Returns the packed codes of st.out."""
+        """x: fp32 NHWC CUDA tensor, or None to run the layers on the input
+        codes already in place.  Returns the packed codes of st.out."""
         st, bits = self.st, self.bits
-        B.dsq_quantize_act(x, bits, st.in_lo, st.in_hi, out=self.codes["in"])
+        if x is not None:
+            B.dsq_quantize_act(x, bits, st.in_lo, st.in_hi, out=self.codes["in"])
         for L, w in self.layers:
             H, W, Cc = self.shapes[L.src]
             shape = (self.batch, H, W, Cc)
