@@ -85,6 +85,7 @@ _HOOKS = {
     "dsq_set_dependent_launch": (_int, [_int]),
     "dsq_set_wait_limit_ns": (_int, [C.c_longlong]),
     "dsq_set_test_skip_b_round": (_int, [_int]),
+    "dsq_set_conv3_window": (_int, [_int]),
 }
 for _name, (_res, _args) in list(_SIGNATURES.items()) + list(_HOOKS.items()):
     _f = getattr(lib, _name)       # AttributeError if a symbol is missing
@@ -342,6 +343,10 @@ def dsq_set_wait_limit_ns(ns):
 def dsq_set_test_skip_b_round(r):
     """Test hook: the B producer leaves out round r (-1 = off)."""
     _check(lib.dsq_set_test_skip_b_round(int(r)), "dsq_set_test_skip_b_round")
+
+
+def dsq_set_conv3_window(mode):
+    _check(lib.dsq_set_conv3_window(int(mode)), "dsq_set_conv3_window")
 
 
 def dsq_set_dependent_launch(on):

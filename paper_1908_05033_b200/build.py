@@ -7,12 +7,13 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libdsq_b200.so")
-SOURCES = ["dsq_elementwise.cu", "dsq_dwconv.cu", "dsq_tc.cu"]
-HEADERS = ["dsq_common.cuh", "dsq_epilogue.cuh", "dsq_ptx.cuh",
+SOURCES = ["dsq_elementwise.cu", "dsq_dwconv.cu", "dsq_tc.cu", "dsq_conv3.cu"]
+HEADERS = ["dsq_common.cuh", "dsq_epilogue.cuh", "dsq_ptx.cuh", "dsq_tc_common.cuh",
+           "dsq_tc_host.h", "dsq_hooks.h",
            os.path.join("..", "..", "include", "dsq.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo",
               "-std=c++17", "--expt-relaxed-constexpr", "-Xcompiler", "-fPIC",
-              "-Xcompiler", "-fvisibility=default", "--fmad=false"]
+              "-Xcompiler", "-fvisibility=default", "--fmad=false", "--threads", "0"]
 
 
 def _stale() -> bool:

@@ -55,6 +55,9 @@ def main(argv=None):
     ap.add_argument("--tile-n", type=int, default=0)
     ap.add_argument("--round-k", type=int, default=0)
     ap.add_argument("--pairs", type=int, default=0, help="0 auto, 1 never, 2 wherever possible")
+    ap.add_argument("--window", type=int, default=1,
+                    help="3x3 stride-1 convolutions: 1 shared-memory window kernel, 0 im2col kernel")
+    ap.add_argument("--residual", action="store_true")
     a = ap.parse_args(argv)
     dev = "cuda"
     ws = B.new_workspace(dev)
@@ -65,6 +68,7 @@ def main(argv=None):
     B.dsq_set_tile_n(a.tile_n)
     B.dsq_set_round_k_steps(a.round_k)
     B.dsq_set_cta_pairs(a.pairs)
+    B.dsq_set_conv3_window(a.window)
     out = {"case": a.case, "bits": bits, "tile_n": a.tile_n}
     if a.case == "gemm":
         n = a.size
@@ -88,9 +92,12 @@ def main(argv=None):
         ho = (a.hw + 2 * (a.ksize // 2) - a.ksize) // a.stride + 1
         codes = torch.empty((a.batch, ho, ho, B.dsq_row_pitch(a.cout, bits)),
                             dtype=torch.uint8, device=dev)
+        res = torch.randint(0, 256, codes.shape, dtype=torch.uint8, device=dev,
+                            generator=gen) if a.residual else None
         fn = lambda: B.dsq_conv2d(act, shape, (bits, 0.0, 2.0), blob, conv, scale, bias, ws,
                                   w_offset=0.5, requant=(bits, 0.0, 2.0), out_codes=codes,
-                                  want_f32=a.f32_out)
+                                  want_f32=a.f32_out, residual=res,
+                                  residual_q=(bits, 0.0, 2.0) if a.residual else None)
         ms, all_ms = _timeit(fn, a.iters, flush)
         macs = a.batch * ho * ho * a.cout * a.ksize * a.ksize * a.cin
         out.update(shape=list(shape), cout=a.cout, ksize=a.ksize, stride=a.stride, ms=ms,

@@ -33,6 +33,14 @@ int dsq_set_dependent_launch(int on);
  * restores the default). */
 int dsq_set_wait_limit_ns(long long ns);
 
+/* 3x3 stride-1 convolutions on an expanded shared-memory window
+ * (dsq_conv3.cu): 1 = where it is the faster kernel (default), 0 = never (the
+ * im2col kernel takes them), 3 = wherever the geometry allows, 2 = as 3 with
+ * the row phase of the window written into the A descriptor's base-offset
+ * field (a probe of that field's meaning: the tensor core swizzles by
+ * absolute shared-memory address, so this gives wrong numbers). */
+int dsq_set_conv3_window(int mode);
+
 /* Test hook: in every later launch the thread that issues the TMA copies of
  * the packed B operand leaves out the copy of round `round` of its CTA
  * (0 = the first) and issues nothing after it; -1 switches the hook off.

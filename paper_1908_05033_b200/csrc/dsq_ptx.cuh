@@ -155,6 +155,12 @@ __device__ __forceinline__ uint4 lds_128(uint32_t addr)
                  : "memory");
     return v;
 }
+__device__ __forceinline__ void sts_128(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d)
+{
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c),
+                 "r"(d)
+                 : "memory");
+}
 // 256-bit global store (one full 32-byte sector per lane); dst 32-byte aligned
 __device__ __forceinline__ void stg_256(void *dst, uint32_t a, uint32_t b, uint32_t c, uint32_t d,
                                         uint32_t e, uint32_t f, uint32_t g, uint32_t h)
@@ -162,6 +168,13 @@ __device__ __forceinline__ void stg_256(void *dst, uint32_t a, uint32_t b, uint3
     asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst), "r"(a),
                  "r"(b), "r"(c), "r"(d), "r"(e), "r"(f), "r"(g), "r"(h)
                  : "memory");
+}
+
+// Barrier among `nthreads` threads (a multiple of 32) of the CTA on hardware
+// barrier `id` (1..15; 0 is __syncthreads).
+__device__ __forceinline__ void named_barrier_sync(int id, int nthreads)
+{
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
 }
 
 // ---- proxy / tcgen05 fences ------------------------------------------------
@@ -350,6 +363,55 @@ __device__ __forceinline__ void mma_i8_ts_x4(uint32_t d_tmem, uint32_t a_tmem, u
 }
 #undef DSQ_MMA_X4_BODY
 
+// One tcgen05.mma kind::i8 with BOTH operands read through shared-memory
+// descriptors (given as their two 32-bit halves), issued by one elected lane
+// of a converged warp; all lanes call with warp-uniform arguments.
+__device__ __forceinline__ void mma_i8_ss_elect(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi,
+                                                uint32_t b_lo, uint32_t b_hi, uint32_t idesc,
+                                                uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p, pe;\n\t.reg .b64 da, db;\n\t"
+        "setp.ne.b32 p, %6, 0;\n\t"
+        "mov.b64 da, {%1, %2};\n\tmov.b64 db, {%3, %4};\n\t"
+        "elect.sync _|pe, 0xffffffff;\n\t"
+        "@pe tcgen05.mma.cta_group::1.kind::i8 [%0], da, db, %5, p;\n\t}" ::"r"(d_tmem),
+        "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
+// Four such instructions in one block (one K step of 128 bytes): the B
+// descriptor advances 32 bytes (2 units of 16 bytes in its low word) per
+// instruction, the low words of the four A descriptors are given one by one
+// (0xFFFFFFFF = leave this instruction out); the first instruction takes the
+// caller's accumulate flag, the others accumulate.  a_lo0 must be valid.
+__device__ __forceinline__ void mma_i8_ss_x4_elect(uint32_t d_tmem, uint32_t a_lo0, uint32_t a_lo1,
+                                                   uint32_t a_lo2, uint32_t a_lo3, uint32_t a_hi,
+                                                   uint32_t b_lo, uint32_t b_hi, uint32_t idesc,
+                                                   uint32_t accumulate_first)
+{
+    asm volatile(
+        "{\n\t.reg .pred p0, p1, pe, v1, v2, v3;\n\t"
+        ".reg .b64 da0, da1, da2, da3, db0, db1, db2, db3;\n\t.reg .b32 l1, l2, l3;\n\t"
+        "setp.ne.b32 p0, %9, 0;\n\tsetp.eq.b32 p1, %9, %9;\n\t"
+        "add.u32 l1, %6, 2;\n\tadd.u32 l2, %6, 4;\n\tadd.u32 l3, %6, 6;\n\t"
+        "mov.b64 da0, {%1, %5};\n\tmov.b64 da1, {%2, %5};\n\t"
+        "mov.b64 da2, {%3, %5};\n\tmov.b64 da3, {%4, %5};\n\t"
+        "mov.b64 db0, {%6, %7};\n\tmov.b64 db1, {l1, %7};\n\t"
+        "mov.b64 db2, {l2, %7};\n\tmov.b64 db3, {l3, %7};\n\t"
+        "elect.sync _|pe, 0xffffffff;\n\t"
+        "setp.ne.b32 v1, %2, 0xFFFFFFFF;\n\tsetp.ne.b32 v2, %3, 0xFFFFFFFF;\n\t"
+        "setp.ne.b32 v3, %4, 0xFFFFFFFF;\n\t"
+        "and.pred v1, v1, pe;\n\tand.pred v2, v2, pe;\n\tand.pred v3, v3, pe;\n\t"
+        "@pe tcgen05.mma.cta_group::1.kind::i8 [%0], da0, db0, %8, p0;\n\t"
+        "@v1 tcgen05.mma.cta_group::1.kind::i8 [%0], da1, db1, %8, p1;\n\t"
+        "@v2 tcgen05.mma.cta_group::1.kind::i8 [%0], da2, db2, %8, p1;\n\t"
+        "@v3 tcgen05.mma.cta_group::1.kind::i8 [%0], da3, db3, %8, p1;\n\t}" ::"r"(d_tmem),
+        "r"(a_lo0), "r"(a_lo1), "r"(a_lo2), "r"(a_lo3), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc),
+        "r"(accumulate_first)
+        : "memory");
+}
+
 // tcgen05.commit by one elected lane of a converged warp (all lanes call).
 __device__ __forceinline__ void mma_commit_elect(uint32_t bar)
 {
@@ -415,6 +477,18 @@ __device__ __forceinline__ void tmem_ld_32x32(uint32_t taddr, uint32_t (&r)[32])
           "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
           "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]),
           "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+// 32 lanes x 16 columns.
+__device__ __forceinline__ void tmem_ld_32x16(uint32_t taddr, uint32_t (&r)[16])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]),
+          "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]),
+          "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
         : "r"(taddr)
         : "memory");
 }

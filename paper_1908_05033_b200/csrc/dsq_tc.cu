@@ -47,11 +47,8 @@
 // is released and the kernel returns.
 #include <cuda.h>
 
-#include "dsq_epilogue.cuh"
-#include "dsq_hooks.h"
-#include "dsq_ptx.cuh"
-
-using namespace dsq_ptx;
+#include "dsq_tc_common.cuh"
+#include "dsq_tc_host.h"
 
 // Scratch of dsq_gemm_static_ws: the workspace (status word, failure detail)
 // that dsq_gemm normally receives from its caller, held by the library
@@ -120,9 +117,6 @@ static_assert(WARP_A0 + NUM_A_WARPS == WARP_B0 && WARP_B0 + NUM_B_WARPS == WARP_
                   WARP_E0 + NUM_E_WARPS == WARP_TMA_A && WARP_TMA_A + 1 == NUM_WARPS,
               "warp roles");
 constexpr int NUM_THREADS = NUM_WARPS * 32;
-constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;   // default: a wait gives up after 2 s
-// once a CTA has given up, copies and MMAs already in flight get this long to land
-constexpr unsigned long long DRAIN_LIMIT_NS = 20000000ull;
 
 enum { MODE_CONV = 0, MODE_GEMM = 1 };
 // epilogue variants (template parameter): GEMM; convolution writing codes
@@ -179,144 +173,6 @@ struct TcParams {
     uint32_t orv;                     // OR-ed into every signed byte
     int *ws;
 };
-
-// ---------------------------------------------------------------------------
-// bounded wait
-// ---------------------------------------------------------------------------
-struct Ctl {
-    volatile int *abort_flag;   // shared memory
-    int *ws;
-    unsigned long long limit_ns;
-};
-
-// Slow path of a wait.  Not inlined on purpose: the kernel has a dozen wait
-// sites and its code must stay small enough for the instruction caches.
-// CLUSTER: acquire at cluster scope (the barrier also collects arrivals that
-// threads of the peer CTA released at cluster scope).
-template <bool CLUSTER>
-__device__ __noinline__ bool wait_bar_slow(uint32_t bar, uint32_t parity, const Ctl &c, int tag)
-{
-    const uint64_t t0 = global_timer_ns();
-    for (uint32_t it = 1;; ++it) {
-        if (CLUSTER ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity)) return true;
-        if ((it & 63u) == 0u) {
-            if (*c.abort_flag) return false;
-            if (global_timer_ns() - t0 > c.limit_ns) break;
-        }
-    }
-    if (atomicCAS(c.ws + DSQ_WS_STATUS, 0, (int)DSQ_ERR_TIMEOUT) == 0)
-        c.ws[DSQ_WS_DETAIL] = tag;
-    *c.abort_flag = 1;
-    return false;
-}
-
-// Bounded wait of ONE thread (the TMA producer threads).
-__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, const Ctl &c, int tag)
-{
-    if (mbar_try_wait(bar, parity)) return true;
-    return wait_bar_slow<false>(bar, parity, c, tag);
-}
-
-// Bounded wait of a whole converged warp.  All 32 lanes get the same answer:
-// the code behind a wait holds warp-wide instructions (tcgen05.ld / st,
-// __syncwarp), so the lanes must not part ways when one of them sees the phase
-// complete and another the abort flag.
-template <bool CLUSTER = false>
-__device__ __forceinline__ bool wait_bar_warp(uint32_t bar, uint32_t parity, const Ctl &c, int tag)
-{
-    bool ok = CLUSTER ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity);
-    if (!ok) ok = wait_bar_slow<CLUSTER>(bar, parity, c, tag);
-    return __all_sync(0xffffffffu, ok);
-}
-
-// Wait used while leaving after a failure: ignores the abort flag (what is in
-// flight must still land before shared or tensor memory is given up), bounded
-// by DRAIN_LIMIT_NS.
-__device__ __noinline__ void wait_bar_drain(uint32_t bar, uint32_t parity)
-{
-    const uint64_t t0 = global_timer_ns();
-    for (uint32_t it = 1;; ++it) {
-        if (mbar_try_wait(bar, parity)) return;
-        if ((it & 15u) == 0u && global_timer_ns() - t0 > DRAIN_LIMIT_NS) return;
-    }
-}
-
-// ---------------------------------------------------------------------------
-// packed -> int8 expansion.  One 128-code K step of a row is CH packed
-// 16-byte chunks and 32 words (128 bytes) of int8.  Word order (the same for
-// both operands): 4-bit chunk j gives words 8j..8j+3 from the even nibbles of
-// its four words and 8j+4..8j+7 from the odd nibbles; 2-bit chunk j gives
-// words 16j+4c..16j+4c+3 from bit pair c of every byte; 3-bit rows keep the
-// natural order.
-// ---------------------------------------------------------------------------
-template <int BITS, bool SIGNED>
-__device__ __forceinline__ uint32_t expand_word(uint32_t w, int c, uint32_t orv)
-{
-    if (BITS == 4) {
-        if (!SIGNED) return (c == 0 ? w : (w >> 4)) & 0x0F0F0F0Fu;
-        return ((c == 0 ? (w << 4) : w) & 0xF0F0F0F0u) | orv;
-    } else {
-        if (!SIGNED) return (w >> (2 * c)) & 0x03030303u;
-        return ((c == 3 ? w : (w << (6 - 2 * c))) & 0xC0C0C0C0u) | orv;
-    }
-}
-
-// words 4q..4q+3 of a 3-bit row step held in w[12]
-template <bool SIGNED>
-__device__ __forceinline__ uint4 expand3_chunk(const uint32_t (&w)[12], int q, uint32_t orv)
-{
-    uint32_t o[4];
-#pragma unroll
-    for (int t = 0; t < 4; ++t) {
-        const int bit = (16 * q + 4 * t) * 3;
-        const int wi = bit >> 5, sh = bit & 31;
-        const uint32_t hi = wi + 1 < 12 ? w[wi + 1] : 0u;
-        const uint32_t x = __funnelshift_r(w[wi], hi, sh);
-        uint32_t b = (x & 7u) | ((x & 0x38u) << 5) | ((x & 0x1C0u) << 10) |
-                     ((x & 0xE00u) << 15);
-        if (SIGNED) b = (b << 5) | orv;
-        o[t] = b;
-    }
-    return make_uint4(o[0], o[1], o[2], o[3]);
-}
-
-template <int BITS>
-struct Chunks {
-    static constexpr int CH = BITS;              // packed 16-byte chunks per row step
-    static constexpr int OUT = (BITS == 4) ? 2 : 4;   // int8 chunks per packed chunk (2/4-bit)
-};
-
-// whole row step in registers: v[CH] -> o[32]
-template <int BITS, bool SIGNED>
-__device__ __forceinline__ void expand_row_regs(const uint4 (&v)[Chunks<BITS>::CH],
-                                                uint32_t orv, uint32_t (&o)[32])
-{
-    if (BITS == 3) {
-        uint32_t w[12];
-#pragma unroll
-        for (int l = 0; l < 3; ++l) {
-            w[4 * l] = v[l].x; w[4 * l + 1] = v[l].y;
-            w[4 * l + 2] = v[l].z; w[4 * l + 3] = v[l].w;
-        }
-#pragma unroll
-        for (int q = 0; q < 8; ++q) {
-            const uint4 c = expand3_chunk<SIGNED>(w, q, orv);
-            o[4 * q] = c.x; o[4 * q + 1] = c.y; o[4 * q + 2] = c.z; o[4 * q + 3] = c.w;
-        }
-    } else {
-        constexpr int OUT = Chunks<BITS>::OUT;
-#pragma unroll
-        for (int j = 0; j < Chunks<BITS>::CH; ++j)
-#pragma unroll
-            for (int c = 0; c < OUT; ++c) {
-                const int b = (j * OUT + c) * 4;
-                o[b] = expand_word<BITS, SIGNED>(v[j].x, c, orv);
-                o[b + 1] = expand_word<BITS, SIGNED>(v[j].y, c, orv);
-                o[b + 2] = expand_word<BITS, SIGNED>(v[j].z, c, orv);
-                o[b + 3] = expand_word<BITS, SIGNED>(v[j].w, c, orv);
-            }
-    }
-}
 
 // ---------------------------------------------------------------------------
 // the kernel
@@ -1364,26 +1220,8 @@ __global__ void __launch_bounds__(128, 1) mma_rate_kernel(int iters, int *ws)
 // ---------------------------------------------------------------------------
 // host side
 // ---------------------------------------------------------------------------
-typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *,
-                                  const cuuint64_t *, const cuuint64_t *, const cuuint32_t *,
-                                  const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn get_encode_fn()
-{
-    static EncodeTiledFn fn = nullptr;
-    static bool tried = false;
-    if (!tried) {
-        tried = true;
-        void *sym = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) ==
-                cudaSuccess &&
-            qres == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(sym);
-    }
-    return fn;
-}
+typedef DsqEncodeTiledFn EncodeTiledFn;
+EncodeTiledFn get_encode_fn() { return dsq_encode_tiled_fn(); }
 
 // 2-D byte map over packed rows: inner dimension = row bytes, outer = rows.
 struct TcMaps { CUtensorMap b, a; };   // the two operands
@@ -1458,27 +1296,8 @@ int a_run_log2(int P, int bits, int ks)
     return l;
 }
 
-typedef CUresult (*EncodeIm2colFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *,
-                                   const cuuint64_t *, const cuuint64_t *, const int *,
-                                   const int *, cuuint32_t, cuuint32_t, const cuuint32_t *,
-                                   CUtensorMapInterleave, CUtensorMapSwizzle,
-                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeIm2colFn get_encode_im2col_fn()
-{
-    static EncodeIm2colFn fn = nullptr;
-    static bool tried = false;
-    if (!tried) {
-        tried = true;
-        void *sym = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeIm2col", &sym, cudaEnableDefault, &qres) ==
-                cudaSuccess &&
-            qres == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeIm2colFn>(sym);
-    }
-    return fn;
-}
+typedef DsqEncodeIm2colFn EncodeIm2colFn;
+EncodeIm2colFn get_encode_im2col_fn() { return dsq_encode_im2col_fn(); }
 
 CUtensorMapSwizzle swizzle_for_span(int bytes)
 {
@@ -1568,6 +1387,7 @@ std::atomic<int> g_forced_ks{0};      // dsq_set_round_k_steps: 0 automatic, 1 s
 std::atomic<int> g_pair_mode{0};      // dsq_set_cta_pairs: 0 automatic, 1 never, 2 wherever possible
 std::atomic<unsigned long long> g_wait_ns{WAIT_LIMIT_NS};   // dsq_set_wait_limit_ns
 std::atomic<int> g_skip_b_round{-1};  // dsq_set_test_skip_b_round
+std::atomic<int> g_window3{1};        // dsq_set_conv3_window
 
 int pick_bn(int m_tiles, int ncols, int bits)
 {
@@ -1734,6 +1554,49 @@ int pick_pm(const TcParams &p, int bits, bool im2col)
 
 }  // namespace
 
+// ---- shared with the other tensor-core translation unit (dsq_tc_host.h) -------
+DsqLaunchHooks dsq_launch_hooks()
+{
+    DsqLaunchHooks h;
+    h.pdl = g_pdl.load();
+    h.wait_ns = g_wait_ns.load();
+    h.skip_b_round = g_skip_b_round.load();
+    h.window3 = g_window3.load();
+    return h;
+}
+
+static void *driver_entry_point(const char *name)
+{
+    void *sym = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint(name, &sym, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess)
+        return nullptr;
+    return sym;
+}
+
+DsqEncodeTiledFn dsq_encode_tiled_fn()
+{
+    static std::atomic<void *> fn{nullptr};
+    void *f = fn.load(std::memory_order_acquire);
+    if (!f) {
+        f = driver_entry_point("cuTensorMapEncodeTiled");
+        fn.store(f, std::memory_order_release);
+    }
+    return reinterpret_cast<DsqEncodeTiledFn>(f);
+}
+
+DsqEncodeIm2colFn dsq_encode_im2col_fn()
+{
+    static std::atomic<void *> fn{nullptr};
+    void *f = fn.load(std::memory_order_acquire);
+    if (!f) {
+        f = driver_entry_point("cuTensorMapEncodeIm2col");
+        fn.store(f, std::memory_order_release);
+    }
+    return reinterpret_cast<DsqEncodeIm2colFn>(f);
+}
+
 extern "C" {
 
 int dsq_set_round_k_steps(int ks)
@@ -1760,6 +1623,13 @@ int dsq_set_dependent_launch(int on)
 int dsq_set_test_skip_b_round(int round)
 {
     g_skip_b_round = round < 0 ? -1 : round;
+    return DSQ_OK;
+}
+
+int dsq_set_conv3_window(int mode)
+{
+    if (mode < 0 || mode > 3) return DSQ_ERR_SHAPE;
+    g_window3 = mode;
     return DSQ_OK;
 }
 
@@ -1874,6 +1744,17 @@ int dsq_conv2d(const void *act_codes, const dsq_nhwc_t *shape, const dsq_quant_t
     st = dsq_make_epi(ep, bits, y_f32, y_codes, acc_out, &e);
     if (st) return st;
 
+    // largest |2*acc + S_a| below 2^22: the epilogue may convert integers to
+    // float through the 1.5 * 2^23 bias trick, which is exact there
+    const int small_acc = (double)taps * conv->Cin * (double)((1 << bits) - 1) *
+                              (2.0 * (double)(1 << (bits - 1)) + 1.0) < 4194304.0;
+    const int epi = (y_f32 || acc_out || !y_codes) ? EPI_GENERAL
+                    : (e.residual ? EPI_CODES_RES : EPI_CODES);
+    // 3x3 stride-1 convolutions: every input pixel expanded once (dsq_conv3.cu)
+    st = dsq_conv3_window(act_codes, shape, bits, w_packed, conv, e, epi, small_acc, workspace,
+                          (cudaStream_t)stream);
+    if (st != DSQ_ERR_UNSUPPORTED) return st;
+
     const size_t P = dsq_row_pitch(conv->Cin, bits);
     const size_t row_bytes = (size_t)taps * P;
     TcParams p = {};
@@ -1912,12 +1793,7 @@ int dsq_conv2d(const void *act_codes, const dsq_nhwc_t *shape, const dsq_quant_t
     // a 1x1 stride-1 unpadded convolution reads the pixel rows as they lie
     st = setup_a_tma(&p, &tmap.a, act_codes, M, bits, ks, plain_rows, shape, conv->KH, pm == 5);
     if (st) return st;
-    // largest |2*acc + S_a| below 2^22: the epilogue may convert integers to
-    // float through the 1.5 * 2^23 bias trick, which is exact there
-    p.small_acc = (double)taps * conv->Cin * (double)((1 << bits) - 1) *
-                          (2.0 * (double)(1 << (bits - 1)) + 1.0) < 4194304.0;
-    const int epi = (y_f32 || acc_out || !y_codes) ? EPI_GENERAL
-                    : (e.residual ? EPI_CODES_RES : EPI_CODES);
+    p.small_acc = small_acc;
     return dispatch_tc(bits, epi, pm, tmap, p, (cudaStream_t)stream);
 }
 

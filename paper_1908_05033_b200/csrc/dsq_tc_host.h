@@ -1,0 +1,46 @@
+// Host-side pieces shared by the two tensor-core translation units
+// (dsq_tc.cu, dsq_conv3.cu).  Internal to the library.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include "dsq_epilogue.cuh"
+
+#define DSQ_HIDDEN __attribute__((visibility("hidden")))
+
+// current values of the process-wide hooks (csrc/dsq_hooks.h)
+struct DsqLaunchHooks {
+    int pdl;                    // programmatic dependent launch on / off
+    unsigned long long wait_ns; // limit of the device-side waits
+    int skip_b_round;           // test hook, -1 = off
+    int window3;                // dsq_set_conv3_window
+};
+DSQ_HIDDEN DsqLaunchHooks dsq_launch_hooks();
+
+typedef CUresult (*DsqEncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *,
+                                     const cuuint64_t *, const cuuint64_t *, const cuuint32_t *,
+                                     const cuuint32_t *, CUtensorMapInterleave,
+                                     CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                     CUtensorMapFloatOOBfill);
+typedef CUresult (*DsqEncodeIm2colFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *,
+                                      const cuuint64_t *, const cuuint64_t *, const int *,
+                                      const int *, cuuint32_t, cuuint32_t, const cuuint32_t *,
+                                      CUtensorMapInterleave, CUtensorMapSwizzle,
+                                      CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+// driver entry points (looked up once; nullptr when the driver lacks them)
+DSQ_HIDDEN DsqEncodeTiledFn dsq_encode_tiled_fn();
+DSQ_HIDDEN DsqEncodeIm2colFn dsq_encode_im2col_fn();
+
+// epilogue variants of the convolution kernels: codes only, without / with a
+// residual operand; any outputs
+enum { DSQ_EPI_CODES = 1, DSQ_EPI_CODES_RES = 2, DSQ_EPI_GENERAL = 3 };
+
+// 3x3, stride 1, pad 1 convolution on an expanded shared-memory window
+// (dsq_conv3.cu).  Arguments are those of dsq_conv2d after validation.
+// Returns DSQ_ERR_UNSUPPORTED without launching anything when the geometry is
+// not one it handles; the caller then takes the im2col kernel.
+DSQ_HIDDEN int dsq_conv3_window(const void *act_codes, const dsq_nhwc_t *shape, int bits,
+                                const void *w_packed, const dsq_conv_t *conv, const DsqEpi &e,
+                                int epi_kind, int small_acc, void *workspace,
+                                cudaStream_t stream);

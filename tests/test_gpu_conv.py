@@ -200,3 +200,48 @@ def test_depthwise(dsq, geom, bits, w_off):
     dw_case(dsq, *geom, bits, w_off)
     if geom[4] == 1:
         dw_case(dsq, *geom, bits, w_off, residual=True)
+
+
+WINDOW_GEOMS = [  # N, H, W, Cin, Cout: 3x3, stride 1, pad 1 on the shared-memory window
+    (1, 3, 3, 64, 64), (2, 9, 7, 64, 40), (2, 9, 7, 128, 200), (1, 1, 1, 128, 64),
+    (3, 7, 7, 512, 512), (2, 28, 28, 256, 300), (5, 14, 14, 256, 256),
+    (1, 20, 150, 64, 64),      # wide image: three bands of 136 pixels
+    (1, 6, 300, 128, 72), (2, 56, 56, 128, 128), (70, 5, 5, 64, 96)]
+
+
+@pytest.mark.parametrize("bits", [2, 4])
+@pytest.mark.parametrize("geom", WINDOW_GEOMS)
+def test_conv3x3_window_kernel(dsq, geom, bits):
+    """3x3 stride-1 convolutions whose A operand is an expanded window of the
+    input in shared memory (one constant row shift per filter tap): image sizes
+    from 1x1 to wider than a window, tiles that span several images, channel
+    counts with a ragged last N tile, one to four planes of 128 channels, with
+    and without a residual operand, every element against the oracle."""
+    n, h, w, ci, co = geom
+    dsq.dsq_set_conv3_window(3)        # this kernel wherever the geometry allows
+    try:
+        conv_case(dsq, n, h, w, ci, co, 3, 1, 1, bits, 0.5, residual=(n % 2 == 0),
+                  seed=n + h + ci)
+        conv_case(dsq, n, h, w, ci, co, 3, 1, 1, bits, 0.0, per_channel=True, seed=co)
+    finally:
+        dsq.dsq_set_conv3_window(1)
+
+
+@pytest.mark.parametrize("bits", [2, 4])
+def test_conv3x3_window_and_im2col_kernels_agree(dsq, bits):
+    """The same convolution through both tensor-core kernels (hook) gives the
+    same codes; both are compared with the oracle elsewhere."""
+    c = dsq_inputs.conv3x3_case(N=3, H=19, W=23, Cin=128, Cout=128, bits=bits)
+    ws = dsq.new_workspace()
+    act = dsq.dsq_quantize_act(T(c["x"]), bits, 0.0, 2.0)
+    blob, conv = dsq.dsq_pack_weights(T(c["w"]), bits, -0.1, 0.1, ws, stride=1, pad=1)
+    args = (act, c["x"].shape, (bits, 0.0, 2.0), blob, conv, T(c["scale"]), T(c["bias"]), ws)
+    dsq.dsq_set_conv3_window(3)
+    try:
+        a, _, _ = dsq.dsq_conv2d(*args, w_offset=0.5, requant=(bits, 0.0, 1.5))
+        dsq.dsq_set_conv3_window(0)
+        b, _, _ = dsq.dsq_conv2d(*args, w_offset=0.5, requant=(bits, 0.0, 1.5))
+    finally:
+        dsq.dsq_set_conv3_window(1)
+    assert dsq.dsq_workspace_status(ws) == 0
+    assert torch.equal(a, b)
