@@ -33,6 +33,13 @@
 //     of the whole layer sit in shared memory, the residual words of a tile
 //     are fetched before its accumulators are waited for.
 //
+// Measured: with the A operand read through a shared-memory descriptor an
+// instruction takes about 110-130 clocks whatever its N (the tensor core
+// fetches A at roughly 32 bytes a clock), so only 256-wide N tiles run the
+// tensor pipe at its full rate; a variant that copied each K step of the
+// window to tensor memory (ld.shared + tcgen05.st, A taken from there) was
+// slower than this one at every layer size and is not kept.
+//
 // Wide images (W + 2 > 139) would need a window of more than 416 pixels; they
 // are staged as three bands of 136 pixels, one per filter row, instead.
 //
@@ -557,7 +564,6 @@ dsq_win3_kernel(const __grid_constant__ CUtensorMap tmap_b,
         const float *lut = reinterpret_cast<const float *>(smem + L.lut);
         const DsqEpi &e = p.e;
         constexpr int CWU = BITS / 2;                        // code words per 16 columns
-        constexpr int MAX_UNITS = 256 / 16 / W3_EPQ;         // units of a warp per tile
         // scale (halved for the symmetric weight grid) and bias of every output
         // channel, once per CTA; columns past Cout get 0
         for (int c = threadIdx.x - W3_WARP_E0 * 32; c < p.cout_pad; c += W3_NUM_E_WARPS * 32) {
@@ -589,35 +595,37 @@ dsq_win3_kernel(const __grid_constant__ CUtensorMap tmap_b,
             const bool row_ok = pos.n < p.N && pos.h < p.H && pos.w < p.W;
             const int64_t m = ((int64_t)pos.n * p.H + pos.h) * p.W + pos.w;
             pos = w3_add(pos, p.t_dn, p.t_dh, p.t_dw, p.Hp, p.Wp);
-            // residual codes of this row's units, fetched while the tile's
-            // instructions are still running
-            uint32_t resw[MAX_UNITS][CWU];
+            // residual codes of a unit of this row are fetched one unit ahead (the
+            // first unit's while the tile's instructions are still running); the
+            // unit loop is not unrolled: the kernel's roles share the instruction
+            // caches, and every role runs faster when the whole kernel is small
+            uint32_t res_nx[CWU];
+            auto fetch_res = [&](int u) {
 #pragma unroll
-            for (int i = 0; i < MAX_UNITS; ++i) {
-#pragma unroll
-                for (int w = 0; w < CWU; ++w) resw[i][w] = 0u;
-                const int u = k + i * W3_EPQ;
+                for (int w = 0; w < CWU; ++w) res_nx[w] = 0u;
                 const int byte0 = (n_tile * BN + u * 16) * BITS / 8;
                 if (EPI != DSQ_EPI_CODES && e.residual && row_ok && u < units &&
                     byte0 < p.out_pitch) {
                     const uint32_t *rp =
                         reinterpret_cast<const uint32_t *>(e.residual + m * p.out_pitch + byte0);
 #pragma unroll
-                    for (int w = 0; w < CWU; ++w) resw[i][w] = __ldg(rp + w);
+                    for (int w = 0; w < CWU; ++w) res_nx[w] = __ldg(rp + w);
                 }
-            }
+            };
+            fetch_res(k);
             if (warp == W3_WARP_E0) W3_STAMP(7, it);
             if (!(ok = wait_bar_warp(bar_acc_full(as), (it >> 1) & 1u, ctl, 8))) break;
             if (warp == W3_WARP_E0) W3_STAMP(8, it);
             tc_fence_after_sync();
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + as * BN;
+#pragma unroll 1
+            for (int u = k; u < units; u += W3_EPQ) {
+                uint32_t r[16], resw[CWU];
 #pragma unroll
-            for (int i = 0; i < MAX_UNITS; ++i) {
-                const int u = k + i * W3_EPQ;
-                if (u >= units) break;                       // warp-uniform
-                uint32_t r[16];
+                for (int w = 0; w < CWU; ++w) resw[w] = res_nx[w];
                 __syncwarp();
                 tmem_ld_32x16(taddr + u * 16, r);
+                fetch_res(u + W3_EPQ);
                 tmem_ld_wait();
                 const int n0 = n_tile * BN + u * 16;
                 const int byte0 = n0 * BITS / 8;
@@ -626,12 +634,12 @@ dsq_win3_kernel(const __grid_constant__ CUtensorMap tmap_b,
                 if (EPI == DSQ_EPI_CODES || EPI == DSQ_EPI_CODES_RES) {
                     if (byte0 >= p.out_pitch) continue;
                     w3_codes_unit<BITS, EPI == DSQ_EPI_CODES_RES>(
-                        r, sm_scale + n0, sm_bias + n0, resw[i], lut, p.shift, e.rq.inv, p.r_hi, cw);
+                        r, sm_scale + n0, sm_bias + n0, resw, lut, p.shift, e.rq.inv, p.r_hi, cw);
                 } else {
                     constexpr uint32_t MASK = (1u << BITS) - 1u;
 #pragma unroll
                     for (int w = 0; w < CWU; ++w) cw[w] = 0u;
-#pragma unroll
+#pragma unroll 4
                     for (int c = 0; c < 16; ++c) {
                         const int v = (int)r[c] >> p.shift;
                         if (n0 + c < p.Ncols) {
@@ -639,7 +647,7 @@ dsq_win3_kernel(const __grid_constant__ CUtensorMap tmap_b,
                             float y = dsq_epi_y(v, sm_scale[n0 + c], sm_bias[n0 + c]);
                             if (e.residual) {
                                 const uint32_t qr =
-                                    (resw[i][(c * BITS) >> 5] >> ((c * BITS) & 31)) & MASK;
+                                    (resw[(c * BITS) >> 5] >> ((c * BITS) & 31)) & MASK;
                                 y = dsq_epi_residual(y, qr, e.res_delta, e.res_lo);
                             }
                             if (e.has_requant)
