@@ -572,6 +572,27 @@ def run_ours(args):
         extras["quantize_act_b4_1GiB"] = {"GB/s": gbs, "frac_of_hbm_peak": gbs / peaks["hbm_gbs"],
                                           "ms": qms, "bytes_per_element": 4.5}
         del big, outq
+        # training-side soft quantiser (Eq. 5 forward, Eq. 10-13 backward), 512 MiB fp32
+        xs_ = torch.empty(1 << 27, dtype=torch.float32, device=dev).normal_()
+        gs_ = torch.empty_like(xs_).normal_()
+        ys_ = torch.empty_like(xs_)
+        gp_ = torch.empty(3, dtype=torch.float64, device=dev)
+        for name, fn, bpe in (("fwd", lambda: dsq.dsq_soft_quantize_fwd(xs_, 4, -1.0, 2.0, 0.2, out=ys_), 8.0),
+                              ("bwd", lambda: dsq.dsq_soft_quantize_bwd(xs_, gs_, 4, -1.0, 2.0, 0.2, out=ys_,
+                                                                        grad_params=gp_), 12.0)):
+            for _ in range(3):
+                fn()
+            e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(10):
+                fn()
+            e1.record(); torch.cuda.synchronize()
+            sms = e0.elapsed_time(e1) / 10
+            sgbs = xs_.numel() * bpe / (sms * 1e-3) / 1e9
+            extras["soft_quantize_" + name + "_b4_512MiB"] = {
+                "GB/s": sgbs, "frac_of_hbm_peak": sgbs / peaks["hbm_gbs"], "ms": sms,
+                "bytes_per_element": bpe}
+        del xs_, gs_, ys_, gp_
         # 4096^3 4-bit GEMM
         A, Bm, rs = dsq_inputs.gemm_case(4096, 4096, 4096, 4)
         Ap = dsq.dsq_pack_codes(torch.from_numpy(A).to(dev), 4)

@@ -247,6 +247,36 @@ int dsq_gemm_static_ws(const void *A_codes, const void *B_codes, int64_t M,
 int dsq_maxpool2x2(const void *codes_in, const dsq_nhwc_t *shape, int bits,
                    void *codes_out, size_t bytes, void *stream);
 
+/* ---- training side: the soft quantiser and its gradients ---------------- */
+
+/* Forward of DSQ's differentiable soft quantiser (paper Sec. 3.2-3.3,
+ * Eq. 3-8; Algorithm 1 feed-forward step 2 composed with step 4):
+ *   y = l (x < l);  u (x > u);  l + Delta (i + (phi(x) + 1)/2) for x in P_i,
+ *   phi(x) = s tanh(k (x - m_i)),  m_i = l + (i + 1/2) Delta,
+ *   s = 1/(1 - alpha),  k = log(2/alpha - 1)/Delta,  Delta = (u - l)/(2^b - 1),
+ *   P_i = [l + i Delta, l + (i+1) Delta), i = 0 .. 2^b - 2.
+ * x, y: fp32 device arrays of n elements (16-byte aligned); q->bits in 1..8
+ * (1 = the binary case, one interval); 0 < alpha < 1 (the paper keeps it in
+ * (0, 0.5)), else DSQ_ERR_RANGE.  Arithmetic is binary32; NaN stays NaN.
+ * HBM-bound: 8 bytes per element. */
+int dsq_soft_quantize_fwd(const float *x, int64_t n, const dsq_quant_t *q,
+                          float alpha, float *y, void *stream);
+
+/* Back-propagation through y = Q_S(x) (paper Eq. 10-13 and the
+ * back-propagation lines of Algorithm 1), the interval index taken as
+ * piecewise constant:
+ *   grad_x[j] = grad_y[j] * dQ_S/dx            (0 outside [l, u])
+ *   grad_params[0] = sum_j grad_y[j] * dQ_S/dalpha            (Eq. 10)
+ *   grad_params[1] = sum_j grad_y[j] * dQ_S/dl   (1 for x < l; Eq. 11)
+ *   grad_params[2] = sum_j grad_y[j] * dQ_S/du   (1 for x > u; Eq. 12)
+ * grad_params: three doubles in device memory (8-byte aligned), overwritten
+ * (cleared on `stream`, then accumulated with double-precision atomic adds:
+ * the order of the additions, and so the last bits, may differ from run to
+ * run).  Element terms are binary32.  HBM-bound: 12 bytes per element. */
+int dsq_soft_quantize_bwd(const float *x, const float *grad_y, int64_t n,
+                          const dsq_quant_t *q, float alpha, float *grad_x,
+                          double *grad_params, void *stream);
+
 /* ---- format helpers (tests, tooling) ----------------------------------- */
 
 /* int8 codes [rows][k] (dense) -> packed rows.  Values are truncated to

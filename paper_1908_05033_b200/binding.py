@@ -70,6 +70,9 @@ _SIGNATURES = {
                                   _int, _vp]),
     "dsq_maxpool2x2": (_int, [_vp, C.POINTER(dsq_nhwc_t), _int, _vp, _sz,
                               _vp]),
+    "dsq_soft_quantize_fwd": (_int, [_vp, _i64, C.POINTER(dsq_quant_t), C.c_float, _vp, _vp]),
+    "dsq_soft_quantize_bwd": (_int, [_vp, _vp, _i64, C.POINTER(dsq_quant_t), C.c_float, _vp,
+                                     _vp, _vp]),
     "dsq_pack_codes": (_int, [_vp, _i64, _i64, _int, _vp, _sz, _vp]),
     "dsq_unpack": (_int, [_vp, _i64, _i64, _int, _int, _vp, _vp]),
     "dsq_probe_i8_mma_rate": (_int, [_int, C.POINTER(C.c_float),
@@ -307,6 +310,30 @@ def dsq_maxpool2x2(codes, shape, bits, out=None):
     _check(lib.dsq_maxpool2x2(_p(codes), C.byref(nhwc), bits, _p(out),
                               out.numel(), _stream()), "dsq_maxpool2x2")
     return out
+
+
+# ---- training side: soft quantiser -----------------------------------------------
+def dsq_soft_quantize_fwd(x, bits, lo, hi, alpha, out=None):
+    """y = Q_S(x) (Eq. 5), fp32 CUDA tensor of any shape."""
+    _need(x, torch.float32, "x")
+    y = out if out is not None else torch.empty_like(x)
+    q = dsq_quant_t(bits, lo, hi)
+    _check(lib.dsq_soft_quantize_fwd(_p(x), x.numel(), C.byref(q), alpha, _p(y), _stream()),
+           "dsq_soft_quantize_fwd")
+    return y
+
+
+def dsq_soft_quantize_bwd(x, grad_y, bits, lo, hi, alpha, out=None, grad_params=None):
+    """Returns (grad_x fp32 like x, grad_params fp64 [3] = dL/d(alpha, l, u))."""
+    _need(x, torch.float32, "x")
+    _need(grad_y, torch.float32, "grad_y")
+    gx = out if out is not None else torch.empty_like(x)
+    gp = grad_params if grad_params is not None else torch.empty(
+        3, dtype=torch.float64, device=x.device)
+    q = dsq_quant_t(bits, lo, hi)
+    _check(lib.dsq_soft_quantize_bwd(_p(x), _p(grad_y), x.numel(), C.byref(q), alpha, _p(gx),
+                                     _p(gp), _stream()), "dsq_soft_quantize_bwd")
+    return gx, gp
 
 
 # ---- GEMM -------------------------------------------------------------------------

@@ -4,6 +4,7 @@
     python -m paper_1908_05033_b200.cases conv --cin 64 --cout 64 --hw 56 --batch 64 --ksize 3
     python -m paper_1908_05033_b200.cases quant --mb 1024 --bits 4
     python -m paper_1908_05033_b200.cases dw --c 192 --hw 56 --batch 64
+    python -m paper_1908_05033_b200.cases soft --mb 1024 --bits 4
 
 Each runs the named kernel `--iters` times on seeded synthetic inputs (an L2
 flush between launches) and prints the median CUDA-event time with the
@@ -38,7 +39,7 @@ def _timeit(fn, iters, flush):
 
 def main(argv=None):
     ap = argparse.ArgumentParser()
-    ap.add_argument("case", choices=["gemm", "conv", "quant", "dw"])
+    ap.add_argument("case", choices=["gemm", "conv", "quant", "dw", "soft"])
     ap.add_argument("--size", type=int, default=4096)
     ap.add_argument("--bits", type=int, default=4)
     ap.add_argument("--iters", type=int, default=5)
@@ -111,6 +112,19 @@ def main(argv=None):
                              flush)
         nbytes = rows * 64 * 4 + o.numel()
         out.update(elements=rows * 64, ms=ms, gbs=nbytes / (ms * 1e-3) / 1e9, all_ms=all_ms)
+    elif a.case == "soft":
+        # training-side soft quantiser: forward (8 B / element) and backward (12 B / element)
+        n = a.mb * (1 << 20) // 4
+        x = torch.randn(n, device=dev, generator=gen)
+        g = torch.randn(n, device=dev, generator=gen)
+        y = torch.empty_like(x)
+        gp = torch.empty(3, dtype=torch.float64, device=dev)
+        ms, all_ms = _timeit(lambda: B.dsq_soft_quantize_fwd(x, bits, -1.0, 2.0, 0.2, out=y),
+                             a.iters, flush)
+        msb, all_b = _timeit(lambda: B.dsq_soft_quantize_bwd(x, g, bits, -1.0, 2.0, 0.2, out=y,
+                                                             grad_params=gp), a.iters, flush)
+        out.update(elements=n, fwd_ms=ms, fwd_gbs=8.0 * n / (ms * 1e-3) / 1e9, bwd_ms=msb,
+                   bwd_gbs=12.0 * n / (msb * 1e-3) / 1e9, all_ms=all_ms + all_b)
     else:
         shape = (a.batch, a.hw, a.hw, a.c)
         pitch = B.dsq_row_pitch(a.c, bits)

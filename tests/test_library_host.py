@@ -112,6 +112,16 @@ def test_validation_status_codes_without_a_gpu():
     assert lib.dsq_conv2d(fake, C.byref(shape), C.byref(q4), fake, C.byref(conv),
                           C.byref(ep), None, fake, None, fake, 256, None) == -3
 
+    # soft quantiser: alpha outside (0, 1), bits outside 1..8, NULL
+    qs = B.dsq_quant_t(4, 0.0, 1.0)
+    assert lib.dsq_soft_quantize_fwd(fake, 16, C.byref(qs), C.c_float(0.0), fake, None) == -6
+    assert lib.dsq_soft_quantize_fwd(fake, 16, C.byref(qs), C.c_float(1.5), fake, None) == -6
+    assert lib.dsq_soft_quantize_fwd(fake, 16, C.byref(B.dsq_quant_t(0, 0.0, 1.0)), C.c_float(0.2),
+                                     fake, None) == -3
+    assert lib.dsq_soft_quantize_fwd(None, 16, C.byref(qs), C.c_float(0.2), fake, None) == -1
+    assert lib.dsq_soft_quantize_bwd(fake, fake, 16, C.byref(qs), C.c_float(0.2), fake, None, None) == -1
+    assert lib.dsq_soft_quantize_bwd(fake, fake, 0, C.byref(qs), C.c_float(0.2), fake, fake, None) == -4
+
     # depthwise wants groups = C
     assert lib.dsq_dwconv2d(fake, C.byref(shape), C.byref(q4), fake, C.byref(conv),
                             C.byref(ep), fake, None, None, None) == -4
