@@ -173,8 +173,8 @@ int dsq_quantize_act(const float *x, const dsq_nhwc_t *shape,
  *              ep->requant.bits == act_q->bits)
  *   acc_out    nullable: raw int32 accumulators [N][Ho][Wo][Cout]
  *              (2*acc + S_a when w_offset = 0.5)
- * KH = KW in {1, 3}, stride in {1, 2}; bits in {2, 4} (3-bit convolution is
- * not implemented: DSQ_ERR_UNSUPPORTED). */
+ * KH = KW in {1, 3}, stride in {1, 2}; bits in {2, 3, 4} (3-bit convolution:
+ * the paper's Table 8 times it on every layer shape). */
 int dsq_conv2d(const void *act_codes, const dsq_nhwc_t *shape,
                const dsq_quant_t *act_q, const void *w_packed,
                const dsq_conv_t *conv, const dsq_epilogue_t *ep,
@@ -187,7 +187,7 @@ int dsq_conv2d(const void *act_codes, const dsq_nhwc_t *shape,
  * per channel):
  * acc[n][ho][wo][c] = sum over the 3x3 taps of q_a * c_w, then the same
  * epilogue with per-channel S_a.  Same arguments as dsq_conv2d;
- * conv->groups = Cin = Cout = shape->C, KH = KW = 3, pad = 1, bits in {2,4}.
+ * conv->groups = Cin = Cout = shape->C, KH = KW = 3, pad = 1, bits in {2,3,4}.
  * HBM-bound: bits/8 bytes in and out per element. */
 int dsq_dwconv2d(const void *act_codes, const dsq_nhwc_t *shape,
                  const dsq_quant_t *act_q, const void *w_packed,

@@ -90,6 +90,8 @@ struct W3Params {
     int E;                             // int8 bytes per pixel = Cin
     int npl, kpp, ksteps;              // planes of 128 channels, K steps per plane, total
     int PB, cpp;                       // packed bytes per pixel and plane; 16-byte chunks of it
+    int two_taps;                      // 64-channel rows of 2 / 4 bits: a K step is two filter taps
+    int xstep;                         // bytes between two K steps of a plane in a weight row
     int apx;                           // pixels of an A slot
     int a_box, a_nload, nbands, band_px;
     int tap_stride;                    // slot rows between two filter rows
@@ -288,10 +290,12 @@ dsq_win3_kernel(const __grid_constant__ CUtensorMap tmap_b,
         uint32_t *tab = reinterpret_cast<uint32_t *>(smem + L.a_tab);
         for (int i = lane; i < 4 * p.kpp; i += 32) {
             const int kk = i >> 2, j = i & 3;
-            const int tap = p.E == 64 ? 2 * kk + (j >> 1) : kk;
-            const int within = p.E == 64 ? 32 * (j & 1) : 32 * j;
+            const int tap = p.two_taps ? 2 * kk + (j >> 1) : kk;
+            const int within = p.two_taps ? 32 * (j & 1) : 32 * j;
             const int kh = tap / 3, kw = tap - 3 * kh;
-            tab[i] = tap < 9 ? (uint32_t)((kh * p.tap_stride + kw) * 8 + (within >> 4)) : 0xFFFFFFFFu;
+            tab[i] = tap < 9 && within < p.E
+                         ? (uint32_t)((kh * p.tap_stride + kw) * 8 + (within >> 4))
+                         : 0xFFFFFFFFu;
         }
     }
     if (warp == W3_WARP_TMA_B && lane == 0) tma_prefetch_desc(&tmap_b);
@@ -318,7 +322,7 @@ dsq_win3_kernel(const __grid_constant__ CUtensorMap tmap_b,
             const int y = n_tile * BN;
             // byte offset of a K step in a weight row of 9 taps x Cin codes: tap kk,
             // plane pl (64-channel inputs: two taps per K step)
-            const int xstep = p.E == 64 ? 16 * BITS : (p.E * BITS) / 8;
+            const int xstep = p.xstep;
             int s = 0, kk = 0, xk = 0, xpl = 0;
 #pragma unroll 1
             for (uint32_t g = 0; g < n_b_fills; ++g) {
@@ -465,6 +469,29 @@ dsq_win3_kernel(const __grid_constant__ CUtensorMap tmap_b,
             if (warp == W3_WARP_A0) W3_STAMP(2, g);
             const uint32_t src = smem_u32(smem + L.a_stage) + ss * a_stage_bytes;
             const uint32_t dst = smem_u32(smem + L.a_slots) + slot * a_slot_bytes;
+            if (BITS == 3) {
+                // 3-bit rows: one task per pixel (8 codes per 3 bytes from the
+                // row's start): its 32 or 48 packed bytes -> 64 or 128 int8 bytes
+                const int nq = p.E >= 128 ? 8 : 4;
+#pragma unroll 1
+                for (int px = tid; px < p.apx; px += W3_NUM_A_WARPS * 32) {
+                    uint32_t w[12];
+#pragma unroll
+                    for (int l = 0; l < 3; ++l) {
+                        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+                        if (l < p.cpp) v = lds_128(src + (uint32_t)(px * p.PB + 16 * l));
+                        w[4 * l] = v.x; w[4 * l + 1] = v.y; w[4 * l + 2] = v.z; w[4 * l + 3] = v.w;
+                    }
+                    const uint32_t row = dst + (uint32_t)px * 128u;
+                    const int sw = px & 7;
+#pragma unroll
+                    for (int q = 0; q < 8; ++q)
+                        if (q < nq) {
+                            const uint4 c = expand3_chunk<false>(w, q, 0u);
+                            sts_128(row + (uint32_t)((q ^ sw) << 4), c.x, c.y, c.z, c.w);
+                        }
+                }
+            } else
 #pragma unroll 4
             for (int t = tid; t < n_tasks; t += W3_NUM_A_WARPS * 32) {
                 const int px = t >> lcpp, ch = t & (p.cpp - 1);
@@ -510,6 +537,35 @@ dsq_win3_kernel(const __grid_constant__ CUtensorMap tmap_b,
             const uint4 *src = reinterpret_cast<const uint4 *>(smem + L.b_packed + sp * b_packed_bytes);
             uint8_t *rowp = smem + L.b_tiles + st * b_stage_bytes + row0 * 128;
             bool waited = p.b_res != 0;
+            if (BITS == 3) {
+                // 3-bit rows: one thread per row of 48 packed bytes
+                uint32_t w[2][12];
+#pragma unroll
+                for (int i = 0; i < 2; ++i)
+                    if (tid + i * BT < BN) {
+                        const uint4 *r4 = reinterpret_cast<const uint4 *>(
+                            smem + L.b_packed + sp * b_packed_bytes + (tid + i * BT) * 48);
+#pragma unroll
+                        for (int l = 0; l < 3; ++l) {
+                            const uint4 v = r4[l];
+                            w[i][4 * l] = v.x; w[i][4 * l + 1] = v.y;
+                            w[i][4 * l + 2] = v.z; w[i][4 * l + 3] = v.w;
+                        }
+                    }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_bp_empty(sp));
+                if (!waited && !(ok = wait_bar_warp(bar_b_empty(st), phu ^ 1u, ctl, 7))) break;
+#pragma unroll
+                for (int i = 0; i < 2; ++i)
+                    if (tid + i * BT < BN) {
+                        uint8_t *rp = smem + L.b_tiles + st * b_stage_bytes + (tid + i * BT) * 128;
+                        const int sw3 = (tid + i * BT) & 7;
+#pragma unroll
+                        for (int q = 0; q < 8; ++q)
+                            *reinterpret_cast<uint4 *>(rp + ((q ^ sw3) << 4)) =
+                                expand3_chunk<true>(w[i], q, p.orv);
+                    }
+            } else
             // 128 rows at a time (register budget)
 #pragma unroll 1
             for (int r0 = 0; r0 < BN; r0 += 128) {
@@ -563,7 +619,10 @@ dsq_win3_kernel(const __grid_constant__ CUtensorMap tmap_b,
         float *sm_bias = sm_scale + p.cout_pad;
         const float *lut = reinterpret_cast<const float *>(smem + L.lut);
         const DsqEpi &e = p.e;
-        constexpr int CWU = BITS / 2;                        // code words per 16 columns
+        // a unit = the columns whose codes fill whole 32-bit words: 16 columns
+        // (32 for 3-bit codes, where 16 would be 6 bytes)
+        constexpr int UW = BITS == 3 ? 32 : 16;
+        constexpr int CWU = UW * BITS / 32;                  // code words per unit
         // scale (halved for the symmetric weight grid) and bias of every output
         // channel, once per CTA; columns past Cout get 0
         for (int c = threadIdx.x - W3_WARP_E0 * 32; c < p.cout_pad; c += W3_NUM_E_WARPS * 32) {
@@ -577,7 +636,7 @@ dsq_win3_kernel(const __grid_constant__ CUtensorMap tmap_b,
             sm_bias[c] = bi;
         }
         named_barrier_sync(1, W3_NUM_E_WARPS * 32);
-        const int units = BN / 16;
+        const int units = BN / UW;
         // this thread's row of the CTA's first tile: image, row, column in the
         // padded stacked numbering (positions in its padding have no output)
         W3Pos pos;
@@ -603,13 +662,15 @@ dsq_win3_kernel(const __grid_constant__ CUtensorMap tmap_b,
             auto fetch_res = [&](int u) {
 #pragma unroll
                 for (int w = 0; w < CWU; ++w) res_nx[w] = 0u;
-                const int byte0 = (n_tile * BN + u * 16) * BITS / 8;
+                const int byte0 = (n_tile * BN + u * UW) * BITS / 8;
                 if (EPI != DSQ_EPI_CODES && e.residual && row_ok && u < units &&
                     byte0 < p.out_pitch) {
                     const uint32_t *rp =
                         reinterpret_cast<const uint32_t *>(e.residual + m * p.out_pitch + byte0);
+                    // (a unit of 3-bit codes may reach past the end of the row)
 #pragma unroll
-                    for (int w = 0; w < CWU; ++w) res_nx[w] = __ldg(rp + w);
+                    for (int w = 0; w < CWU; ++w)
+                        if (BITS != 3 || byte0 + 4 * w < p.out_pitch) res_nx[w] = __ldg(rp + w);
                 }
             };
             fetch_res(k);
@@ -620,18 +681,19 @@ dsq_win3_kernel(const __grid_constant__ CUtensorMap tmap_b,
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + as * BN;
 #pragma unroll 1
             for (int u = k; u < units; u += W3_EPQ) {
-                uint32_t r[16], resw[CWU];
+                uint32_t r[UW], resw[CWU];
 #pragma unroll
                 for (int w = 0; w < CWU; ++w) resw[w] = res_nx[w];
                 __syncwarp();
-                tmem_ld_32x16(taddr + u * 16, r);
+                if constexpr (UW == 32) tmem_ld_32x32(taddr + u * UW, r);
+                else tmem_ld_32x16(taddr + u * UW, r);
                 fetch_res(u + W3_EPQ);
                 tmem_ld_wait();
-                const int n0 = n_tile * BN + u * 16;
+                const int n0 = n_tile * BN + u * UW;
                 const int byte0 = n0 * BITS / 8;
                 if (!row_ok) continue;
                 uint32_t cw[CWU];
-                if (EPI == DSQ_EPI_CODES || EPI == DSQ_EPI_CODES_RES) {
+                if constexpr (BITS != 3 && (EPI == DSQ_EPI_CODES || EPI == DSQ_EPI_CODES_RES)) {
                     if (byte0 >= p.out_pitch) continue;
                     w3_codes_unit<BITS, EPI == DSQ_EPI_CODES_RES>(
                         r, sm_scale + n0, sm_bias + n0, resw, lut, p.shift, e.rq.inv, p.r_hi, cw);
@@ -639,26 +701,33 @@ dsq_win3_kernel(const __grid_constant__ CUtensorMap tmap_b,
                     constexpr uint32_t MASK = (1u << BITS) - 1u;
 #pragma unroll
                     for (int w = 0; w < CWU; ++w) cw[w] = 0u;
-#pragma unroll 4
-                    for (int c = 0; c < 16; ++c) {
+#pragma unroll
+                    for (int c = 0; c < UW; ++c) {
                         const int v = (int)r[c] >> p.shift;
+                        // field c of the unit: word fw, bit fs (a 3-bit field may
+                        // straddle two words; never the last word)
+                        const int fw = (c * BITS) >> 5, fs = (c * BITS) & 31;
+                        const int fw1 = fw + 1 < CWU ? fw + 1 : fw;
                         if (n0 + c < p.Ncols) {
                             if (e.acc_out) e.acc_out[m * p.Ncols + n0 + c] = v;
                             float y = dsq_epi_y(v, sm_scale[n0 + c], sm_bias[n0 + c]);
                             if (e.residual) {
                                 const uint32_t qr =
-                                    (resw[(c * BITS) >> 5] >> ((c * BITS) & 31)) & MASK;
+                                    __funnelshift_r(resw[fw], fw + 1 < CWU ? resw[fw1] : 0u, fs) & MASK;
                                 y = dsq_epi_residual(y, qr, e.res_delta, e.res_lo);
                             }
-                            if (e.has_requant)
-                                cw[(c * BITS) >> 5] |= dsq_code(y, e.rq) << ((c * BITS) & 31);
+                            if (e.has_requant) {
+                                const uint32_t q = dsq_code(y, e.rq);
+                                cw[fw] |= q << fs;
+                                if (BITS == 3 && fs > 29) cw[fw1] |= q >> (32 - fs);
+                            }
                             if (e.y_f32) e.y_f32[m * p.Ncols + n0 + c] = y;
                         }
                     }
                     if (!e.y_codes || byte0 >= p.out_pitch) continue;
                 }
                 // columns past Cout are padding lanes of the packed row: zero
-                const int nvalid_bits = min(16, max(0, p.Ncols - n0)) * BITS;
+                const int nvalid_bits = min(UW, max(0, p.Ncols - n0)) * BITS;
 #pragma unroll
                 for (int w = 0; w < CWU; ++w) {
                     const int nb = nvalid_bits - 32 * w;
@@ -667,7 +736,17 @@ dsq_win3_kernel(const __grid_constant__ CUtensorMap tmap_b,
                 uint32_t *dst = reinterpret_cast<uint32_t *>(e.y_codes + m * p.out_pitch + byte0);
                 if (CWU == 2)
                     *reinterpret_cast<uint2 *>(dst) = make_uint2(cw[0], cw[CWU - 1]);
-                else
+                else if (CWU == 3) {
+                    // 12 bytes, as far as the row goes
+                    dst[0] = cw[0];
+                    if (byte0 + 4 < p.out_pitch) dst[1] = cw[1];
+                    if (byte0 + 8 < p.out_pitch) dst[2] = cw[CWU - 1];
+                    // 3-bit rows: the N tiles may end before the row's pitch does
+                    // (64 columns = 24 bytes, pitch 32); the spare bytes are zero
+                    if (n_tile == p.n_tiles - 1 && u == units - 1)
+                        for (int b = p.cout_pad * BITS / 8; b < p.out_pitch; b += 4)
+                            *reinterpret_cast<uint32_t *>(e.y_codes + m * p.out_pitch + b) = 0u;
+                } else
                     *dst = cw[0];
             }
             tc_fence_before_sync();
@@ -745,7 +824,8 @@ int dsq_conv3_window(const void *act_codes, const dsq_nhwc_t *shape, int bits,
     if (!hooks.window3) return DSQ_ERR_UNSUPPORTED;
     if (conv->KH != 3 || conv->KW != 3 || conv->stride != 1 || conv->pad != 1)
         return DSQ_ERR_UNSUPPORTED;
-    if (bits != 2 && bits != 4) return DSQ_ERR_UNSUPPORTED;
+    if (bits < 2 || bits > 4) return DSQ_ERR_UNSUPPORTED;
+    if (bits == 3) epi_kind = DSQ_EPI_GENERAL;   // the lean codes epilogue packs whole nibbles / pairs
     const int Cin = conv->Cin, Cout = conv->Cout;
     if (!(Cin == 64 || (Cin % 128 == 0 && Cin <= 1024))) return DSQ_ERR_UNSUPPORTED;
     if (shape->W + 2 > 32000 || shape->H + 2 > 32000) return DSQ_ERR_UNSUPPORTED;
@@ -774,12 +854,14 @@ int dsq_conv3_window(const void *act_codes, const dsq_nhwc_t *shape, int bits,
     p.n_tiles = (Cout + p.BN - 1) / p.BN;
     p.Ncols = Cout;
     p.E = Cin;
+    p.two_taps = Cin == 64 && bits != 3;
     p.npl = Cin == 64 ? 1 : Cin / 128;
-    p.kpp = Cin == 64 ? 5 : 9;
+    p.kpp = p.two_taps ? 5 : 9;
     p.ksteps = p.npl * p.kpp;
     const int P = (int)dsq_row_pitch(Cin, bits);           // packed bytes per pixel
     p.PB = Cin == 64 ? P : 16 * bits;
     p.cpp = p.PB / 16;
+    p.xstep = p.two_taps ? 16 * bits : P;
     const int need = W3_BM + 2 + 2 * p.Wp;
     if (need <= W3_MAX_WINDOW_PX) {
         p.nbands = 1;
@@ -887,5 +969,6 @@ int dsq_conv3_window(const void *act_codes, const dsq_nhwc_t *shape, int bits,
             return DSQ_ERR_UNSUPPORTED;
     }
     if (bits == 4) return w3_dispatch<4>(epi_kind, tb, ta, p, stream, hooks.pdl);
+    if (bits == 3) return w3_launch<3, DSQ_EPI_GENERAL>(tb, ta, p, stream, hooks.pdl);
     return w3_dispatch<2>(epi_kind, tb, ta, p, stream, hooks.pdl);
 }

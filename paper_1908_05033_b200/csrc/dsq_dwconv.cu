@@ -13,6 +13,8 @@ template <int BITS>
 __device__ __forceinline__ uint32_t load_unit(const uint8_t *p)
 {
     if (BITS == 4) return __ldg(reinterpret_cast<const uint32_t *>(p));
+    if (BITS == 3)      // 8 codes = 3 bytes at an odd offset: byte loads
+        return (uint32_t)__ldg(p) | ((uint32_t)__ldg(p + 1) << 8) | ((uint32_t)__ldg(p + 2) << 16);
     return __ldg(reinterpret_cast<const uint16_t *>(p));
 }
 
@@ -36,7 +38,7 @@ dwconv3x3_kernel(const uint8_t *__restrict__ act, const uint8_t *__restrict__ wg
     constexpr uint32_t MASK = (1u << BITS) - 1u;
     constexpr int OW = 4;                    // outputs per thread along W
     constexpr int IW = (OW - 1) * STRIDE + 3;
-    const int units = pitch / UB;
+    const int units = BITS == 3 ? (C + 7) / 8 : pitch / UB;
     const int strips = (Wo + OW - 1) / OW;
     const int64_t total = (int64_t)N * Ho * strips * units;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total;
@@ -131,7 +133,13 @@ dwconv3x3_kernel(const uint8_t *__restrict__ act, const uint8_t *__restrict__ wg
                 if (wo0 + o >= Wo) continue;
                 uint8_t *dst = e.y_codes + (pix0 + o) * pitch + u * UB;
                 if (BITS == 4) *reinterpret_cast<uint32_t *>(dst) = cw[o];
-                else *reinterpret_cast<uint16_t *>(dst) = (uint16_t)cw[o];
+                else if (BITS == 3) {
+                    dst[0] = (uint8_t)cw[o]; dst[1] = (uint8_t)(cw[o] >> 8);
+                    dst[2] = (uint8_t)(cw[o] >> 16);
+                    // the row's spare bytes behind the last unit are zero
+                    if (u == units - 1)
+                        for (int b = 3 * units; b < pitch; ++b) dst[b - u * UB] = 0;
+                } else *reinterpret_cast<uint16_t *>(dst) = (uint16_t)cw[o];
             }
         }
     }
@@ -150,7 +158,6 @@ extern "C" int dsq_dwconv2d(const void *act_codes, const dsq_nhwc_t *shape,
     int st = dsq_check_quant(act_q);
     if (st) return st;
     const int bits = act_q->bits;
-    if (bits == 3) return DSQ_ERR_UNSUPPORTED;
     if (shape->N <= 0 || shape->H <= 0 || shape->W <= 0 || shape->C <= 0)
         return DSQ_ERR_SHAPE;
     if (conv->groups != shape->C || conv->Cin != shape->C || conv->Cout != shape->C)
@@ -166,7 +173,8 @@ extern "C" int dsq_dwconv2d(const void *act_codes, const dsq_nhwc_t *shape,
     const int Ho = (shape->H + 2 - 3) / conv->stride + 1;
     const int Wo = (shape->W + 2 - 3) / conv->stride + 1;
     const int pitch = (int)dsq_row_pitch(shape->C, bits);
-    const int64_t total = (int64_t)shape->N * Ho * ((Wo + 3) / 4) * (pitch / bits);
+    const int64_t total = (int64_t)shape->N * Ho * ((Wo + 3) / 4) *
+                          (bits == 3 ? (shape->C + 7) / 8 : pitch / bits);
     int64_t g = (total + 255) / 256;
     if (g > 148 * 32) g = 148 * 32;
     if (g < 1) g = 1;
@@ -177,6 +185,8 @@ extern "C" int dsq_dwconv2d(const void *act_codes, const dsq_nhwc_t *shape,
                                                   Ho, Wo, pitch, e)
     if (bits == 4 && conv->stride == 1) DSQ_DW_LAUNCH(4, 1);
     else if (bits == 4) DSQ_DW_LAUNCH(4, 2);
+    else if (bits == 3 && conv->stride == 1) DSQ_DW_LAUNCH(3, 1);
+    else if (bits == 3) DSQ_DW_LAUNCH(3, 2);
     else if (conv->stride == 1) DSQ_DW_LAUNCH(2, 1);
     else DSQ_DW_LAUNCH(2, 2);
 #undef DSQ_DW_LAUNCH

@@ -164,6 +164,13 @@ struct TcParams {
     //      rows of up to 2 KB instead of one pixel's P bytes (the TMA unit spends
     //      a few cycles per row whatever its length).  a_bw = W*P.
     int a_tma, a_lc, a_nsub, a_kchunks, a_nr, a_bw;
+    // 3-bit convolution: a pixel's packed row (P bytes, 8 codes per 3 bytes
+    // from the row's start) is not a whole number of 48-byte K steps unless
+    // Cin is a multiple of 128, so every filter tap starts a K step of its
+    // own: Pk = P rounded up to 48 bytes, the A gather fills the rest of a
+    // tap's last K step with zeros, and B's K step (tap, s) lies at byte
+    // tap * P + 48 s of a weight row (spt K steps per tap; 0 = dense rows).
+    int Pk, spt;
     // epilogue
     int mode, shift, out_pitch, small_acc;
     DsqEpi e;
@@ -372,7 +379,7 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
         // keep that pipeline busy)
         if (lane == 0) {
             uint32_t g = 0, ph = 0, issued_b = 0;
-            int s = 0, ks = 0, tile = tile0;
+            int s = 0, ks = 0, tile = tile0, btap = 0, bsub = 0;
 #pragma unroll 1
             for (; g < n_b_steps; ++g) {
                 if (!wait_bar(bar_p_empty(s), ph ^ 1u, ctl, 1)) break;
@@ -388,11 +395,12 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
                                     (tile % p.n_tiles) * BN + (int)rank * BNL, bar_p_full(s));
                 } else
                 tma_load_2d(smem_u32(smem + L.b_packed + s * b_packed_bytes), &tmap_b,
-                            ks * (KS * 16 * BITS),
+                            p.spt ? btap * p.P + bsub * (16 * BITS) : ks * (KS * 16 * BITS),
                             (tile % p.n_tiles) * BN + (int)rank * BNL, bar_p_full(s));
                 ++issued_b;
                 if (++s == S_P) { s = 0; ph ^= 1u; }
-                if (++ks == p.rounds) { ks = 0; tile += tstep; }
+                if (p.spt && ++bsub == p.spt) { bsub = 0; ++btap; }
+                if (++ks == p.rounds) { ks = 0; tile += tstep; btap = bsub = 0; }
             }
             // let outstanding copies land before the CTA can exit
             for (uint32_t k = (issued_b > (uint32_t)S_P ? issued_b - S_P : 0); k < issued_b; ++k)
@@ -567,11 +575,13 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
 #pragma unroll
                 for (int j = 0; j < KS * CH; ++j) {
                     if ((j & crm) == 0) {          // a new run starts
-                        const bool ok = tap < 32 && ((tap_mask >> tap) & 1u);
+                        // (chunks past the pixel's P bytes, 3-bit rows only, are zeros)
+                        const bool real = off < p.P;
+                        const bool ok = real && tap < 32 && ((tap_mask >> tap) & 1u);
                         run = ok ? (unsigned long long)reinterpret_cast<uintptr_t>(src) : 0ull;
                         off += 16 << lcr;
-                        src += 16 << lcr;
-                        if (off == p.P) {
+                        if (real) src += 16 << lcr;
+                        if (off == p.Pk) {
                             off = 0;
                             ++tap;
                             if (++kw == p.KW) { kw = 0; src += row_jump; }
@@ -1070,8 +1080,10 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
                     if (e.residual && byte0 < p.out_pitch) {
                         const uint32_t *rp = reinterpret_cast<const uint32_t *>(
                             e.residual + m * p.out_pitch + byte0);
+                        // (a block of 3-bit codes may reach past the end of the row)
 #pragma unroll
-                        for (int w = 0; w < CW; ++w) resw[w] = __ldg(rp + w);
+                        for (int w = 0; w < CW; ++w)
+                            if (BITS != 3 || byte0 + 4 * w < p.out_pitch) resw[w] = __ldg(rp + w);
                     }
                     uint32_t cw[CW];
 #pragma unroll
@@ -1104,14 +1116,20 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
                             float y = 0.f;
                             if (n < p.Ncols) {
                                 y = dsq_epi_y((int)r[c], scs[u], bis[u]);
+                                // field c of the 32-column block: word fw, bit fs (a
+                                // 3-bit field may straddle two words; never the last)
+                                const int fw = (c * BITS) >> 5, fs = (c * BITS) & 31;
+                                const int fw1 = fw + 1 < CW ? fw + 1 : fw;
                                 if (e.residual) {
                                     const uint32_t qr =
-                                        (resw[(c * BITS) >> 5] >> ((c * BITS) & 31)) & MASK;
+                                        __funnelshift_r(resw[fw], fw + 1 < CW ? resw[fw1] : 0u, fs) & MASK;
                                     y = dsq_epi_residual(y, qr, e.res_delta, e.res_lo);
                                 }
-                                if (e.has_requant)
-                                    cw[(c * BITS) >> 5] |= dsq_code(y, e.rq)
-                                                           << ((c * BITS) & 31);
+                                if (e.has_requant) {
+                                    const uint32_t q = dsq_code(y, e.rq);
+                                    cw[fw] |= q << fs;
+                                    if (BITS == 3 && fs > 29) cw[fw1] |= q >> (32 - fs);
+                                }
                             }
                             y4[u] = y;
                         }
@@ -1133,7 +1151,17 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
                         if (CW == 4)
                             *reinterpret_cast<uint4 *>(dst) =
                                 make_uint4(cw[0], cw[1], cw[2], cw[CW - 1]);
-                        else
+                        else if (CW == 3) {
+                            // 12 bytes, as far as the row goes
+                            dst[0] = cw[0];
+                            if (byte0 + 4 < p.out_pitch) dst[1] = cw[1];
+                            if (byte0 + 8 < p.out_pitch) dst[2] = cw[CW - 1];
+                            // 3-bit rows: the N tiles may end before the row's pitch
+                            // does (64 columns = 24 bytes, pitch 32): spare bytes are zero
+                            if (n_tile == p.n_tiles - 1 && c0 + 32 >= BN)
+                                for (int b = p.n_tiles * BN * BITS / 8; b < p.out_pitch; b += 4)
+                                    *reinterpret_cast<uint32_t *>(e.y_codes + m * p.out_pitch + b) = 0u;
+                        } else
                             *reinterpret_cast<uint2 *>(dst) = make_uint2(cw[0], cw[CW - 1]);
                     }
                 }
@@ -1528,6 +1556,9 @@ int dispatch_tc(int bits, int epi, int pm, const TcMaps &tmap, const TcParams &p
     if (bits == 4) return launch_bits<4>(epi, pm, tmap, p, s);
     if (bits == 2) return launch_bits<2>(epi, pm, tmap, p, s);
     if (bits == 3 && epi == EPI_GEMM) return launch_tc<3, true, EPI_GEMM, 1, 0>(tmap, p, s);
+    // 3-bit convolutions: single K steps, rows gathered with cp.async, the
+    // epilogue that handles fields straddling two words
+    if (bits == 3) return launch_tc<3, false, EPI_GENERAL, 1, 0>(tmap, p, s);
     return DSQ_ERR_UNSUPPORTED;
 }
 
@@ -1693,6 +1724,7 @@ int dsq_gemm(const void *A_codes, const void *B_codes, int64_t M, int64_t N, int
     p.act = (const uint8_t *)A_codes;
     p.H = 1; p.W = (int)M; p.Ho = 1; p.Wo = (int)M;
     p.stride = 1; p.pad = 0; p.KW = 1; p.taps = 1; p.P = (int)pitch;
+    p.Pk = p.P;
     p.a_lcr = a_run_log2(p.P, bits, ks);
     p.mode = MODE_GEMM;
     p.shift = 8 - bits;
@@ -1721,7 +1753,6 @@ int dsq_conv2d(const void *act_codes, const dsq_nhwc_t *shape, const dsq_quant_t
     int st = dsq_check_quant(act_q);
     if (st) return st;
     const int bits = act_q->bits;
-    if (bits == 3) return DSQ_ERR_UNSUPPORTED;
     if (shape->N <= 0 || shape->H <= 0 || shape->W <= 0 || shape->C <= 0 || conv->Cout <= 0)
         return DSQ_ERR_SHAPE;
     if (conv->groups != 1 || conv->Cin != shape->C) return DSQ_ERR_SHAPE;
@@ -1761,6 +1792,13 @@ int dsq_conv2d(const void *act_codes, const dsq_nhwc_t *shape, const dsq_quant_t
     p.M = (int)M;
     p.Ncols = conv->Cout;
     p.ksteps = (int)((row_bytes + 16 * bits - 1) / (16 * bits));
+    p.Pk = (int)P;
+    if (bits == 3) {
+        // every tap starts a K step of its own (see TcParams::Pk)
+        p.spt = (int)((P + 47) / 48);
+        p.Pk = p.spt * 48;
+        p.ksteps = taps * p.spt;
+    }
     p.m_tiles = (int)((M + BM - 1) / BM);
     p.BN = pick_bn(p.m_tiles, conv->Cout, bits);
     p.n_tiles = (conv->Cout + p.BN - 1) / p.BN;

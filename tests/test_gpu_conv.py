@@ -77,6 +77,19 @@ def conv_case(dsq, N_, H, W, Ci, Co, k, s, p, bits, w_off, residual=False,
     assert torch.equal(codes, codes2)
 
 
+@pytest.mark.parametrize("bits", [2, 3, 4])
+def test_table8_layer_shapes_at_every_bit_width(dsq, bits):
+    """The four 3x3 layer shapes of the paper's Table 8 (batch 1, stride 1,
+    pad 1) at 4, 3 and 2 bits, every accumulator and code against the oracle."""
+    import os
+    here = os.path.dirname(__file__)
+    for line in open(os.path.join(here, "golden", "table8_shapes.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        ci, h, w, co = map(int, line.split())
+        conv_case(dsq, 1, h, w, ci, co, 3, 1, 1, bits, 0.5, seed=ci)
+
+
 def test_workload_1_single_3x3_conv(dsq):
     """64x56x56 -> 64, 3x3, stride 1, pad 1, 4-bit (Table 8, first row)."""
     c = dsq_inputs.conv3x3_case()
@@ -110,7 +123,7 @@ GEOMS = [  # N, H, W, Cin, Cout, k, stride, pad
     (1, 17, 13, 100, 300, 3, 2, 1), (1, 12, 12, 960, 160, 1, 1, 0)]
 
 
-@pytest.mark.parametrize("bits", [2, 4])
+@pytest.mark.parametrize("bits", [2, 3, 4])
 @pytest.mark.parametrize("w_off", [0.0, 0.5])
 @pytest.mark.parametrize("geom", GEOMS)
 def test_conv_geometries(dsq, geom, bits, w_off):
@@ -128,7 +141,7 @@ def test_conv_whole_k_rounds(dsq, geom, bits):
     conv_case(dsq, n, h, w, 64, 64, 3, 1, 1, bits, 0.5, residual=(n == 6), seed=n + h)
 
 
-@pytest.mark.parametrize("bits", [2, 4])
+@pytest.mark.parametrize("bits", [2, 3, 4])
 def test_conv_residual_and_per_channel(dsq, bits):
     conv_case(dsq, 2, 14, 14, 64, 64, 3, 1, 1, bits, 0.5, residual=True)
     conv_case(dsq, 1, 10, 10, 48, 200, 1, 1, 0, bits, 0.5, residual=True,
@@ -137,7 +150,7 @@ def test_conv_residual_and_per_channel(dsq, bits):
               per_channel=True, out_rng=(-1.0, 1.0))
 
 
-@pytest.mark.parametrize("bits", [2, 4])
+@pytest.mark.parametrize("bits", [2, 3, 4])
 def test_conv_extreme_codes(dsq, bits):
     """All activations at the top code, all weights at the bottom code."""
     half = 1 << (bits - 1)
@@ -191,7 +204,7 @@ def dw_case(dsq, N_, H, W, Cc, s, bits, w_off, residual=False, seed=6):
     assert np.array_equal(N(codes).reshape(ref_codes.shape), ref_codes)
 
 
-@pytest.mark.parametrize("bits", [2, 4])
+@pytest.mark.parametrize("bits", [2, 3, 4])
 @pytest.mark.parametrize("w_off", [0.0, 0.5])
 @pytest.mark.parametrize("geom", [(1, 8, 8, 32, 1), (2, 9, 7, 144, 2),
                                   (1, 12, 12, 96, 1), (1, 3, 3, 20, 2),
@@ -209,7 +222,7 @@ WINDOW_GEOMS = [  # N, H, W, Cin, Cout: 3x3, stride 1, pad 1 on the shared-memor
     (1, 6, 300, 128, 72), (2, 56, 56, 128, 128), (70, 5, 5, 64, 96)]
 
 
-@pytest.mark.parametrize("bits", [2, 4])
+@pytest.mark.parametrize("bits", [2, 3, 4])
 @pytest.mark.parametrize("geom", WINDOW_GEOMS)
 def test_conv3x3_window_kernel(dsq, geom, bits):
     """3x3 stride-1 convolutions whose A operand is an expanded window of the
@@ -227,7 +240,7 @@ def test_conv3x3_window_kernel(dsq, geom, bits):
         dsq.dsq_set_conv3_window(1)
 
 
-@pytest.mark.parametrize("bits", [2, 4])
+@pytest.mark.parametrize("bits", [2, 3, 4])
 def test_conv3x3_window_and_im2col_kernels_agree(dsq, bits):
     """The same convolution through both tensor-core kernels (hook) gives the
     same codes; both are compared with the oracle elsewhere."""

@@ -49,7 +49,7 @@ def assert_not_degenerate(st, ref):
         assert len(np.unique(ref[name])) >= min(4, 2 ** st.bits), name
 
 
-@pytest.mark.parametrize("bits", [2, 4])
+@pytest.mark.parametrize("bits", [2, 3, 4])
 @pytest.mark.parametrize("w_offset", [0.0, 0.5])
 def test_tiny_stack_every_layer(dsq, bits, w_offset):
     st = dsq_inputs.tiny_stack(bits=bits)
@@ -97,6 +97,16 @@ def test_resnet18_stack_graph_replay_matches_eager(dsq):
 
 def test_resnet18_stack_batch1_every_layer(dsq):
     st = dsq_inputs.resnet18_stack()
+    _, ref = compare_stack(st, 3, 1)
+    assert_not_degenerate(st, ref)
+
+
+def test_resnet18_stack_3bit_batch1_every_layer(dsq):
+    """The ResNet-18-shaped stack at 3 bits (the paper's Table 8 times 3-bit
+    convolutions on its layer shapes): 3x3 stride-1 layers on the window
+    kernel or the im2col kernel, strided and 1x1 layers on the im2col kernel
+    with one K step group per filter tap."""
+    st = dsq_inputs.resnet18_stack(bits=3)
     _, ref = compare_stack(st, 3, 1)
     assert_not_degenerate(st, ref)
 

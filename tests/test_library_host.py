@@ -102,7 +102,7 @@ def test_validation_status_codes_without_a_gpu():
     assert call(conv=B.dsq_conv_t(64, 3, 3, 64, 3, 1, 1)) == -8
     assert call(conv=B.dsq_conv_t(64, 3, 3, 32, 1, 1, 1)) == -4
     assert call(q=B.dsq_quant_t(4, -1.0, 2.0)) == -8
-    assert call(q=B.dsq_quant_t(3, 0.0, 2.0)) == -8
+    assert call(q=B.dsq_quant_t(5, 0.0, 2.0)) == -3
     ep2 = B.dsq_epilogue_t()
     ep2.scale, ep2.bias, ep2.w_offset = 0x2000, 0x3000, 0.25
     assert call(ep=ep2) == -8
