@@ -92,11 +92,17 @@ typedef struct dsq_conv_t {
  *                    in-image filter taps.  This is the paper's weight grid
  *                    l_w + Delta_w*q_w with a symmetric clip l_w = -u_w, for
  *                    which w^ = Delta_w * (c + 1/2); scale = Delta_a*Delta_w.
+ *   any other w_offset o_w (the clip bounds l_w, u_w are learnt separately,
+ *                    Sec. 3.4, so in general o_w = l_w/Delta_w + 2^(b-1)):
+ *                    y = fmaf(fmaf(o_w, (float)S_a, (float)acc), scale[co], bias[co]).
+ *                    S_a is summed from the input codes by the epilogue (one
+ *                    extra read of the filter window per output pixel): slower
+ *                    than the two forms above.
  *   residual_codes : y = y + fmaf((float)q_r, Delta_r, l_r), q_r the unsigned
  *                    code at the same output position (packed NHWC, same
  *                    shape as the output), (l_r, Delta_r) from residual_q
  *   requant.bits>0 : codes = quantise(y; requant)  (ReLU is the clip at lo=0)
- * Other w_offset values return DSQ_ERR_UNSUPPORTED. */
+ * A non-finite w_offset returns DSQ_ERR_RANGE. */
 typedef struct dsq_epilogue_t {
     const float *scale;          /* [Cout], required */
     const float *bias;           /* [Cout], required */

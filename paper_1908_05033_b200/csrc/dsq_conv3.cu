@@ -109,6 +109,8 @@ struct W3Params {
     float r_hi;                        // fmaf(hi - lo, inv, 0.5f) of the requantiser
     DsqEpi e;
     uint32_t orv;
+    const uint8_t *act;                // input codes and pixel pitch (general weight offset: S_a)
+    int P;
     int *ws;
 };
 
@@ -653,6 +655,11 @@ dsq_win3_kernel(const __grid_constant__ CUtensorMap tmap_b,
             const int as = it & 1;
             const bool row_ok = pos.n < p.N && pos.h < p.H && pos.w < p.W;
             const int64_t m = ((int64_t)pos.n * p.H + pos.h) * p.W + pos.w;
+            // general weight-grid offset: S_a of this output pixel, summed from
+            // the input codes under its 3 x 3 window
+            int s_a = 0;
+            if (EPI == DSQ_EPI_GENERAL && e.general_offset && row_ok)
+                s_a = dsq_window_sa<BITS>(p.act, pos.n, pos.h, pos.w, p.H, p.W, 3, 1, 1, p.P);
             pos = w3_add(pos, p.t_dn, p.t_dh, p.t_dw, p.Hp, p.Wp);
             // residual codes of a unit of this row are fetched one unit ahead (the
             // first unit's while the tile's instructions are still running); the
@@ -710,7 +717,10 @@ dsq_win3_kernel(const __grid_constant__ CUtensorMap tmap_b,
                         const int fw1 = fw + 1 < CWU ? fw + 1 : fw;
                         if (n0 + c < p.Ncols) {
                             if (e.acc_out) e.acc_out[m * p.Ncols + n0 + c] = v;
-                            float y = dsq_epi_y(v, sm_scale[n0 + c], sm_bias[n0 + c]);
+                            float y = e.general_offset
+                                          ? dsq_epi_y_offset(v, s_a, e.w_offset, sm_scale[n0 + c],
+                                                             sm_bias[n0 + c])
+                                          : dsq_epi_y(v, sm_scale[n0 + c], sm_bias[n0 + c]);
                             if (e.residual) {
                                 const uint32_t qr =
                                     __funnelshift_r(resw[fw], fw + 1 < CWU ? resw[fw1] : 0u, fs) & MASK;
@@ -826,6 +836,7 @@ int dsq_conv3_window(const void *act_codes, const dsq_nhwc_t *shape, int bits,
         return DSQ_ERR_UNSUPPORTED;
     if (bits < 2 || bits > 4) return DSQ_ERR_UNSUPPORTED;
     if (bits == 3) epi_kind = DSQ_EPI_GENERAL;   // the lean codes epilogue packs whole nibbles / pairs
+    if (e.general_offset) epi_kind = DSQ_EPI_GENERAL;
     const int Cin = conv->Cin, Cout = conv->Cout;
     if (!(Cin == 64 || (Cin % 128 == 0 && Cin <= 1024))) return DSQ_ERR_UNSUPPORTED;
     if (shape->W + 2 > 32000 || shape->H + 2 > 32000) return DSQ_ERR_UNSUPPORTED;
@@ -935,6 +946,8 @@ int dsq_conv3_window(const void *act_codes, const dsq_nhwc_t *shape, int bits,
         p.orv = 0;
     }
     p.ws = (int *)workspace;
+    p.act = (const uint8_t *)act_codes;
+    p.P = P;
 
     // weights: Cout rows of 9 taps x P bytes; one box = BN rows x one K step
     DsqEncodeTiledFn enc = dsq_encode_tiled_fn();

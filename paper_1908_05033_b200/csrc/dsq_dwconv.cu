@@ -87,9 +87,9 @@ dwconv3x3_kernel(const uint8_t *__restrict__ act, const uint8_t *__restrict__ wg
                 const int c = ((int)(wv[k] << (32 - BITS * (f + 1)))) >> (32 - BITS);
                 wq[k] = e.half_offset ? 2 * c + 1 : c;
             }
-            int acc[OW];
+            int acc[OW], sa[OW];
 #pragma unroll
-            for (int o = 0; o < OW; ++o) acc[o] = 0;
+            for (int o = 0; o < OW; ++o) acc[o] = sa[o] = 0;
 #pragma unroll
             for (int r = 0; r < 3; ++r) {
                 int q[IW];
@@ -98,7 +98,10 @@ dwconv3x3_kernel(const uint8_t *__restrict__ act, const uint8_t *__restrict__ wg
 #pragma unroll
                 for (int o = 0; o < OW; ++o)
 #pragma unroll
-                    for (int kw = 0; kw < 3; ++kw) acc[o] += q[o * STRIDE + kw] * wq[r * 3 + kw];
+                    for (int kw = 0; kw < 3; ++kw) {
+                        acc[o] += q[o * STRIDE + kw] * wq[r * 3 + kw];
+                        sa[o] += q[o * STRIDE + kw];      // (dead unless the offset is general)
+                    }
             }
             float sc = __ldg(e.scale + ch);
             if (e.half_offset) sc = __fmul_rn(sc, 0.5f);
@@ -109,6 +112,9 @@ dwconv3x3_kernel(const uint8_t *__restrict__ act, const uint8_t *__restrict__ wg
                 // |acc| <= 9*15*17: the 1.5*2^23 bias trick converts exactly
                 const float vf = __fsub_rn(__int_as_float(0x4B400000 + acc[o]), 12582912.0f);
                 float y = __fmaf_rn(vf, sc, bi);
+                // general weight-grid offset: per-channel S_a (taps outside the
+                // image were loaded as code 0)
+                if (e.general_offset) y = dsq_epi_y_offset(acc[o], sa[o], e.w_offset, sc, bi);
                 if (e.residual) {
                     const uint32_t qr = (res[o] >> (BITS * f)) & MASK;
                     y = __fadd_rn(y, __fmaf_rn(__fsub_rn(__int_as_float(0x4B000000 | qr),

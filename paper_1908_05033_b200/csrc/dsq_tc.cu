@@ -919,6 +919,14 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + as * BN;
             float rs = 0.f;
             if (EPI == EPI_GEMM && p.row_scale && row_ok) rs = __ldg(p.row_scale + m);
+            // general weight-grid offset: S_a of this output pixel, summed from
+            // the input codes under its filter window
+            int s_a = 0;
+            if (EPI == EPI_GENERAL && p.e.general_offset && row_ok) {
+                const int wo = (int)(m % p.Wo), t = (int)(m / p.Wo);
+                s_a = dsq_window_sa<BITS>(p.act, t / p.Ho, t % p.Ho, wo, p.H, p.W, p.KW, p.stride,
+                                          p.pad, p.P);
+            }
             // per-warp staging of the chunk's 32 scale / bias values: lane i fetches
             // column i (prefetched one chunk ahead), the warp reads them back as
             // broadcast 128-bit shared loads
@@ -1115,7 +1123,9 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
                             const int n = n0 + c;
                             float y = 0.f;
                             if (n < p.Ncols) {
-                                y = dsq_epi_y((int)r[c], scs[u], bis[u]);
+                                y = e.general_offset
+                                        ? dsq_epi_y_offset((int)r[c], s_a, e.w_offset, scs[u], bis[u])
+                                        : dsq_epi_y((int)r[c], scs[u], bis[u]);
                                 // field c of the 32-column block: word fw, bit fs (a
                                 // 3-bit field may straddle two words; never the last)
                                 const int fw = (c * BITS) >> 5, fs = (c * BITS) & 31;
@@ -1779,8 +1789,9 @@ int dsq_conv2d(const void *act_codes, const dsq_nhwc_t *shape, const dsq_quant_t
     // float through the 1.5 * 2^23 bias trick, which is exact there
     const int small_acc = (double)taps * conv->Cin * (double)((1 << bits) - 1) *
                               (2.0 * (double)(1 << (bits - 1)) + 1.0) < 4194304.0;
-    const int epi = (y_f32 || acc_out || !y_codes) ? EPI_GENERAL
-                    : (e.residual ? EPI_CODES_RES : EPI_CODES);
+    const int epi = (y_f32 || acc_out || !y_codes || e.general_offset)
+                        ? EPI_GENERAL
+                        : (e.residual ? EPI_CODES_RES : EPI_CODES);
     // 3x3 stride-1 convolutions: every input pixel expanded once (dsq_conv3.cu)
     st = dsq_conv3_window(act_codes, shape, bits, w_packed, conv, e, epi, small_acc, workspace,
                           (cudaStream_t)stream);

@@ -65,7 +65,7 @@ def conv_case(dsq, N_, H, W, Ci, Co, k, s, p, bits, w_off, residual=False,
         ws, w_offset=w_off, residual=res_t, residual_q=res_q,
         requant=(bits,) + out_rng, want_f32=True, want_acc=True)
     assert dsq.dsq_workspace_status(ws) == 0
-    want_acc = 2 * acc + sa[..., None] if w_off else acc
+    want_acc = 2 * acc + sa[..., None] if w_off == 0.5 else acc
     assert np.array_equal(N(accg), want_acc)
     assert_f32_close(N(yg), y)
     assert np.array_equal(N(codes).reshape(ref_codes.shape), ref_codes)
@@ -198,7 +198,7 @@ def dw_case(dsq, N_, H, W, Cc, s, bits, w_off, residual=False, seed=6):
         act, (N_, H, W, Cc), (bits, 0.0, 6.0), blob, conv, T(scale), T(bias),
         w_offset=w_off, residual=res_t, residual_q=res_q,
         requant=(bits, 0.0, 6.0), want_f32=True, want_acc=True)
-    want_acc = 2 * acc + sa if w_off else acc
+    want_acc = 2 * acc + sa if w_off == 0.5 else acc
     assert np.array_equal(N(accg), want_acc)
     assert_f32_close(N(yg), y)
     assert np.array_equal(N(codes).reshape(ref_codes.shape), ref_codes)
@@ -258,3 +258,19 @@ def test_conv3x3_window_and_im2col_kernels_agree(dsq, bits):
         dsq.dsq_set_conv3_window(1)
     assert dsq.dsq_workspace_status(ws) == 0
     assert torch.equal(a, b)
+
+
+@pytest.mark.parametrize("bits", [2, 3, 4])
+@pytest.mark.parametrize("w_off", [0.3, -1.25, 2.0])
+def test_general_weight_offset(dsq, bits, w_off):
+    """Asymmetric learnt weight clips (Sec. 3.4: l_w and u_w are learnt
+    separately) give a weight grid l_w + Delta_w q_w whose offset from the signed
+    storage, o_w = l_w/Delta_w + 2^(b-1), is neither 0 nor 1/2: the epilogue then
+    needs S_a next to the accumulator.  Dense convolutions on both tensor-core
+    kernels and depthwise, against the oracle's general branch."""
+    for geom in [(2, 9, 7, 64, 40, 3, 1, 1), (1, 12, 12, 128, 72, 3, 1, 1),
+                 (2, 14, 14, 64, 128, 1, 2, 0), (1, 17, 13, 128, 300, 3, 2, 1),
+                 (1, 12, 12, 960, 160, 1, 1, 0)]:
+        conv_case(dsq, *geom, bits, w_off, residual=(geom[0] == 2), seed=geom[3])
+    dw_case(dsq, 2, 9, 7, 144, 2, bits, w_off)
+    dw_case(dsq, 1, 12, 12, 96, 1, bits, w_off, residual=True)

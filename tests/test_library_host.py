@@ -104,8 +104,8 @@ def test_validation_status_codes_without_a_gpu():
     assert call(q=B.dsq_quant_t(4, -1.0, 2.0)) == -8
     assert call(q=B.dsq_quant_t(5, 0.0, 2.0)) == -3
     ep2 = B.dsq_epilogue_t()
-    ep2.scale, ep2.bias, ep2.w_offset = 0x2000, 0x3000, 0.25
-    assert call(ep=ep2) == -8
+    ep2.scale, ep2.bias, ep2.w_offset = 0x2000, 0x3000, float("nan")
+    assert call(ep=ep2) == -6
     ep3 = B.dsq_epilogue_t()
     assert call(ep=ep3) == -1            # scale / bias missing
     # code output requested but no requantiser given
