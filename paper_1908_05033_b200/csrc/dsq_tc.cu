@@ -173,6 +173,7 @@ struct TcParams {
     int Pk, spt;
     // epilogue
     int mode, shift, out_pitch, small_acc;
+    float r_hi;                       // fmaf(hi - lo, inv, 0.5f) of the requantiser
     DsqEpi e;
     int32_t *C_i32;
     const float *row_scale;
@@ -185,7 +186,7 @@ struct TcParams {
 // the kernel
 // ---------------------------------------------------------------------------
 struct SmemLayout {
-    uint32_t b_tiles, b_packed, a_ring, epi, bars, tmem_slot, abort_flag, total;
+    uint32_t b_tiles, b_packed, a_ring, epi, lut, bars, tmem_slot, abort_flag, total;
 };
 
 constexpr int MAX_S_P = 4;
@@ -209,6 +210,7 @@ __host__ __device__ inline SmemLayout smem_layout(int BN, int bits, int s_p, int
     L.a_ring = o;   o += a_slots * ks * BM * 16 * bits;
     // per-warp scale / bias staging (any warp may take part in an epilogue)
     L.epi = o;      o += epi_slots * 64 * 4;
+    L.lut = o;      o += 16 * 4;             // dequantised residual values (codes epilogue)
     o = (o + 127u) & ~127u;
     L.bars = o;     o += 8 * (2 * SU_MAX + MAX_B_STAGES + 2 * MAX_S_P + 4 + 2 * MAX_A_SLOTS + 2);
     L.tmem_slot = o; o += 8;
@@ -351,6 +353,10 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
         tma_prefetch_desc(&tmap_b);
         if (A_TMA) tma_prefetch_desc(&tmap_a);
     }
+    // the 2^BITS dequantised values of a residual code
+    if (EPI == EPI_CODES_RES && warp == WARP_TMA_A && lane < (1 << BITS))
+        reinterpret_cast<float *>(smem + L.lut)[lane] =
+            __fmaf_rn((float)lane, p.e.res_delta, p.e.res_lo);
     tc_fence_before_sync();
     __syncthreads();
     // no arrival may reach the peer before its barriers exist
@@ -957,8 +963,10 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
                 tmem_ld_wait();
                 const int n0 = n_tile * BN + c0;
                 if (!row_ok) continue;
+                if (EPI == EPI_GEMM || EPI == EPI_GENERAL) {
 #pragma unroll
-                for (int c = 0; c < 32; ++c) r[c] = (uint32_t)((int)r[c] >> p.shift);
+                    for (int c = 0; c < 32; ++c) r[c] = (uint32_t)((int)r[c] >> p.shift);
+                }
                 const bool full = n0 + 32 <= p.Ncols && (p.Ncols & 3) == 0;
                 if (EPI == EPI_GEMM) {
                     if (n0 >= p.Ncols) continue;
@@ -1012,10 +1020,17 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
                         }
                     }
                 } else if (EPI == EPI_CODES || EPI == EPI_CODES_RES) {
-                    // codes-only convolution epilogue (the form the stacks use):
-                    // four columns at a time, their scale / bias vectors fetched
-                    // one group ahead; exact int->float and floor are taken with
-                    // the 2^23 bias trick so the conversion unit stays idle
+                    // codes-only convolution epilogue (the form the stacks use).
+                    // Per element, bit-identical to the pinned sequence:
+                    //   v  = raw >> shift; vf = (float)v (1.5 * 2^23 trick where the
+                    //        accumulator is below 2^22)
+                    //   y  = fma(vf, scale, bias) (+ lut[q_r]: lut[q] = fma(q, Delta_r, l_r))
+                    //   r  = min(fma(max(y, lo) - lo, inv, 0.5), r_hi)
+                    // (clipping y at hi first, or r at r_hi = fma(hi - lo, inv, 0.5)
+                    // afterwards, gives the same r: fma is monotone; floor(r) <= qmax
+                    // because floor(r_hi) = qmax, checked by the host).  The bits of
+                    // r + 2^23 rounded down are 0x4B000000 + floor(r): the codes are
+                    // summed into their fields, the constant leaves once per word.
                     const DsqEpi &e = p.e;
                     constexpr uint32_t MASK = (1u << BITS) - 1u;
                     constexpr int CW = BITS;                 // code words per 32 columns
@@ -1033,6 +1048,7 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
                     uint32_t cw[CW];
 #pragma unroll
                     for (int w = 0; w < CW; ++w) cw[w] = 0u;
+                    const float *lut = reinterpret_cast<const float *>(smem + L.lut);
                     const float4 *sc4 = reinterpret_cast<const float4 *>(epi_scale);
                     const float4 *bi4 = reinterpret_cast<const float4 *>(epi_bias);
                     float4 s_nx = sc4[0], b_nx = bi4[0];
@@ -1045,24 +1061,27 @@ dsq_tc_kernel(const __grid_constant__ CUtensorMap tmap_b,
 #pragma unroll
                         for (int u = 0; u < 4; ++u) {
                             const int c = 4 * v + u;
+                            const int vi = (int)r[c] >> p.shift;
                             const float vf = p.small_acc
-                                ? __fsub_rn(__int_as_float(0x4B400000 + (int)r[c]), 12582912.0f)
-                                : (float)(int)r[c];
+                                ? __fsub_rn(__int_as_float(0x4B400000 + vi), 12582912.0f)
+                                : (float)vi;
                             float y = __fmaf_rn(vf, scs[u], bis[u]);
                             if (EPI == EPI_CODES_RES) {
                                 const uint32_t qr =
                                     (resw[(c * BITS) >> 5] >> ((c * BITS) & 31)) & MASK;
-                                const float qf =
-                                    __fsub_rn(__int_as_float(0x4B000000 | qr), 8388608.0f);
-                                y = __fadd_rn(y, __fmaf_rn(qf, e.res_delta, e.res_lo));
+                                y = __fadd_rn(y, lut[qr]);
                             }
-                            const float xc = fminf(fmaxf(y, e.rq.lo), e.rq.hi);
-                            const float rr = __fmaf_rn(__fsub_rn(xc, e.rq.lo), e.rq.inv, 0.5f);
-                            const uint32_t q =
-                                min((uint32_t)__float_as_int(__fadd_rd(rr, 8388608.0f)) - 0x4B000000u,
-                                    (uint32_t)e.rq.qmax);
-                            cw[(c * BITS) >> 5] |= q << ((c * BITS) & 31);
+                            const float d = __fsub_rn(fmaxf(y, e.rq.lo), e.rq.lo);
+                            const float rr = fminf(__fmaf_rn(d, e.rq.inv, 0.5f), p.r_hi);
+                            cw[(c * BITS) >> 5] +=
+                                (uint32_t)__float_as_int(__fadd_rd(rr, 8388608.0f)) << ((c * BITS) & 31);
                         }
+                    }
+                    {
+                        // 0x4B000000 summed over the fields of a word (mod 2^32)
+                        constexpr uint32_t FIELDS = BITS == 4 ? 0x11111111u : 0x55555555u;
+#pragma unroll
+                        for (int w = 0; w < CW; ++w) cw[w] -= 0x4B000000u * FIELDS;
                     }
                     // columns past Cout are padding lanes of the packed row: zero
                     const int nvalid_bits = min(32, max(0, p.Ncols - n0)) * BITS;
@@ -1843,7 +1862,14 @@ int dsq_conv2d(const void *act_codes, const dsq_nhwc_t *shape, const dsq_quant_t
     st = setup_a_tma(&p, &tmap.a, act_codes, M, bits, ks, plain_rows, shape, conv->KH, pm == 5);
     if (st) return st;
     p.small_acc = small_acc;
-    return dispatch_tc(bits, epi, pm, tmap, p, (cudaStream_t)stream);
+    int epi_im2col = epi;
+    if (epi != EPI_GENERAL) {
+        // the codes epilogue clips after the requantiser's multiply: it needs
+        // floor(fma(hi - lo, inv, 0.5)) = qmax (true for every sane range)
+        p.r_hi = fmaf(e.rq.hi - e.rq.lo, e.rq.inv, 0.5f);
+        if ((int)floorf(p.r_hi) != e.rq.qmax) epi_im2col = EPI_GENERAL;
+    }
+    return dispatch_tc(bits, epi_im2col, pm, tmap, p, (cudaStream_t)stream);
 }
 
 int dsq_probe_i8_mma_rate(int iters, float *ms_out, double *macs_out, void *workspace,
