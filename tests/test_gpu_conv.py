@@ -202,13 +202,19 @@ def dw_case(dsq, N_, H, W, Cc, s, bits, w_off, residual=False, seed=6):
     assert np.array_equal(N(accg), want_acc)
     assert_f32_close(N(yg), y)
     assert np.array_equal(N(codes).reshape(ref_codes.shape), ref_codes)
+    # codes-only call (the form the stacks use; 4-bit takes the dp4a kernel)
+    codes2, _, _ = dsq.dsq_dwconv2d(
+        act, (N_, H, W, Cc), (bits, 0.0, 6.0), blob, conv, T(scale), T(bias),
+        w_offset=w_off, residual=res_t, residual_q=res_q, requant=(bits, 0.0, 6.0))
+    assert torch.equal(codes, codes2)
 
 
 @pytest.mark.parametrize("bits", [2, 3, 4])
 @pytest.mark.parametrize("w_off", [0.0, 0.5])
 @pytest.mark.parametrize("geom", [(1, 8, 8, 32, 1), (2, 9, 7, 144, 2),
                                   (1, 12, 12, 96, 1), (1, 3, 3, 20, 2),
-                                  (2, 28, 28, 192, 2), (1, 1, 1, 8, 1)])
+                                  (2, 28, 28, 192, 2), (1, 1, 1, 8, 1),
+                                  (3, 57, 61, 96, 1), (2, 30, 31, 40, 2), (1, 5, 2, 960, 1)])
 def test_depthwise(dsq, geom, bits, w_off):
     dw_case(dsq, *geom, bits, w_off)
     if geom[4] == 1:
