@@ -97,9 +97,12 @@ struct W3Params {
     int tap_stride;                    // slot rows between two filter rows
     int as_slots, bp_slots, b_stages, b_res;
     int cout_pad;                      // Cout rounded up to the N tiling
+    int tr;                            // transposed tiles (kernel form TR)
     int mstep;                         // M tiles between two tiles of a CTA
     int t_dn, t_dh, t_dw;              // mstep * 128 positions as images, padded rows, columns
-    int ld_dh[3], ld_dw[3];            // start of every load of a fill, from the tile's start
+    // start of every load of a fill, from the tile's start: images, padded rows
+    // (< Hp), padded columns (< Wp)
+    int ld_dn[3], ld_dh[3], ld_dw[3];
     int smem_bytes;
     unsigned long long wait_ns;
     int skip_b_round;
@@ -205,13 +208,39 @@ __device__ __forceinline__ W3Pos w3_add(W3Pos a, int dn, int dh, int dw, int Hp,
     return a;
 }
 
-template <int BITS, int EPI>
+// Transposed tiles (template parameter TR).  An instruction whose A operand
+// comes through a shared-memory descriptor takes ~130 clocks whatever its N, so
+// it should carry N = 256.  With the roles swapped - A = 128 weight rows of the K
+// step, B = 256 rows of the window - every instruction is 128 x 256 x 32 even
+// for 64 or 128 output channels.  The accumulator then has output CHANNELS on
+// the tensor-memory lanes and POSITIONS in the columns: an epilogue thread owns
+// one channel, gathers its codes of 8 (16 at 2 bits) positions in a word and an
+// 8 x 8 (16 x 16) transpose of bit fields across the lanes of a channel group
+// (shuffles) turns that into the packed NHWC words of those positions.
+template <int BITS>
+__device__ __forceinline__ uint32_t w3_transpose_fields(uint32_t x, int lane)
+{
+    constexpr int E = 32 / BITS;                 // fields per word = lanes per group
+#pragma unroll
+    for (int d = E / 2; d >= 1; d >>= 1) {
+        const int block = BITS * d;
+        const uint32_t M = block == 16 ? 0x0000FFFFu : block == 8 ? 0x00FF00FFu
+                           : block == 4 ? 0x0F0F0F0Fu : 0x33333333u;
+        const uint32_t px = __shfl_xor_sync(0xffffffffu, x, d);
+        x = (lane & d) ? (((px >> block) & M) | (x & ~M)) : ((x & M) | ((px << block) & ~M));
+    }
+    return x;
+}
+
+template <int BITS, int EPI, bool TR>
 __global__ void __launch_bounds__(W3_THREADS, 1)
 dsq_win3_kernel(const __grid_constant__ CUtensorMap tmap_b,
                 const __grid_constant__ CUtensorMap tmap_a, const W3Params p)
 {
     constexpr int CH = Chunks<BITS>::CH;       // packed 16-byte chunks per 128 codes
     constexpr int OUT = Chunks<BITS>::OUT;     // int8 chunks per packed chunk
+    constexpr int TP = TR ? 256 : W3_BM;       // positions of a tile
+    static_assert(!TR || BITS != 3, "transposed tiles: 2- and 4-bit codes");
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>(
         (reinterpret_cast<uintptr_t>(smem_raw) + 1023u) & ~(uintptr_t)1023u);
@@ -356,7 +385,7 @@ dsq_win3_kernel(const __grid_constant__ CUtensorMap tmap_b,
             // first position of the CTA's first tile (the only division)
             W3Pos base;
             {
-                const int g0 = m_first * W3_BM;
+                const int g0 = m_first * TP;
                 base.n = g0 / img_positions;
                 const int rem = g0 - base.n * img_positions;
                 base.h = rem / p.Wp;
@@ -369,12 +398,23 @@ dsq_win3_kernel(const __grid_constant__ CUtensorMap tmap_b,
                 // output reads: they are left out (and not counted)
                 int nl = 0;
                 for (int i = 0; i < nld; ++i)
-                    nl += w3_add(base, 0, p.ld_dh[i], p.ld_dw[i], p.Hp, p.Wp).n < p.N;
+                    nl += w3_add(base, p.ld_dn[i], p.ld_dh[i], p.ld_dw[i], p.Hp, p.Wp).n < p.N;
                 mbar_arrive_expect_tx(bar_as_full(s), (uint32_t)(nl * p.a_box * p.PB));
                 const uint32_t dst0 = smem_u32(smem + L.a_stage) + s * a_stage_bytes;
                 for (int i = 0; i < nld; ++i) {
-                    const W3Pos q = w3_add(base, 0, p.ld_dh[i], p.ld_dw[i], p.Hp, p.Wp);
+                    // (start coordinates always lie inside the map's bounding box:
+                    // 0 <= q.h < Hp, 0 <= q.w < Wp, q.n < N)
+                    const W3Pos q = w3_add(base, p.ld_dn[i], p.ld_dh[i], p.ld_dw[i], p.Hp, p.Wp);
                     if (q.n >= p.N) continue;
+                    // an im2col load must start inside the map's bounding box: a
+                    // position outside it is never issued (the roles then run into
+                    // their wait limit and the kernel reports the failure)
+                    if (q.n < 0 || q.h < 0 || q.h >= p.Hp || q.w < 0 || q.w >= p.Wp) {
+                        if (atomicCAS(p.ws + DSQ_WS_STATUS, 0, (int)DSQ_ERR_SHAPE) == 0)
+                            p.ws[DSQ_WS_DETAIL] = 16;
+                        *ctl.abort_flag = 1;
+                        continue;
+                    }
                     // bounding box = image grown by one pixel: base positions
                     // -2 .. W-1 / -2 .. H-1, filter offset (1, 1)
                     tma_load_im2col_4d(dst0 + (uint32_t)(i * p.a_box * p.PB), &tmap_a, pl * p.PB,
@@ -394,7 +434,8 @@ dsq_win3_kernel(const __grid_constant__ CUtensorMap tmap_b,
         }
     } else if (warp == W3_WARP_MMA) {
         // ---------------- MMA issuer (whole warp, uniform; one lane issues) --------
-        const uint32_t idesc = idesc_i8(BN, false, true, W3_BM);
+        // (TR: A = 128 weight rows, signed; B = 256 window rows, unsigned)
+        const uint32_t idesc = TR ? idesc_i8(256, true, false, 128) : idesc_i8(BN, false, true, W3_BM);
         const uint64_t desc0 = smem_desc_sw128(0u);
         const uint32_t desc_hi = (uint32_t)(desc0 >> 32), desc_lo = (uint32_t)desc0;
         const uint32_t a_lo_base = desc_lo + (smem_u32(smem + L.a_slots) >> 4);
@@ -410,7 +451,7 @@ dsq_win3_kernel(const __grid_constant__ CUtensorMap tmap_b,
             if (!(ok = wait_bar_warp(bar_acc_empty(as), ((it >> 1) & 1) ^ 1u, ctl, 3))) break;
             W3_STAMP(4, it);
             tc_fence_after_sync();
-            const uint32_t d_tmem = tmem_base + as * BN;
+            const uint32_t d_tmem = tmem_base + as * (TR ? 256 : BN);
             uint32_t first = 0u;                    // 0: the tile's first instruction overwrites
 #pragma unroll 1
             for (int pl = 0; ok && pl < p.npl; ++pl) {
@@ -428,6 +469,13 @@ dsq_win3_kernel(const __grid_constant__ CUtensorMap tmap_b,
                     }
                     // (a slot lies below 256 KB, so the sums stay inside the
                     // 14-bit address field; 0xFFFFFFFF marks no instruction)
+                    if (TR)
+                        mma_i8_ss_x4b_elect(d_tmem, b_lo_base + st * (b_stage_bytes >> 4), desc_hi,
+                                            a_lo + t.x, t.y == 0xFFFFFFFFu ? t.y : a_lo + t.y,
+                                            t.z == 0xFFFFFFFFu ? t.z : a_lo + t.z,
+                                            t.w == 0xFFFFFFFFu ? t.w : a_lo + t.w, desc_hi, idesc,
+                                            first);
+                    else
                     mma_i8_ss_x4_elect(d_tmem, a_lo + t.x, t.y == 0xFFFFFFFFu ? t.y : a_lo + t.y,
                                        t.z == 0xFFFFFFFFu ? t.z : a_lo + t.z,
                                        t.w == 0xFFFFFFFFu ? t.w : a_lo + t.w, desc_hi,
@@ -616,6 +664,141 @@ dsq_win3_kernel(const __grid_constant__ CUtensorMap tmap_b,
         // ---------------- epilogue: four warps per tensor-memory lane quarter -----------
         const int quarter = warp & 3;
         const int k = (warp - W3_WARP_E0) >> 2;              // which of the quarter's warps
+        if constexpr (TR) {
+            // thread = output channel (tensor-memory lane), columns = positions;
+            // warp k of a quarter takes columns 64 k .. 64 k + 63 in units of 16
+            constexpr int E = 32 / BITS;                     // positions per code word
+            constexpr int CWU = 16 / E;                      // code words per unit: 2 (4-bit), 1 (2-bit)
+            constexpr uint32_t MASK = (1u << BITS) - 1u;
+            const DsqEpi &e = p.e;
+            const float *lut = reinterpret_cast<const float *>(smem + L.lut);
+            const int ch = n_tile * 128 + quarter * 32 + lane;
+            // a warp has work while its first code word lies inside the output row:
+            // channels past Cout are padding lanes of the packed row and get zeros
+            // (warp-uniform)
+            const bool warp_live = (n_tile * 128 + quarter * 32) * BITS / 8 < p.out_pitch;
+            float sc = 0.f, bi = 0.f;
+            if (ch < p.Ncols) {
+                sc = __ldg(e.scale + ch);
+                if (e.half_offset) sc = __fmul_rn(sc, 0.5f);
+                bi = __ldg(e.bias + ch);
+            }
+            const int pw = p.out_pitch / 4;                  // words of an output pixel
+            const int cg = (n_tile * 128 + quarter * 32 + (lane & ~(E - 1))) / E;   // this lane group's word
+            const uint32_t *res32 = reinterpret_cast<const uint32_t *>(e.residual);
+            uint32_t *y32 = reinterpret_cast<uint32_t *>(e.y_codes);
+            // output pixel (or -1) of the warp's 64 columns: lane L follows columns
+            // 64 k + 2 L and 64 k + 2 L + 1; the others get them by shuffle
+            W3Pos pos0, pos1;
+            {
+                const int g0 = m_first * TP + 64 * k + 2 * lane;
+                pos0.n = g0 / img_positions;
+                const int rem = g0 - pos0.n * img_positions;
+                pos0.h = rem / p.Wp;
+                pos0.w = rem - pos0.h * p.Wp;
+                pos1 = w3_add(pos0, 0, 0, 1, p.Hp, p.Wp);
+            }
+            bool ok = true;
+#pragma unroll 1
+            for (int it = 0; ok && it < my_tiles; ++it) {
+                const int as = it & 1;
+                const int m0 = (pos0.n < p.N && pos0.h < p.H && pos0.w < p.W)
+                                   ? (pos0.n * p.H + pos0.h) * p.W + pos0.w : -1;
+                const int m1 = (pos1.n < p.N && pos1.h < p.H && pos1.w < p.W)
+                                   ? (pos1.n * p.H + pos1.h) * p.W + pos1.w : -1;
+                pos0 = w3_add(pos0, p.t_dn, p.t_dh, p.t_dw, p.Hp, p.Wp);
+                pos1 = w3_add(pos1, p.t_dn, p.t_dh, p.t_dw, p.Hp, p.Wp);
+                if (!(ok = wait_bar_warp(bar_acc_full(as), (it >> 1) & 1u, ctl, 8))) break;
+                tc_fence_after_sync();
+                const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + as * 256;
+#pragma unroll 1
+                for (int u = 0; warp_live && u < 4; ++u) {
+                    const int col0 = 64 * k + 16 * u;
+                    uint32_t r[16], cw[CWU], resT[CWU];
+                    int mp[CWU];
+                    __syncwarp();
+                    tmem_ld_32x16(taddr + col0, r);
+                    // Word w of the unit covers E positions; lane i of a channel group
+                    // owns position i of them: it stores that position's word at the
+                    // end, and it fetches that position's residual word now.  The same
+                    // transpose that turns "E positions of my channel" into "E channels
+                    // of my position" is its own inverse, so it also turns the fetched
+                    // words into "residual codes of my channel at E positions".
+#pragma unroll
+                    for (int w = 0; w < CWU; ++w) {
+                        const int cpos = 16 * u + w * E + (lane & (E - 1));   // column of the warp
+                        const int mp_a = __shfl_sync(0xffffffffu, m0, cpos >> 1);
+                        const int mp_b = __shfl_sync(0xffffffffu, m1, cpos >> 1);
+                        mp[w] = (cpos & 1) ? mp_b : mp_a;
+                        uint32_t word = 0u;
+                        if (EPI != DSQ_EPI_CODES && e.residual && mp[w] >= 0 && 4 * cg < p.out_pitch)
+                            word = __ldg(res32 + (int64_t)mp[w] * pw + cg);
+                        resT[w] = 0u;
+                        if (EPI != DSQ_EPI_CODES) resT[w] = w3_transpose_fields<BITS>(word, lane);
+                        cw[w] = 0u;
+                    }
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        // column 16 u + j of the warp: held by lane 8 u + j / 2
+                        const int mj = __shfl_sync(0xffffffffu, (j & 1) ? m1 : m0, 8 * u + (j >> 1));
+                        const int vi = (int)r[j] >> p.shift;
+                        if constexpr (EPI == DSQ_EPI_CODES || EPI == DSQ_EPI_CODES_RES) {
+                            const float vf = __fsub_rn(__int_as_float(0x4B400000 + vi), 12582912.0f);
+                            float y = __fmaf_rn(vf, sc, bi);
+                            if (EPI == DSQ_EPI_CODES_RES) {
+                                // (positions without an output and channels past Cout
+                                // carry no residual: their codes are not stored / are 0)
+                                const uint32_t qr = (resT[(j * BITS) >> 5] >> ((j * BITS) & 31)) & MASK;
+                                y = __fadd_rn(y, ch < p.Ncols ? lut[qr] : 0.0f);
+                            }
+                            const float rr = fminf(__fmaf_rn(fmaxf(y, 0.0f), e.rq.inv, 0.5f), p.r_hi);
+                            cw[(j * BITS) >> 5] +=
+                                (uint32_t)__float_as_int(__fadd_rd(rr, 8388608.0f)) << ((j * BITS) & 31);
+                        } else {
+                            if (mj >= 0 && ch < p.Ncols) {
+                                if (e.acc_out) e.acc_out[(int64_t)mj * p.Ncols + ch] = vi;
+                                float y;
+                                if (e.general_offset) {
+                                    // S_a of the position (recomputed by every channel's
+                                    // thread: this form is not a fast path)
+                                    const int wo = mj % p.W, t2 = mj / p.W;
+                                    const int s_a = dsq_window_sa<BITS>(p.act, t2 / p.H, t2 % p.H, wo,
+                                                                        p.H, p.W, 3, 1, 1, p.P);
+                                    y = dsq_epi_y_offset(vi, s_a, e.w_offset, sc, bi);
+                                } else {
+                                    y = dsq_epi_y(vi, sc, bi);
+                                }
+                                if (e.residual) {
+                                    const uint32_t qr = (resT[(j * BITS) >> 5] >> ((j * BITS) & 31)) & MASK;
+                                    y = dsq_epi_residual(y, qr, e.res_delta, e.res_lo);
+                                }
+                                if (e.has_requant)
+                                    cw[(j * BITS) >> 5] |= dsq_code(y, e.rq) << ((j * BITS) & 31);
+                                if (e.y_f32) e.y_f32[(int64_t)mj * p.Ncols + ch] = y;
+                            }
+                        }
+                    }
+                    if constexpr (EPI == DSQ_EPI_CODES || EPI == DSQ_EPI_CODES_RES) {
+                        constexpr uint32_t FIELDS = BITS == 4 ? 0x11111111u : 0x55555555u;
+#pragma unroll
+                        for (int w = 0; w < CWU; ++w) cw[w] -= 0x4B000000u * FIELDS;
+                    }
+                    if (e.y_codes) {
+                        // fields of E positions of one channel -> fields of the E
+                        // channels of this lane group at one position
+#pragma unroll
+                        for (int w = 0; w < CWU; ++w) {
+                            const uint32_t word = w3_transpose_fields<BITS>(cw[w], lane);
+                            if (mp[w] >= 0 && 4 * cg < p.out_pitch) y32[(int64_t)mp[w] * pw + cg] = word;
+                        }
+                    }
+                }
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_acc_empty(as));
+            }
+        } else {
         const int row_in_tile = quarter * 32 + lane;
         float *sm_scale = reinterpret_cast<float *>(smem + L.epi);
         float *sm_bias = sm_scale + p.cout_pad;
@@ -764,6 +947,7 @@ dsq_win3_kernel(const __grid_constant__ CUtensorMap tmap_b,
             if (lane == 0) mbar_arrive(bar_acc_empty(as));
             if (warp == W3_WARP_E0) W3_STAMP(9, it);
         }
+        }   // !TR
     }
 
     // ---------------- teardown ------------------------------------------------------
@@ -776,7 +960,7 @@ dsq_win3_kernel(const __grid_constant__ CUtensorMap tmap_b,
     }
 }
 
-template <int BITS, int EPI>
+template <int BITS, int EPI, bool TR = false>
 int w3_launch(const CUtensorMap &tb, const CUtensorMap &ta, const W3Params &p, cudaStream_t s,
               int pdl)
 {
@@ -785,7 +969,7 @@ int w3_launch(const CUtensorMap &tb, const CUtensorMap &ta, const W3Params &p, c
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0) return DSQ_ERR_CUDA;
     const unsigned long long dev_bit = dev < 64 ? 1ull << dev : 0ull;
     if (!(configured.load(std::memory_order_acquire) & dev_bit)) {
-        if (cudaFuncSetAttribute(dsq_win3_kernel<BITS, EPI>,
+        if (cudaFuncSetAttribute(dsq_win3_kernel<BITS, EPI, TR>,
                                  cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  227 * 1024) != cudaSuccess)
             return DSQ_ERR_CUDA;
@@ -806,7 +990,7 @@ int w3_launch(const CUtensorMap &tb, const CUtensorMap &ta, const W3Params &p, c
     }
     cfg.attrs = attr;
     cfg.numAttrs = na;
-    if (cudaLaunchKernelEx(&cfg, dsq_win3_kernel<BITS, EPI>, tb, ta, p) != cudaSuccess) {
+    if (cudaLaunchKernelEx(&cfg, dsq_win3_kernel<BITS, EPI, TR>, tb, ta, p) != cudaSuccess) {
         cudaGetLastError();
         return DSQ_ERR_CUDA;
     }
@@ -817,6 +1001,13 @@ template <int BITS>
 int w3_dispatch(int epi, const CUtensorMap &tb, const CUtensorMap &ta, const W3Params &p,
                 cudaStream_t s, int pdl)
 {
+    if (p.tr) {
+        switch (epi) {
+        case DSQ_EPI_CODES: return w3_launch<BITS, DSQ_EPI_CODES, true>(tb, ta, p, s, pdl);
+        case DSQ_EPI_CODES_RES: return w3_launch<BITS, DSQ_EPI_CODES_RES, true>(tb, ta, p, s, pdl);
+        default: return w3_launch<BITS, DSQ_EPI_GENERAL, true>(tb, ta, p, s, pdl);
+        }
+    }
     switch (epi) {
     case DSQ_EPI_CODES: return w3_launch<BITS, DSQ_EPI_CODES>(tb, ta, p, s, pdl);
     case DSQ_EPI_CODES_RES: return w3_launch<BITS, DSQ_EPI_CODES_RES>(tb, ta, p, s, pdl);
@@ -840,13 +1031,15 @@ int dsq_conv3_window(const void *act_codes, const dsq_nhwc_t *shape, int bits,
     const int Cin = conv->Cin, Cout = conv->Cout;
     if (!(Cin == 64 || (Cin % 128 == 0 && Cin <= 1024))) return DSQ_ERR_UNSUPPORTED;
     if (shape->W + 2 > 32000 || shape->H + 2 > 32000) return DSQ_ERR_UNSUPPORTED;
-    // Where it pays (measured against the im2col kernel on the ResNet-18- and
-    // VGG-16-shaped layers): large images or few input channels.  Small images
-    // with many channels are few tiles with long K loops, which the im2col
-    // kernel's CTA pairs run faster.  (Hook value 3 takes the window kernel
-    // wherever the geometry allows.)
-    if (hooks.window3 != 3 && !(shape->H * shape->W >= 2500 || Cin <= 128))
-        return DSQ_ERR_UNSUPPORTED;
+    // Which kernel (hook value 1 = automatic; measured on the ResNet-18- and
+    // VGG-16-shaped layers, per layer, 20 launches back to back):
+    //  * more than 64 output channels: transposed tiles wherever they fit, except
+    //    7x7-sized images with >= 512 input channels (a handful of tiles with very
+    //    long K loops, where the im2col kernel's CTA pairs are faster);
+    //  * up to 64 output channels (half of a transposed tile's 128 weight rows
+    //    would be idle): plain tiles.
+    const bool tiny_deep = shape->H * shape->W <= 64 && Cin >= 512;
+    if (hooks.window3 == 1 && tiny_deep) return DSQ_ERR_UNSUPPORTED;
     // the lean codes epilogue wants the requantiser range to start at 0, the
     // accumulator to fit the 2^22 conversion trick and floor(r_hi) = qmax
     float r_hi = 0.f;
@@ -860,9 +1053,6 @@ int dsq_conv3_window(const void *act_codes, const dsq_nhwc_t *shape, int bits,
     p.Hp = p.H + 2; p.Wp = p.W + 2;
     const int64_t G = ((int64_t)p.N - 1) * p.Hp * p.Wp + (int64_t)p.H * p.Wp;
     if (G > (1ll << 30)) return DSQ_ERR_UNSUPPORTED;
-    p.m_tiles = (int)((G + W3_BM - 1) / W3_BM);
-    p.BN = Cout >= 256 ? 256 : ((Cout + 63) / 64) * 64;
-    p.n_tiles = (Cout + p.BN - 1) / p.BN;
     p.Ncols = Cout;
     p.E = Cin;
     p.two_taps = Cin == 64 && bits != 3;
@@ -873,43 +1063,63 @@ int dsq_conv3_window(const void *act_codes, const dsq_nhwc_t *shape, int bits,
     p.PB = Cin == 64 ? P : 16 * bits;
     p.cpp = p.PB / 16;
     p.xstep = p.two_taps ? 16 * bits : P;
-    const int need = W3_BM + 2 + 2 * p.Wp;
-    if (need <= W3_MAX_WINDOW_PX) {
-        p.nbands = 1;
-        p.a_nload = (need + 255) / 256;
-        p.a_box = (((need + p.a_nload - 1) / p.a_nload) + 7) / 8 * 8;
-        p.band_px = p.a_nload * p.a_box;
-        p.apx = p.band_px;
-        p.tap_stride = p.Wp;
-    } else {
-        p.nbands = 3;
-        p.a_nload = 1;
-        p.a_box = W3_BAND_PX;
-        p.band_px = W3_BAND_PX;
-        p.apx = 3 * W3_BAND_PX;
-        p.tap_stride = W3_BAND_PX;
-    }
-    // shared memory: resident B where one N tile's K steps all fit, else rings
-    p.cout_pad = p.n_tiles * p.BN;
-    if (p.cout_pad > W3_MAX_COUT) return DSQ_ERR_UNSUPPORTED;
-    p.b_res = 0;
+    // Tiling, window and shared memory for one of the two kernel forms.
+    // Transposed (tr): tiles of 256 positions x 128 output channels, A = weights.
+    // Plain: 128 positions x up to 256 channels, A = window.
+    auto configure = [&](int tr) -> int {
+        p.tr = tr;
+        const int tile_pos = tr ? 256 : W3_BM;
+        p.m_tiles = (int)((G + tile_pos - 1) / tile_pos);
+        p.BN = tr ? 128 : (Cout >= 256 ? 256 : ((Cout + 63) / 64) * 64);
+        p.n_tiles = (Cout + p.BN - 1) / p.BN;
+        p.cout_pad = p.n_tiles * p.BN;
+        if (p.cout_pad > W3_MAX_COUT) return 0;
+        const int need = tile_pos + 2 + 2 * p.Wp;
+        if (need <= (tr ? 768 : W3_MAX_WINDOW_PX)) {
+            p.nbands = 1;
+            p.a_nload = (need + 255) / 256;
+            p.a_box = (((need + p.a_nload - 1) / p.a_nload) + 7) / 8 * 8;
+            p.band_px = p.a_nload * p.a_box;
+            p.apx = p.band_px;
+            p.tap_stride = p.Wp;
+        } else if (!tr) {
+            p.nbands = 3;
+            p.a_nload = 1;
+            p.a_box = W3_BAND_PX;
+            p.band_px = W3_BAND_PX;
+            p.apx = 3 * W3_BAND_PX;
+            p.tap_stride = W3_BAND_PX;
+        } else {
+            return 0;
+        }
+        // shared memory: resident B where one N tile's K steps all fit, else rings
+        p.b_res = 0;
+        if (p.ksteps <= W3_MAX_BST) {
+            for (int as = W3_MAX_AS; as >= 2; --as) {
+                const W3Smem L = w3_layout(p.apx, p.BN, bits, p.PB, as, p.ksteps, 2, p.cout_pad);
+                if (L.total + 1024 <= 227u * 1024u) {
+                    p.b_res = 1; p.b_stages = p.ksteps; p.as_slots = as; p.bp_slots = 2;
+                    return 1;
+                }
+            }
+        }
+        // {A staging slots, expanded B stages, packed B slots}: the packed ring is
+        // what hides the latency of the weight loads, so it goes first
+        const int tries[6][3] = {{3, 3, 4}, {2, 3, 4}, {2, 2, 4}, {2, 2, 3}, {2, 2, 2}, {1, 2, 2}};
+        for (int t = 0; t < 6; ++t) {
+            const W3Smem L = w3_layout(p.apx, p.BN, bits, p.PB, tries[t][0], tries[t][1],
+                                       tries[t][2], p.cout_pad);
+            if (L.total + 1024 <= 227u * 1024u) {
+                p.as_slots = tries[t][0]; p.b_stages = tries[t][1]; p.bp_slots = tries[t][2];
+                return 1;
+            }
+        }
+        return 0;
+    };
     int found = 0;
-    if (p.n_tiles == 1 && p.ksteps <= W3_MAX_BST) {
-        const W3Smem L = w3_layout(p.apx, p.BN, bits, p.PB, W3_MAX_AS, p.ksteps, 2, p.cout_pad);
-        if (L.total + 1024 <= 227u * 1024u) {
-            p.b_res = 1; p.b_stages = p.ksteps; p.as_slots = W3_MAX_AS; p.bp_slots = 2; found = 1;
-        }
-    }
-    // {A staging slots, expanded B stages, packed B slots}: the packed ring is
-    // what hides the latency of the weight loads, so it goes first
-    const int tries[6][3] = {{3, 3, 4}, {2, 3, 4}, {2, 2, 4}, {2, 2, 3}, {2, 2, 2}, {1, 2, 2}};
-    for (int t = 0; !found && t < 6; ++t) {
-        const W3Smem L = w3_layout(p.apx, p.BN, bits, p.PB, tries[t][0], tries[t][1], tries[t][2],
-                                   p.cout_pad);
-        if (L.total + 1024 <= 227u * 1024u) {
-            p.as_slots = tries[t][0]; p.b_stages = tries[t][1]; p.bp_slots = tries[t][2]; found = 1;
-        }
-    }
+    const bool want_tr = hooks.window3 == 3 || (hooks.window3 == 1 && Cout > 64);
+    if (bits != 3 && want_tr) found = configure(1);
+    if (!found) found = configure(0);
     if (!found) return DSQ_ERR_UNSUPPORTED;
     p.smem_bytes = (int)w3_layout(p.apx, p.BN, bits, p.PB, p.as_slots, p.b_stages, p.bp_slots,
                                   p.cout_pad).total + 1024;
@@ -921,15 +1131,18 @@ int dsq_conv3_window(const void *act_codes, const dsq_nhwc_t *shape, int bits,
     if (p.mstep > p.m_tiles) p.mstep = p.m_tiles;
     if (p.mstep < 1) return DSQ_ERR_UNSUPPORTED;
     {
-        const int64_t d = (int64_t)p.mstep * W3_BM, img = (int64_t)p.Hp * p.Wp;
+        const int64_t d = (int64_t)p.mstep * (p.tr ? 256 : W3_BM), img = (int64_t)p.Hp * p.Wp;
         p.t_dn = (int)(d / img);
         p.t_dh = (int)((d % img) / p.Wp);
         p.t_dw = (int)((d % img) % p.Wp);
         for (int b = 0; b < p.nbands; ++b)
             for (int i = 0; i < p.a_nload; ++i) {
+                // (every digit below its base, so that one carry per digit is
+                // enough when the kernel adds them to a position)
                 const int off = p.nbands > 1 ? b * p.Wp : i * p.a_box;
-                p.ld_dh[b * p.a_nload + i] = off / p.Wp;
-                p.ld_dw[b * p.a_nload + i] = off % p.Wp;
+                p.ld_dn[b * p.a_nload + i] = (int)(off / img);
+                p.ld_dh[b * p.a_nload + i] = (int)((off % img) / p.Wp);
+                p.ld_dw[b * p.a_nload + i] = (int)((off % img) % p.Wp);
             }
     }
     p.wait_ns = hooks.wait_ns;

@@ -35,10 +35,11 @@ int dsq_set_wait_limit_ns(long long ns);
 
 /* 3x3 stride-1 convolutions on an expanded shared-memory window
  * (dsq_conv3.cu): 1 = where it is the faster kernel (default), 0 = never (the
- * im2col kernel takes them), 3 = wherever the geometry allows, 2 = as 3 with
- * the row phase of the window written into the A descriptor's base-offset
- * field (a probe of that field's meaning: the tensor core swizzles by
- * absolute shared-memory address, so this gives wrong numbers). */
+ * im2col kernel takes them), 3 = wherever the geometry allows (transposed
+ * tiles where those fit), 4 = as 3 but plain tiles only, 2 = as 4 with the row
+ * phase of the window written into the A descriptor's base-offset field (a
+ * probe of that field's meaning: the tensor core swizzles by absolute
+ * shared-memory address, so this gives wrong numbers). */
 int dsq_set_conv3_window(int mode);
 
 /* Test hook: in every later launch the thread that issues the TMA copies of

@@ -412,6 +412,36 @@ __device__ __forceinline__ void mma_i8_ss_x4_elect(uint32_t d_tmem, uint32_t a_l
         : "memory");
 }
 
+// Same with the roles swapped: the A descriptor advances 32 bytes per
+// instruction, the four B descriptors' low words are given one by one
+// (0xFFFFFFFF = leave this instruction out).
+__device__ __forceinline__ void mma_i8_ss_x4b_elect(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi,
+                                                    uint32_t b_lo0, uint32_t b_lo1, uint32_t b_lo2,
+                                                    uint32_t b_lo3, uint32_t b_hi, uint32_t idesc,
+                                                    uint32_t accumulate_first)
+{
+    asm volatile(
+        "{\n\t.reg .pred p0, p1, pe, v1, v2, v3;\n\t"
+        ".reg .b64 da0, da1, da2, da3, db0, db1, db2, db3;\n\t.reg .b32 l1, l2, l3;\n\t"
+        "setp.ne.b32 p0, %9, 0;\n\tsetp.eq.b32 p1, %9, %9;\n\t"
+        "add.u32 l1, %1, 2;\n\tadd.u32 l2, %1, 4;\n\tadd.u32 l3, %1, 6;\n\t"
+        "mov.b64 da0, {%1, %2};\n\tmov.b64 da1, {l1, %2};\n\t"
+        "mov.b64 da2, {l2, %2};\n\tmov.b64 da3, {l3, %2};\n\t"
+        "mov.b64 db0, {%3, %7};\n\tmov.b64 db1, {%4, %7};\n\t"
+        "mov.b64 db2, {%5, %7};\n\tmov.b64 db3, {%6, %7};\n\t"
+        "elect.sync _|pe, 0xffffffff;\n\t"
+        "setp.ne.b32 v1, %4, 0xFFFFFFFF;\n\tsetp.ne.b32 v2, %5, 0xFFFFFFFF;\n\t"
+        "setp.ne.b32 v3, %6, 0xFFFFFFFF;\n\t"
+        "and.pred v1, v1, pe;\n\tand.pred v2, v2, pe;\n\tand.pred v3, v3, pe;\n\t"
+        "@pe tcgen05.mma.cta_group::1.kind::i8 [%0], da0, db0, %8, p0;\n\t"
+        "@v1 tcgen05.mma.cta_group::1.kind::i8 [%0], da1, db1, %8, p1;\n\t"
+        "@v2 tcgen05.mma.cta_group::1.kind::i8 [%0], da2, db2, %8, p1;\n\t"
+        "@v3 tcgen05.mma.cta_group::1.kind::i8 [%0], da3, db3, %8, p1;\n\t}" ::"r"(d_tmem),
+        "r"(a_lo), "r"(a_hi), "r"(b_lo0), "r"(b_lo1), "r"(b_lo2), "r"(b_lo3), "r"(b_hi), "r"(idesc),
+        "r"(accumulate_first)
+        : "memory");
+}
+
 // tcgen05.commit by one elected lane of a converged warp (all lanes call).
 __device__ __forceinline__ void mma_commit_elect(uint32_t bar)
 {

@@ -1688,7 +1688,7 @@ int dsq_set_test_skip_b_round(int round)
 
 int dsq_set_conv3_window(int mode)
 {
-    if (mode < 0 || mode > 3) return DSQ_ERR_SHAPE;
+    if (mode < 0 || mode > 4) return DSQ_ERR_SHAPE;
     g_window3 = mode;
     return DSQ_OK;
 }

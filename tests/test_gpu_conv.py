@@ -228,16 +228,22 @@ WINDOW_GEOMS = [  # N, H, W, Cin, Cout: 3x3, stride 1, pad 1 on the shared-memor
     (1, 6, 300, 128, 72), (2, 56, 56, 128, 128), (70, 5, 5, 64, 96)]
 
 
+@pytest.mark.parametrize("form", [3, 4])
 @pytest.mark.parametrize("bits", [2, 3, 4])
 @pytest.mark.parametrize("geom", WINDOW_GEOMS)
-def test_conv3x3_window_kernel(dsq, geom, bits):
+def test_conv3x3_window_kernel(dsq, geom, bits, form):
     """3x3 stride-1 convolutions whose A operand is an expanded window of the
     input in shared memory (one constant row shift per filter tap): image sizes
     from 1x1 to wider than a window, tiles that span several images, channel
     counts with a ragged last N tile, one to four planes of 128 channels, with
-    and without a residual operand, every element against the oracle."""
+    and without a residual operand, every element against the oracle.  Both
+    forms of the kernel: form 3 = transposed tiles (256 positions x 128
+    channels, weights as the A operand) where the geometry allows, form 4 =
+    plain tiles only (128 positions x up to 256 channels)."""
     n, h, w, ci, co = geom
-    dsq.dsq_set_conv3_window(3)        # this kernel wherever the geometry allows
+    if bits == 3 and form == 4:
+        pytest.skip("3-bit codes take the plain form in both settings")
+    dsq.dsq_set_conv3_window(form)     # this kernel wherever the geometry allows
     try:
         conv_case(dsq, n, h, w, ci, co, 3, 1, 1, bits, 0.5, residual=(n % 2 == 0),
                   seed=n + h + ci)
