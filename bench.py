@@ -51,7 +51,8 @@ INT8_NOMINAL_TOPS = 4500.0
 def kernel_sources_sha256():
     import hashlib
     h = hashlib.sha256()
-    for f in ("dsq_tc.cu", "dsq_ptx.cuh", "dsq_epilogue.cuh", "dsq_common.cuh"):
+    for f in ("dsq_tc.cu", "dsq_conv3.cu", "dsq_tc_common.cuh", "dsq_ptx.cuh", "dsq_epilogue.cuh",
+              "dsq_common.cuh"):
         h.update(open(os.path.join(ROOT, "paper_1908_05033_b200", "csrc", f), "rb").read())
     return h.hexdigest()
 
@@ -471,7 +472,8 @@ def run_ours(args):
     int8_peak = 2.0 * bf16_peak                 # int8 : bf16 nominal ratio 2
     achieved = 2.0 * macs_step / (conv_in_step_ms * 1e-3) / 1e12
     roofline = {
-        "kernel": f"dsq_tc_kernel (dsq_conv2d), {n_conv} launches per step",
+        "kernel": f"dsq_win3_kernel (3x3 stride 1) + dsq_tc_kernel (1x1, strided) behind dsq_conv2d, "
+                  f"{n_conv} launches per step",
         "bound": "tensor", "achieved": achieved, "peak": int8_peak, "unit": "TOP/s",
         "frac": achieved / int8_peak,
         "peak_source": f"2 x bf16_tflops{'' if burst else '_sustained'} of {peaks['source']} peaks "
