@@ -35,10 +35,10 @@ if ROOT not in sys.path:
 
 import dsq_inputs  # noqa: E402
 
-# DRAM traffic of the dominant kernel (dsq_tc_kernel) per launch in this
+# DRAM traffic of the tensor-core convolution kernels per launch in this
 # workload, from one ncu capture (profiles/bench_launch_list.txt); valid only
 # for the kernel sources it was taken on (checked by hash)
-TRAFFIC = {"bytes_per_launch": 4728441, "sources_sha256": "89bc47d406d28b71028414db5fd3c069869ee66c86bb207ba91c8f00d996b40f"}
+TRAFFIC = {"bytes_per_launch": 4726885, "sources_sha256": "29b376070cc6976455d295b3d50e21a9d3187d1ed26eafb01c642c6828775896"}
 
 WORKLOAD = "resnet18-shaped stack, 4-bit W/A, batch 64, 56x56x64 stem output, 19 convs"
 METRIC = "4-bit ResNet-18 conv-stack throughput (effective low-bit conv TOPS alongside)"
