@@ -214,6 +214,17 @@ int dsq_gemm(const void *A_codes, const void *B_codes, int64_t M, int64_t N,
              int64_t K, int bits, int32_t *C_i32, const float *row_scale,
              float *D_f32, void *workspace, size_t ws_bytes, void *stream);
 
+/* Workspace with which dsq_gemm runs this problem fastest.  Any workspace of
+ * dsq_workspace_bytes() works (one fused kernel that expands the packed codes
+ * tile by tile).  Given this many bytes (the status words, then room for both
+ * operands as 8-bit rows: about (M + N) * K bytes), large problems (M, N, K >=
+ * 1024) take two passes instead: every packed row is expanded to 8-bit lanes
+ * once, then an 8-bit tensor-core GEMM reads the rows by TMA.  Same results
+ * bit for bit.  The area behind the first dsq_workspace_bytes() bytes is
+ * scratch: its contents after the call are unspecified, and calls that may
+ * overlap on the GPU must not share it. */
+size_t dsq_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int bits);
+
 /* dsq_gemm for callers that cannot allocate device memory.  (The paper has
  * no counterpart: this is a deployment convenience of the library.)
  *

@@ -66,6 +66,7 @@ _SIGNATURES = {
                             _vp, _vp, _vp, _vp]),
     "dsq_gemm": (_int, [_vp, _vp, _i64, _i64, _i64, _int, _vp, _vp, _vp, _vp,
                         _sz, _vp]),
+    "dsq_gemm_workspace_bytes": (_sz, [_i64, _i64, _i64, _int]),
     "dsq_gemm_static_ws": (_int, [_vp, _vp, _i64, _i64, _i64, _int, _vp, _vp, _vp,
                                   _int, _vp]),
     "dsq_maxpool2x2": (_int, [_vp, C.POINTER(dsq_nhwc_t), _int, _vp, _sz,
@@ -89,6 +90,7 @@ _HOOKS = {
     "dsq_set_wait_limit_ns": (_int, [C.c_longlong]),
     "dsq_set_test_skip_b_round": (_int, [_int]),
     "dsq_set_conv3_window": (_int, [_int]),
+    "dsq_set_gemm_two_pass": (_int, [_int]),
 }
 for _name, (_res, _args) in list(_SIGNATURES.items()) + list(_HOOKS.items()):
     _f = getattr(lib, _name)       # AttributeError if a symbol is missing
@@ -153,6 +155,19 @@ def dsq_status_string(status):
 # ---- workspace ----------------------------------------------------------------
 def new_workspace(device="cuda"):
     ws = torch.empty(dsq_workspace_bytes(), dtype=torch.uint8, device=device)
+    _check(lib.dsq_workspace_init(_p(ws), ws.numel(), _stream()),
+           "dsq_workspace_init")
+    return ws
+
+
+def dsq_gemm_workspace_bytes(M, N, K, bits):
+    return int(lib.dsq_gemm_workspace_bytes(M, N, K, bits))
+
+
+def new_gemm_workspace(M, N, K, bits, device="cuda"):
+    """Workspace with room for the expanded operands of an M x N x K GEMM (the
+    two-pass path of dsq_gemm); the status words in front are cleared."""
+    ws = torch.empty(dsq_gemm_workspace_bytes(M, N, K, bits), dtype=torch.uint8, device=device)
     _check(lib.dsq_workspace_init(_p(ws), ws.numel(), _stream()),
            "dsq_workspace_init")
     return ws
@@ -358,6 +373,10 @@ def dsq_set_round_k_steps(ks):
     _check(lib.dsq_set_round_k_steps(ks), "dsq_set_round_k_steps")
 
 
+def dsq_set_gemm_two_pass(on):
+    _check(lib.dsq_set_gemm_two_pass(int(on)), "dsq_set_gemm_two_pass")
+
+
 def dsq_set_cta_pairs(mode):
     _check(lib.dsq_set_cta_pairs(mode), "dsq_set_cta_pairs")
 
@@ -410,4 +429,5 @@ def dsq_probe_i8_mma_rate(iters, ws):
 
 __all__ = [n for n in dir() if n.startswith("dsq_")] + [
     "lib", "DsqError", "EXPORTED_SYMBOLS", "HOOK_SYMBOLS", "new_workspace",
+    "new_gemm_workspace",
     "check_workspace"]

@@ -7,7 +7,8 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libdsq_b200.so")
-SOURCES = ["dsq_elementwise.cu", "dsq_dwconv.cu", "dsq_tc.cu", "dsq_conv3.cu", "dsq_soft.cu"]
+SOURCES = ["dsq_elementwise.cu", "dsq_dwconv.cu", "dsq_tc.cu", "dsq_conv3.cu", "dsq_gemm8.cu",
+           "dsq_soft.cu"]
 HEADERS = ["dsq_common.cuh", "dsq_epilogue.cuh", "dsq_ptx.cuh", "dsq_tc_common.cuh",
            "dsq_tc_host.h", "dsq_hooks.h",
            os.path.join("..", "..", "include", "dsq.h")]

@@ -59,6 +59,8 @@ def main(argv=None):
     ap.add_argument("--window", type=int, default=1,
                     help="3x3 stride-1 convolutions: 1 shared-memory window kernel, 0 im2col kernel")
     ap.add_argument("--residual", action="store_true")
+    ap.add_argument("--fused", action="store_true",
+                    help="gemm: the single fused kernel (small workspace) instead of two passes")
     a = ap.parse_args(argv)
     dev = "cuda"
     ws = B.new_workspace(dev)
@@ -77,6 +79,8 @@ def main(argv=None):
         A = torch.randint(0, 256, (n, pitch), dtype=torch.uint8, device=dev, generator=gen)
         Bm = torch.randint(0, 256, (n, pitch), dtype=torch.uint8, device=dev, generator=gen)
         Cm = torch.empty((n, n), dtype=torch.int32, device=dev)
+        if not a.fused:
+            ws = B.new_gemm_workspace(n, n, n, bits, dev)
         ms, all_ms = _timeit(lambda: B.dsq_gemm(A, Bm, n, n, n, bits, ws, out_i32=Cm),
                              a.iters, flush)
         out.update(size=n, ms=ms, tops=2.0 * n ** 3 / (ms * 1e-3) / 1e12, all_ms=all_ms)

@@ -42,6 +42,10 @@ int dsq_set_wait_limit_ns(long long ns);
  * shared-memory address, so this gives wrong numbers). */
 int dsq_set_conv3_window(int mode);
 
+/* dsq_gemm with a workspace large enough for the expanded operands: 1 = take
+ * the two-pass path (default), 0 = always the fused kernel. */
+int dsq_set_gemm_two_pass(int on);
+
 /* Test hook: in every later launch the thread that issues the TMA copies of
  * the packed B operand leaves out the copy of round `round` of its CTA
  * (0 = the first) and issues nothing after it; -1 switches the hook off.

@@ -210,6 +210,20 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *m,
         : "memory");
 }
 
+// Same for a CTA pair (cta_group::2): the copy lands in THIS CTA's shared
+// memory, its bytes are counted on an mbarrier of either CTA of the pair
+// (`bar` is a shared::cluster address, e.g. the leader's barrier through
+// map_to_cta).  No multicast: every CTA fetches its own tile.
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap *m,
+                                                 int x, int y, uint32_t bar_cluster)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes"
+        " [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+        "l"(m), "r"(x), "r"(y), "r"(bar_cluster)
+        : "memory");
+}
+
 // 4-D im2col load over an NHWC tensor (dims C, W, H, N): `pixelsPerColumn`
 // pixels x `channelsPerPixel` bytes.  (w, h) is the position of the filter
 // window's corner for the first pixel (output position * stride - pad); the
@@ -439,6 +453,35 @@ __device__ __forceinline__ void mma_i8_ss_x4b_elect(uint32_t d_tmem, uint32_t a_
         "@v3 tcgen05.mma.cta_group::1.kind::i8 [%0], da3, db3, %8, p1;\n\t}" ::"r"(d_tmem),
         "r"(a_lo), "r"(a_hi), "r"(b_lo0), "r"(b_lo1), "r"(b_lo2), "r"(b_lo3), "r"(b_hi), "r"(idesc),
         "r"(accumulate_first)
+        : "memory");
+}
+
+// One 128-byte K step of a CTA pair's tile with both operands in shared
+// memory (cta_group::2: M = 256, each CTA holds 128 rows of A and half of the
+// B rows at the same shared-memory offsets): four K = 32 instructions, the
+// descriptors advancing 32 bytes each; issued by one elected lane of the
+// converged warp of the pair's leader CTA.
+__device__ __forceinline__ void mma_i8_ss_pair_x4_elect(uint32_t d_tmem, uint32_t a_lo,
+                                                        uint32_t a_hi, uint32_t b_lo,
+                                                        uint32_t b_hi, uint32_t idesc,
+                                                        uint32_t accumulate_first)
+{
+    asm volatile(
+        "{\n\t.reg .pred p0, p1, pe;\n\t"
+        ".reg .b64 da0, da1, da2, da3, db0, db1, db2, db3;\n\t.reg .b32 x1, x2, x3, y1, y2, y3;\n\t"
+        "setp.ne.b32 p0, %6, 0;\n\tsetp.eq.b32 p1, %6, %6;\n\t"
+        "add.u32 x1, %1, 2;\n\tadd.u32 x2, %1, 4;\n\tadd.u32 x3, %1, 6;\n\t"
+        "add.u32 y1, %3, 2;\n\tadd.u32 y2, %3, 4;\n\tadd.u32 y3, %3, 6;\n\t"
+        "mov.b64 da0, {%1, %2};\n\tmov.b64 da1, {x1, %2};\n\t"
+        "mov.b64 da2, {x2, %2};\n\tmov.b64 da3, {x3, %2};\n\t"
+        "mov.b64 db0, {%3, %4};\n\tmov.b64 db1, {y1, %4};\n\t"
+        "mov.b64 db2, {y2, %4};\n\tmov.b64 db3, {y3, %4};\n\t"
+        "elect.sync _|pe, 0xffffffff;\n\t"
+        "@pe tcgen05.mma.cta_group::2.kind::i8 [%0], da0, db0, %5, p0;\n\t"
+        "@pe tcgen05.mma.cta_group::2.kind::i8 [%0], da1, db1, %5, p1;\n\t"
+        "@pe tcgen05.mma.cta_group::2.kind::i8 [%0], da2, db2, %5, p1;\n\t"
+        "@pe tcgen05.mma.cta_group::2.kind::i8 [%0], da3, db3, %5, p1;\n\t}" ::"r"(d_tmem),
+        "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate_first)
         : "memory");
 }
 

@@ -1445,6 +1445,7 @@ std::atomic<int> g_pair_mode{0};      // dsq_set_cta_pairs: 0 automatic, 1 never
 std::atomic<unsigned long long> g_wait_ns{WAIT_LIMIT_NS};   // dsq_set_wait_limit_ns
 std::atomic<int> g_skip_b_round{-1};  // dsq_set_test_skip_b_round
 std::atomic<int> g_window3{1};        // dsq_set_conv3_window
+std::atomic<int> g_two_pass{1};       // dsq_set_gemm_two_pass
 
 int pick_bn(int m_tiles, int ncols, int bits)
 {
@@ -1726,6 +1727,19 @@ static int gemm_check_args(const void *A_codes, const void *B_codes, int64_t M, 
     return DSQ_OK;
 }
 
+size_t dsq_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int bits)
+{
+    if (bits < 2 || bits > 4 || M <= 0 || N <= 0 || K <= 0) return DSQ_WS_BYTES;
+    const size_t need = dsq_gemm8_scratch_bytes(M, N, K);
+    return need ? DSQ_WS_BYTES + 1024 + need : DSQ_WS_BYTES;
+}
+
+int dsq_set_gemm_two_pass(int on)
+{
+    g_two_pass = on ? 1 : 0;
+    return DSQ_OK;
+}
+
 int dsq_gemm(const void *A_codes, const void *B_codes, int64_t M, int64_t N, int64_t K,
              int bits, int32_t *C_i32, const float *row_scale, float *D_f32, void *workspace,
              size_t ws_bytes, void *stream)
@@ -1735,6 +1749,19 @@ int dsq_gemm(const void *A_codes, const void *B_codes, int64_t M, int64_t N, int
     if (st) return st;
     if (!dsq_aligned16(workspace)) return DSQ_ERR_ALIGN;
     if (ws_bytes < DSQ_WS_BYTES) return DSQ_ERR_SIZE;
+
+    // large problems, when the caller's workspace has room for the expanded
+    // operands (dsq_gemm_workspace_bytes): expand every row once, then an
+    // 8-bit GEMM fed by TMA alone
+    const size_t scratch_need = g_two_pass.load() ? dsq_gemm8_scratch_bytes(M, N, K) : 0;
+    if (scratch_need) {
+        const uintptr_t w0 = reinterpret_cast<uintptr_t>(workspace);
+        const uintptr_t s0 = (w0 + DSQ_WS_BYTES + 1023u) & ~(uintptr_t)1023u;
+        if (ws_bytes >= (s0 - w0) + scratch_need)
+            return dsq_gemm8_launch(A_codes, B_codes, M, N, K, bits, C_i32, row_scale, D_f32,
+                                    workspace, reinterpret_cast<void *>(s0),
+                                    (cudaStream_t)stream);
+    }
 
     const size_t pitch = dsq_row_pitch(K, bits);
     TcParams p = {};

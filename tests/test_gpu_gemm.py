@@ -89,6 +89,94 @@ def test_gemm_full_size_sampled(dsq, bits, size):
     assert np.array_equal(Cg, Cg2)
 
 
+def run_two_pass(dsq, A, B, rs, bits, want_i32=True):
+    """dsq_gemm with a workspace that has room for the expanded operands."""
+    M, K = A.shape
+    Nn = B.shape[0]
+    assert dsq.dsq_gemm_workspace_bytes(M, Nn, K, bits) > dsq.dsq_workspace_bytes()
+    ws = dsq.new_gemm_workspace(M, Nn, K, bits)
+    Ap, Bp = dsq.dsq_pack_codes(T(A), bits), dsq.dsq_pack_codes(T(B), bits)
+    Cg, Dg = dsq.dsq_gemm(Ap, Bp, M, Nn, K, bits, ws, row_scale=T(rs), want_i32=want_i32)
+    assert dsq.dsq_workspace_status(ws) == 0
+    return (N(Cg) if want_i32 else None), N(Dg)
+
+
+# the two-pass path (rows expanded to 8-bit once, then an 8-bit GEMM): whole
+# tiles, ragged M / N / K, an N that is not a multiple of 8 (scalar stores), a K
+# that is not a multiple of 16
+TWO_PASS_SIZES = [(1024, 1024, 1024), (1100, 1030, 1050), (1024, 1027, 1031),
+                  (1281, 1536, 2048)]
+
+
+@pytest.mark.parametrize("bits", [2, 3, 4])
+@pytest.mark.parametrize("size", TWO_PASS_SIZES)
+def test_gemm_two_pass_full(dsq, bits, size):
+    M, Nn, K = size
+    A, B, rs = dsq_inputs.gemm_case(M, Nn, K, bits)
+    C = native.gemm(A, B)
+    Cg, Dg = run_two_pass(dsq, A, B, rs, bits)
+    assert np.array_equal(C, Cg)
+    assert np.array_equal(native.gemm_dequant(C, rs), Dg)
+    _, Dg = run_two_pass(dsq, A, B, rs, bits, want_i32=False)
+    assert np.array_equal(native.gemm_dequant(C, rs), Dg)
+
+
+@pytest.mark.parametrize("bits", [2, 3, 4])
+def test_gemm_two_pass_extreme_codes(dsq, bits):
+    half = 1 << (bits - 1)
+    M, Nn, K = 1024, 1024, 8192
+    A = np.full((M, K), -half, np.int8)
+    B = np.full((Nn, K), 2 * half - 1, np.int8)
+    rs = np.ones(M, np.float32)
+    Cg, _ = run_two_pass(dsq, A, B, rs, bits)
+    assert np.all(Cg == K * -half * (2 * half - 1))
+    A[:] = half - 1
+    Cg, _ = run_two_pass(dsq, A, B, rs, bits)
+    assert np.all(Cg == K * (half - 1) * (2 * half - 1))
+
+
+@pytest.mark.parametrize("bits,size", [(4, 4096), (2, 4096), (3, 4096), (4, 8192)])
+def test_gemm_two_pass_full_size_sampled(dsq, bits, size):
+    """Full-size launch as the benchmark times it: sampled dot products and the
+    last rows against the oracle, and every element against the fused kernel."""
+    A, B, rs = dsq_inputs.gemm_case(size, size, size, bits)
+    Cg, Dg = run_two_pass(dsq, A, B, rs, bits)
+    rng = np.random.default_rng(size + bits)
+    rows = np.sort(rng.choice(size, 64, replace=False))
+    cols = np.sort(rng.choice(size, 64, replace=False))
+    C = native.gemm(A[rows], B[cols])
+    assert np.array_equal(C, Cg[np.ix_(rows, cols)])
+    assert np.array_equal(native.gemm_dequant(C, rs[rows]), Dg[np.ix_(rows, cols)])
+    C = native.gemm(A[size - 3:], B)
+    assert np.array_equal(C, Cg[size - 3:])
+    Cf, Df = run(dsq, A, B, rs, bits)                 # fused kernel, small workspace
+    assert np.array_equal(Cf, Cg) and np.array_equal(Df, Dg)
+
+
+def test_gemm_two_pass_repeated_launches_identical(dsq):
+    """300 launches of 4096^3 through the two-pass path (a shared scratch
+    rewritten every call, two accumulators, a CTA pair's barriers crossing SMs):
+    every launch equals the first, whose rows are checked against the oracle."""
+    size, bits = 4096, 4
+    A, B, rs = dsq_inputs.gemm_case(size, size, size, bits)
+    ws = dsq.new_gemm_workspace(size, size, size, bits)
+    Ap, Bp = dsq.dsq_pack_codes(T(A), bits), dsq.dsq_pack_codes(T(B), bits)
+    rst = T(rs)
+    C0, D0 = dsq.dsq_gemm(Ap, Bp, size, size, size, bits, ws, row_scale=rst)
+    C0, D0 = C0.clone(), D0.clone()
+    C = torch.empty_like(C0)
+    D = torch.empty_like(D0)
+    bad = torch.zeros((), dtype=torch.int64, device="cuda")
+    for _ in range(300):
+        dsq.dsq_gemm(Ap, Bp, size, size, size, bits, ws, row_scale=rst, out_i32=C, out_f32=D)
+        bad += (C != C0).any().to(torch.int64) + (D != D0).any().to(torch.int64)
+    assert int(bad.item()) == 0
+    assert dsq.dsq_workspace_status(ws) == 0
+    rows = np.arange(0, size, 257)
+    Cref = native.gemm(A[rows], B)
+    assert np.array_equal(Cref, N(C0)[rows])
+
+
 def test_gemm_repeated_launches_identical(dsq):
     """Regression test of a race between the two CTAs of a pair that showed
     about once in 150 launches (a stale half of the expanded B operand read by

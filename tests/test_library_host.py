@@ -82,6 +82,12 @@ def test_validation_status_codes_without_a_gpu():
     assert lib.dsq_gemm(fake, fake, 128, 128, 128, 4, fake, None, fake, fake, 256, None) == -1
     # K so large that 2^7 * (2^b - 1) * K overflows int32
     assert lib.dsq_gemm(fake, fake, 128, 128, 1 << 21, 4, fake, None, None, fake, 256, None) == -7
+    # workspace query: small problems keep the status words only, large ones get
+    # room for both operands as 8-bit rows (K rounded up to 16)
+    assert lib.dsq_gemm_workspace_bytes(512, 4096, 4096, 4) == lib.dsq_workspace_bytes()
+    assert lib.dsq_gemm_workspace_bytes(4096, 4096, 4096, 7) == lib.dsq_workspace_bytes()
+    assert lib.dsq_gemm_workspace_bytes(4096, 4096, 4096, 4) == 256 + 1024 + 2 * 4096 * 4096
+    assert lib.dsq_gemm_workspace_bytes(1025, 1030, 1031, 2) >= 256 + 1024 + (1025 + 1030) * 1040
     # the no-workspace variant rejects bad arguments before it looks up its
     # scratch or enqueues anything (so this works without a GPU)
     assert lib.dsq_gemm_static_ws(None, fake, 128, 128, 128, 4, fake, None, None, 1, None) == -1
