@@ -77,6 +77,31 @@ def gemm_case(M, N, K, bits, workload_id=2):
     return A, B, row_scale
 
 
+def binary_gemm_case(M, N, K, workload_id=2):
+    """Bit rows (0/1, uniform) of a binary GEMM and row_scale [M]."""
+    rng = rng_for(workload_id, stream=M * 29 + N * 13 + K * 5 + 1)
+    A = rng.integers(0, 2, size=(M, K)).astype(np.int8)
+    B = rng.integers(0, 2, size=(N, K)).astype(np.int8)
+    row_scale = (rng.uniform(0.5, 1.5, size=M) * 2.0 ** -10).astype(np.float32)
+    return A, B, row_scale
+
+
+def weight_only_case(M, N, K, bits, workload_id=2):
+    """Weight-only linear layer: activations X [M,K] ~ N(0,1) rounded to
+    bfloat16 (returned as float32 holding bf16 values), unsigned weight codes
+    [N,K] uniform over the full range, per-channel clip u ~ U(0.05, 0.3) on
+    [-u, u], bias ~ N(0, 0.1)."""
+    rng = rng_for(workload_id, stream=M * 23 + N * 11 + K * 3 + bits)
+    x = rng.standard_normal((M, K)).astype(np.float32)
+    xi = x.view(np.uint32)
+    xi = ((xi + 0x7FFF + ((xi >> 16) & 1)) & 0xFFFF0000).astype(np.uint32)   # round to nearest even
+    x = xi.view(np.float32)
+    q = rng.integers(0, 2 ** bits, size=(N, K)).astype(np.int8)
+    u = rng.uniform(0.05, 0.3, size=N).astype(np.float32)
+    bias = (rng.standard_normal(N) * 0.1).astype(np.float32)
+    return x, q, u, bias
+
+
 # --------------------------------------------------------------------------
 # workloads 3-5: layer stacks.  A stack is a list of Layer records over named
 # code tensors; each tensor has one quantiser range (bits, lo, hi).

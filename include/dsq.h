@@ -225,6 +225,50 @@ int dsq_gemm(const void *A_codes, const void *B_codes, int64_t M, int64_t N,
  * overlap on the GPU must not share it. */
 size_t dsq_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int bits);
 
+/* Binary GEMM (paper Eq. 1, the binary quantiser Q_B = sgn with sgn(0) = +1,
+ * i.e. the 1-bit case of the uniform quantiser on a symmetric range; the 1/1
+ * rows of the paper's Tables 3 and 6):
+ *   C[m][n] = sum_k a[m][k] * b[n][k],  a, b in {-1, +1}
+ * which equals K - 2 * popcount(A[m] xor B[n]) (the xnor-popcount form).
+ *   A_bits  packed rows [M][K], 1 bit per value: bit 1 = +1, bit 0 = -1
+ *           (element j in bit j & 7 of byte j / 8; row pitch
+ *           dsq_row_pitch(K, 1); bits past K are ignored)
+ *   B_bits  packed rows [N][K], same format
+ *   C_i32, row_scale, D_f32 as in dsq_gemm.
+ * On this GPU the +-1 values go through the 8-bit integer tensor-core path:
+ * every row is expanded to int8 once into the workspace, then the same
+ * TMA-fed 8-bit GEMM as dsq_gemm's two-pass path runs.  `workspace` must hold
+ * dsq_binary_gemm_workspace_bytes(M, N, K) bytes (DSQ_ERR_SIZE otherwise),
+ * its first dsq_workspace_bytes() bytes cleared with dsq_workspace_init. */
+size_t dsq_binary_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K);
+int dsq_binary_gemm(const void *A_bits, const void *B_bits, int64_t M, int64_t N,
+                    int64_t K, int32_t *C_i32, const float *row_scale,
+                    float *D_f32, void *workspace, size_t ws_bytes, void *stream);
+
+/* Weight-only low-bit GEMM (the W-bit / 32-bit-activation rows of the paper's
+ * Table 7: weights quantised by Algorithm 1 steps 1, 3, activations left in
+ * floating point; here activations are bf16):
+ *   Y[m][n] = fma(sum_k X[m][k] * v[n][k], col_scale[n], col_bias[n])
+ * with v = 2 c + 1 when w_offset = 0.5 (the paper's grid w^ = l_w + Delta_w q
+ * on a symmetric clip: w^ = (Delta_w / 2)(2 c + 1), so col_scale = Delta_w / 2)
+ * and v = c when w_offset = 0 (w^ = Delta_w c, col_scale = Delta_w); c is the
+ * signed code c = q - 2^(bits-1).  Other offsets: DSQ_ERR_UNSUPPORTED.
+ *   X_bf16    [M][K] bfloat16, row-major, K a multiple of 8 (rows are read by
+ *             TMA: 16-byte pitch), DSQ_ERR_ALIGN otherwise
+ *   W_codes   packed rows [N][K] of SIGNED codes, bits in {1, 2, 3, 4}
+ *   col_scale [N] fp32; col_bias [N] fp32 or NULL
+ *   Y_f32     [M][N] fp32
+ * Products are exact (bf16 times a small integer); they are accumulated in
+ * fp32 by the tensor core in an order of its own, so Y is within
+ * K * 2^-23 * sum_k |X v| * |col_scale| of the exact value.  The weights are
+ * expanded to bf16 once into the workspace (dsq_wgemm_workspace_bytes(N, K)),
+ * then a TMA-fed bf16 tensor-core GEMM runs. */
+size_t dsq_wgemm_workspace_bytes(int64_t N, int64_t K);
+int dsq_wgemm_bf16(const void *X_bf16, const void *W_codes, int64_t M, int64_t N,
+                   int64_t K, int bits, float w_offset, const float *col_scale,
+                   const float *col_bias, float *Y_f32, void *workspace,
+                   size_t ws_bytes, void *stream);
+
 /* dsq_gemm for callers that cannot allocate device memory.  (The paper has
  * no counterpart: this is a deployment convenience of the library.)
  *
@@ -297,7 +341,8 @@ int dsq_soft_quantize_bwd(const float *x, const float *grad_y, int64_t n,
 /* ---- format helpers (tests, tooling) ----------------------------------- */
 
 /* int8 codes [rows][k] (dense) -> packed rows.  Values are truncated to
- * their low `bits` bits. */
+ * their low `bits` bits.  bits in {1, 2, 3, 4} (1: the operands of
+ * dsq_binary_gemm and 1-bit weights of dsq_wgemm_bf16). */
 int dsq_pack_codes(const int8_t *codes, int64_t rows, int64_t k, int bits,
                    void *packed_out, size_t bytes, void *stream);
 

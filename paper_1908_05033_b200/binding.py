@@ -67,6 +67,11 @@ _SIGNATURES = {
     "dsq_gemm": (_int, [_vp, _vp, _i64, _i64, _i64, _int, _vp, _vp, _vp, _vp,
                         _sz, _vp]),
     "dsq_gemm_workspace_bytes": (_sz, [_i64, _i64, _i64, _int]),
+    "dsq_binary_gemm_workspace_bytes": (_sz, [_i64, _i64, _i64]),
+    "dsq_binary_gemm": (_int, [_vp, _vp, _i64, _i64, _i64, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "dsq_wgemm_workspace_bytes": (_sz, [_i64, _i64]),
+    "dsq_wgemm_bf16": (_int, [_vp, _vp, _i64, _i64, _i64, _int, C.c_float, _vp, _vp, _vp, _vp,
+                              _sz, _vp]),
     "dsq_gemm_static_ws": (_int, [_vp, _vp, _i64, _i64, _i64, _int, _vp, _vp, _vp,
                                   _int, _vp]),
     "dsq_maxpool2x2": (_int, [_vp, C.POINTER(dsq_nhwc_t), _int, _vp, _sz,
@@ -367,6 +372,42 @@ def dsq_gemm(A, B, M, N, K, bits, ws, row_scale=None, want_i32=True,
     _check(lib.dsq_gemm(_p(A), _p(B), M, N, K, bits, _p(Cm), _p(row_scale),
                         _p(D), _p(ws), ws.numel(), _stream()), "dsq_gemm")
     return Cm, D
+
+
+def _sized_workspace(nbytes, device):
+    ws = torch.empty(nbytes, dtype=torch.uint8, device=device)
+    _check(lib.dsq_workspace_init(_p(ws), ws.numel(), _stream()), "dsq_workspace_init")
+    return ws
+
+
+def dsq_binary_gemm(A, B, M, N, K, ws=None, row_scale=None, want_i32=True):
+    """A, B: packed 1-bit rows [M, pitch], [N, pitch] (bit 1 = +1, 0 = -1).
+    Returns (C int32 [M,N] | None, D fp32 [M,N] | None)."""
+    _need(A, torch.uint8, "A")
+    _need(B, torch.uint8, "B")
+    if ws is None:
+        ws = _sized_workspace(int(lib.dsq_binary_gemm_workspace_bytes(M, N, K)), A.device)
+    Cm = torch.empty((M, N), dtype=torch.int32, device=A.device) if want_i32 else None
+    D = torch.empty((M, N), dtype=torch.float32, device=A.device) if row_scale is not None else None
+    _check(lib.dsq_binary_gemm(_p(A), _p(B), M, N, K, _p(Cm), _p(row_scale), _p(D), _p(ws),
+                               ws.numel(), _stream()), "dsq_binary_gemm")
+    check_workspace(ws, "dsq_binary_gemm")
+    return Cm, D
+
+
+def dsq_wgemm_bf16(X, W, M, N, K, bits, col_scale, col_bias=None, w_offset=0.5, ws=None,
+                   out=None):
+    """X: bf16 [M, K]; W: packed signed codes [N, pitch].  Returns Y fp32 [M, N]."""
+    _need(X, torch.bfloat16, "X")
+    _need(W, torch.uint8, "W")
+    _need(col_scale, torch.float32, "col_scale")
+    if ws is None:
+        ws = _sized_workspace(int(lib.dsq_wgemm_workspace_bytes(N, K)), X.device)
+    Y = out if out is not None else torch.empty((M, N), dtype=torch.float32, device=X.device)
+    _check(lib.dsq_wgemm_bf16(_p(X), _p(W), M, N, K, bits, w_offset, _p(col_scale),
+                              _p(col_bias), _p(Y), _p(ws), ws.numel(), _stream()),
+           "dsq_wgemm_bf16")
+    return Y
 
 
 def dsq_set_round_k_steps(ks):

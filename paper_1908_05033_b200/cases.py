@@ -39,7 +39,7 @@ def _timeit(fn, iters, flush):
 
 def main(argv=None):
     ap = argparse.ArgumentParser()
-    ap.add_argument("case", choices=["gemm", "conv", "quant", "dw", "soft"])
+    ap.add_argument("case", choices=["gemm", "bgemm", "wgemm", "conv", "quant", "dw", "soft"])
     ap.add_argument("--size", type=int, default=4096)
     ap.add_argument("--bits", type=int, default=4)
     ap.add_argument("--iters", type=int, default=5)
@@ -84,6 +84,30 @@ def main(argv=None):
         ms, all_ms = _timeit(lambda: B.dsq_gemm(A, Bm, n, n, n, bits, ws, out_i32=Cm),
                              a.iters, flush)
         out.update(size=n, ms=ms, tops=2.0 * n ** 3 / (ms * 1e-3) / 1e12, all_ms=all_ms)
+    elif a.case == "bgemm":
+        # binary GEMM: 1-bit rows, values -1 / +1
+        n = a.size
+        pitch = B.dsq_row_pitch(n, 1)
+        A = torch.randint(0, 256, (n, pitch), dtype=torch.uint8, device=dev, generator=gen)
+        Bm = torch.randint(0, 256, (n, pitch), dtype=torch.uint8, device=dev, generator=gen)
+        Cm = torch.empty((n, n), dtype=torch.int32, device=dev)
+        ws = torch.zeros(B.lib.dsq_binary_gemm_workspace_bytes(n, n, n), dtype=torch.uint8, device=dev)
+        ms, all_ms = _timeit(lambda: B._check(B.lib.dsq_binary_gemm(
+            A.data_ptr(), Bm.data_ptr(), n, n, n, Cm.data_ptr(), None, None, ws.data_ptr(),
+            ws.numel(), torch.cuda.current_stream().cuda_stream), "dsq_binary_gemm"), a.iters, flush)
+        out.update(size=n, ms=ms, tops=2.0 * n ** 3 / (ms * 1e-3) / 1e12, all_ms=all_ms)
+    elif a.case == "wgemm":
+        # weight-only: bf16 activations [size, size] x b-bit weights [size, size]
+        n = a.size
+        X = torch.randn((n, n), device=dev, generator=gen).to(torch.bfloat16)
+        W = torch.randint(0, 256, (n, B.dsq_row_pitch(n, bits)), dtype=torch.uint8, device=dev,
+                          generator=gen)
+        sc = torch.full((n,), 0.01, device=dev)
+        Y = torch.empty((n, n), dtype=torch.float32, device=dev)
+        ws = torch.zeros(B.lib.dsq_wgemm_workspace_bytes(n, n), dtype=torch.uint8, device=dev)
+        ms, all_ms = _timeit(lambda: B.dsq_wgemm_bf16(X, W, n, n, n, bits, sc, ws=ws, out=Y),
+                             a.iters, flush)
+        out.update(size=n, ms=ms, tflops=2.0 * n ** 3 / (ms * 1e-3) / 1e12, all_ms=all_ms)
     elif a.case == "conv":
         shape = (a.batch, a.hw, a.hw, a.cin)
         pitch = B.dsq_row_pitch(a.cin, bits)

@@ -424,7 +424,7 @@ int dsq_pack_codes(const int8_t *codes, int64_t rows, int64_t k, int bits,
                    void *packed_out, size_t bytes, void *stream)
 {
     if (!codes || !packed_out) return DSQ_ERR_NULL;
-    if (bits < 2 || bits > 4) return DSQ_ERR_BITS;
+    if (bits < 1 || bits > 4) return DSQ_ERR_BITS;
     if (rows <= 0 || k <= 0 || k > (1 << 28)) return DSQ_ERR_SHAPE;
     if (!dsq_aligned16(packed_out)) return DSQ_ERR_ALIGN;
     const size_t pitch = dsq_row_pitch(k, bits);
@@ -439,7 +439,7 @@ int dsq_unpack(const void *packed, int64_t rows, int64_t k, int bits,
                int is_signed, int8_t *codes_out, void *stream)
 {
     if (!packed || !codes_out) return DSQ_ERR_NULL;
-    if (bits < 2 || bits > 4) return DSQ_ERR_BITS;
+    if (bits < 1 || bits > 4) return DSQ_ERR_BITS;
     if (rows <= 0 || k <= 0 || k > (1 << 28)) return DSQ_ERR_SHAPE;
     if (!dsq_aligned16(packed)) return DSQ_ERR_ALIGN;
     const int pw = (int)(dsq_row_pitch(k, bits) / 4);

@@ -485,6 +485,33 @@ __device__ __forceinline__ void mma_i8_ss_pair_x4_elect(uint32_t d_tmem, uint32_
         : "memory");
 }
 
+// Same for 16-bit floating-point operands (kind::f16: f16 or bf16 per the
+// instruction descriptor, K = 16 elements = 32 bytes per instruction, f32
+// accumulate).
+__device__ __forceinline__ void mma_f16_ss_pair_x4_elect(uint32_t d_tmem, uint32_t a_lo,
+                                                        uint32_t a_hi, uint32_t b_lo,
+                                                        uint32_t b_hi, uint32_t idesc,
+                                                        uint32_t accumulate_first)
+{
+    asm volatile(
+        "{\n\t.reg .pred p0, p1, pe;\n\t"
+        ".reg .b64 da0, da1, da2, da3, db0, db1, db2, db3;\n\t.reg .b32 x1, x2, x3, y1, y2, y3;\n\t"
+        "setp.ne.b32 p0, %6, 0;\n\tsetp.eq.b32 p1, %6, %6;\n\t"
+        "add.u32 x1, %1, 2;\n\tadd.u32 x2, %1, 4;\n\tadd.u32 x3, %1, 6;\n\t"
+        "add.u32 y1, %3, 2;\n\tadd.u32 y2, %3, 4;\n\tadd.u32 y3, %3, 6;\n\t"
+        "mov.b64 da0, {%1, %2};\n\tmov.b64 da1, {x1, %2};\n\t"
+        "mov.b64 da2, {x2, %2};\n\tmov.b64 da3, {x3, %2};\n\t"
+        "mov.b64 db0, {%3, %4};\n\tmov.b64 db1, {y1, %4};\n\t"
+        "mov.b64 db2, {y2, %4};\n\tmov.b64 db3, {y3, %4};\n\t"
+        "elect.sync _|pe, 0xffffffff;\n\t"
+        "@pe tcgen05.mma.cta_group::2.kind::f16 [%0], da0, db0, %5, p0;\n\t"
+        "@pe tcgen05.mma.cta_group::2.kind::f16 [%0], da1, db1, %5, p1;\n\t"
+        "@pe tcgen05.mma.cta_group::2.kind::f16 [%0], da2, db2, %5, p1;\n\t"
+        "@pe tcgen05.mma.cta_group::2.kind::f16 [%0], da3, db3, %5, p1;\n\t}" ::"r"(d_tmem),
+        "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate_first)
+        : "memory");
+}
+
 // tcgen05.commit by one elected lane of a converged warp (all lanes call).
 __device__ __forceinline__ void mma_commit_elect(uint32_t bar)
 {
@@ -594,6 +621,19 @@ __host__ __device__ inline uint32_t idesc_i8(int n, bool a_signed, bool b_signed
     d |= (b_signed ? 1u : 0u) << 10;           // B
     d |= (uint32_t)(n >> 3) << 17;             // N / 8
     d |= (uint32_t)(m >> 4) << 24;             // M / 16 (256: both CTAs of a pair)
+    return d;
+}
+
+// Instruction descriptor for kind::f16 with bf16 operands and an f32
+// accumulator, K-major A and B.
+__host__ __device__ inline uint32_t idesc_bf16(int n, int m = 128)
+{
+    uint32_t d = 0;
+    d |= 1u << 4;                              // D format: F32
+    d |= 1u << 7;                              // A: BF16
+    d |= 1u << 10;                             // B: BF16
+    d |= (uint32_t)(n >> 3) << 17;             // N / 8
+    d |= (uint32_t)(m >> 4) << 24;             // M / 16
     return d;
 }
 
