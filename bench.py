@@ -626,8 +626,47 @@ def run_ours(args):
             g2["path"] = "two passes (expand rows to int8, 8-bit GEMM); both timed"
             g2["fused_kernel"] = time_gemm(size, ws)
             extras[f"gemm_{size}_b4"] = g2
+        # binary GEMM (1-bit rows, +-1 values) and weight-only GEMM (bf16 x 4-bit)
+        Ab, Bb, _ = dsq_inputs.binary_gemm_case(4096, 4096, 4096)
+        Abp = dsq.dsq_pack_codes(torch.from_numpy(Ab).to(dev), 1)
+        Bbp = dsq.dsq_pack_codes(torch.from_numpy(Bb).to(dev), 1)
+        Cb = torch.empty((4096, 4096), dtype=torch.int32, device=dev)
+        bws = torch.zeros(dsq.lib.dsq_binary_gemm_workspace_bytes(4096, 4096, 4096),
+                          dtype=torch.uint8, device=dev)
+        xw, qw, uw, _ = dsq_inputs.weight_only_case(4096, 4096, 4096, 4)
+        Xw = torch.from_numpy(xw).to(dev).to(torch.bfloat16)
+        Ww = dsq.dsq_pack_codes(torch.from_numpy((qw.astype(np.int16) - 8).astype(np.int8)).to(dev), 4)
+        sw = torch.from_numpy((uw / 15).astype(np.float32)).to(dev)
+        Yw = torch.empty((4096, 4096), dtype=torch.float32, device=dev)
+        wws = torch.zeros(dsq.lib.dsq_wgemm_workspace_bytes(4096, 4096), dtype=torch.uint8, device=dev)
+        stream = torch.cuda.current_stream().cuda_stream
+
+        def run_bgemm():
+            st_ = dsq.lib.dsq_binary_gemm(Abp.data_ptr(), Bbp.data_ptr(), 4096, 4096, 4096,
+                                          Cb.data_ptr(), None, None, bws.data_ptr(), bws.numel(), stream)
+            assert st_ == 0
+
+        def time_call(fn):
+            times = []
+            for i in range(13):
+                flush.zero_()
+                e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+                e0.record(); fn(); e1.record(); torch.cuda.synchronize()
+                if i >= 3:
+                    times.append(e0.elapsed_time(e1))
+            return statistics.median(times)
+
+        bms = time_call(run_bgemm)
+        dsq.check_workspace(bws, "extras binary gemm")
+        extras["binary_gemm_4096"] = {"ms": bms, "tops": 2.0 * 4096 ** 3 / (bms * 1e-3) / 1e12,
+                                      "frac_of_nominal_4500": 2.0 * 4096 ** 3 / (bms * 1e-3) / 1e12 / INT8_NOMINAL_TOPS}
+        wms = time_call(lambda: dsq.dsq_wgemm_bf16(Xw, Ww, 4096, 4096, 4096, 4, sw, ws=wws, out=Yw))
+        dsq.check_workspace(wws, "extras weight-only gemm")
+        wt = 2.0 * 4096 ** 3 / (wms * 1e-3) / 1e12
+        extras["weight_only_gemm_4096_w4_bf16"] = {"ms": wms, "tflops": wt,
+                                                   "frac_of_bf16_burst": wt / peaks["bf16_tflops"]}
         dsq.check_workspace(ws, "extras")
-        del flush
+        del flush, Abp, Bbp, Cb, bws, Xw, Ww, Yw, wws
         extras["mobilenetv2_stack_b4_batch64"] = time_other_stack(
             dsq_inputs.mobilenetv2_stack(), 4, torch, dev)
         extras["vgg16_stack_b2_batch32"] = time_other_stack(dsq_inputs.vgg16_stack(), 5, torch, dev)

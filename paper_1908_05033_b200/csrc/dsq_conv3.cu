@@ -96,6 +96,7 @@ struct W3Params {
     int a_box, a_nload, nbands, band_px;
     int tap_stride;                    // slot rows between two filter rows
     int as_slots, bp_slots, b_stages, b_res;
+    int w8;                            // weight K steps come expanded, by TMA, into the operand ring
     int cout_pad;                      // Cout rounded up to the N tiling
     int tr;                            // transposed tiles (kernel form TR)
     int mstep;                         // M tiles between two tiles of a CTA
@@ -301,7 +302,7 @@ dsq_win3_kernel(const __grid_constant__ CUtensorMap tmap_b,
             mbar_init(bar_bp_empty(s), W3_B_GROUP_WARPS);
         }
         for (int s = 0; s < W3_MAX_BST; ++s) {
-            mbar_init(bar_b_full(s), W3_B_GROUP_WARPS);
+            mbar_init(bar_b_full(s), p.w8 ? 1 : W3_B_GROUP_WARPS);   // (w8: TMA producer + bytes)
             mbar_init(bar_b_empty(s), 1);            // tcgen05.commit
         }
         for (int s = 0; s < 2; ++s) {
@@ -347,7 +348,28 @@ dsq_win3_kernel(const __grid_constant__ CUtensorMap tmap_b,
 
     if (warp == W3_WARP_TMA_B) {
         // ---------------- producer: packed B rows of one K step ------------------
-        if (lane == 0) {
+        if (lane == 0 && p.w8) {
+            // weights already expanded (blob's int8 copy): K step g of this CTA's
+            // sequence goes straight into stage g % b_stages of the operand ring
+            uint32_t issued = 0, ph = 0;
+            const int BST = p.b_stages;
+            const int y = n_tile * BN;
+            int s = 0, x = 0;
+#pragma unroll 1
+            for (uint32_t g = 0; g < n_b_fills; ++g) {
+                if (!wait_bar(bar_b_empty(s), ph ^ 1u, ctl, 1)) break;
+                if ((int)g == p.skip_b_round) break;
+                mbar_arrive_expect_tx(bar_b_full(s), b_stage_bytes);
+                tma_load_2d(smem_u32(smem + L.b_tiles + s * b_stage_bytes), &tmap_b, x, y,
+                            bar_b_full(s));
+                ++issued;
+                x += 128;
+                if (x == p.ksteps * 128) x = 0;
+                if (++s == BST) { s = 0; ph ^= 1u; }
+            }
+            for (uint32_t k = (issued > (uint32_t)BST ? issued - BST : 0); k < issued; ++k)
+                wait_bar_drain(bar_b_full(k % BST), (k / BST) & 1u);
+        } else if (lane == 0) {
             uint32_t issued = 0, ph = 0;
             const int BP = p.bp_slots;
             const int y = n_tile * BN;
@@ -579,7 +601,7 @@ dsq_win3_kernel(const __grid_constant__ CUtensorMap tmap_b,
         // own fills: g = group, group + 2, ...
         int sp = group % BP, st = p.b_res ? group : group % BST;
         uint32_t php = (uint32_t)(group / BP) & 1u, phu = p.b_res ? 0u : (uint32_t)(group / BST) & 1u;
-        bool ok = true;
+        bool ok = !p.w8;                           // (w8: nothing to expand)
 #pragma unroll 1
         for (uint32_t g = group; ok && g < n_b_fills; g += 2) {
             if (!(ok = wait_bar_warp(bar_bp_full(sp), php, ctl, 6))) break;

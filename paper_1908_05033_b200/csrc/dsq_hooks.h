@@ -42,6 +42,11 @@ int dsq_set_wait_limit_ns(long long ns);
  * shared-memory address, so this gives wrong numbers). */
 int dsq_set_conv3_window(int mode);
 
+/* Window kernel: 1 = weight tiles come by TMA from the blob's pre-expanded
+ * int8 copy where it exists (default), 0 = always expand the packed rows in
+ * the kernel. */
+int dsq_set_conv3_expanded_weights(int on);
+
 /* dsq_gemm with a workspace large enough for the expanded operands: 1 = take
  * the two-pass path (default), 0 = always the fused kernel. */
 int dsq_set_gemm_two_pass(int on);

@@ -1446,6 +1446,7 @@ std::atomic<unsigned long long> g_wait_ns{WAIT_LIMIT_NS};   // dsq_set_wait_limi
 std::atomic<int> g_skip_b_round{-1};  // dsq_set_test_skip_b_round
 std::atomic<int> g_window3{1};        // dsq_set_conv3_window
 std::atomic<int> g_two_pass{1};       // dsq_set_gemm_two_pass
+std::atomic<int> g_w8{1};             // dsq_set_conv3_expanded_weights
 
 int pick_bn(int m_tiles, int ncols, int bits)
 {
@@ -1623,6 +1624,7 @@ DsqLaunchHooks dsq_launch_hooks()
     h.wait_ns = g_wait_ns.load();
     h.skip_b_round = g_skip_b_round.load();
     h.window3 = g_window3.load();
+    h.w8 = g_w8.load();
     return h;
 }
 
@@ -1732,6 +1734,12 @@ size_t dsq_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int bits)
     if (bits < 2 || bits > 4 || M <= 0 || N <= 0 || K <= 0) return DSQ_WS_BYTES;
     const size_t need = dsq_gemm8_scratch_bytes(M, N, K);
     return need ? DSQ_WS_BYTES + 1024 + need : DSQ_WS_BYTES;
+}
+
+int dsq_set_conv3_expanded_weights(int on)
+{
+    g_w8 = on ? 1 : 0;
+    return DSQ_OK;
 }
 
 int dsq_set_gemm_two_pass(int on)

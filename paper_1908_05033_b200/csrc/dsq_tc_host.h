@@ -15,6 +15,7 @@ struct DsqLaunchHooks {
     unsigned long long wait_ns; // limit of the device-side waits
     int skip_b_round;           // test hook, -1 = off
     int window3;                // dsq_set_conv3_window
+    int w8;                     // dsq_set_conv3_expanded_weights
 };
 DSQ_HIDDEN DsqLaunchHooks dsq_launch_hooks();
 
@@ -55,3 +56,16 @@ DSQ_HIDDEN int dsq_gemm8_launch(const void *A_codes, const void *B_codes, int64_
                                 int64_t K, int bits, int32_t *C_i32, const float *row_scale,
                                 float *D_f32, void *workspace, void *scratch,
                                 cudaStream_t stream);
+
+// Weights of 3x3 stride-1 pad-1 dense convolutions (2- and 4-bit, 64 or a
+// multiple of 128 input channels) are stored twice in the blob
+// dsq_pack_weights writes: the packed rows, and behind them (1024-byte
+// aligned) the same rows already expanded to the int8 bytes the tensor core
+// multiplies for the grid Delta (c + 1/2), laid out K step by K step in the
+// order the window kernel consumes them (Cout rows of ksteps x 128 bytes).
+// The kernel then copies weight tiles by TMA straight into the swizzled operand
+// ring, with no expansion warps.  enabled = 0: this geometry has no such copy.
+struct DsqW8Info { int enabled; size_t offset; int ksteps; size_t bytes; };
+DSQ_HIDDEN DsqW8Info dsq_w8_info(const dsq_conv_t *conv, int bits);
+// builds the expanded copy from the packed rows at the start of `blob`
+DSQ_HIDDEN int dsq_w8_build(void *blob, const dsq_conv_t *conv, int bits, cudaStream_t stream);
