@@ -96,6 +96,7 @@ _HOOKS = {
     "dsq_set_test_skip_b_round": (_int, [_int]),
     "dsq_set_conv3_window": (_int, [_int]),
     "dsq_set_gemm_two_pass": (_int, [_int]),
+    "dsq_set_conv3_expanded_weights": (_int, [_int]),
 }
 for _name, (_res, _args) in list(_SIGNATURES.items()) + list(_HOOKS.items()):
     _f = getattr(lib, _name)       # AttributeError if a symbol is missing
@@ -412,6 +413,10 @@ def dsq_wgemm_bf16(X, W, M, N, K, bits, col_scale, col_bias=None, w_offset=0.5, 
 
 def dsq_set_round_k_steps(ks):
     _check(lib.dsq_set_round_k_steps(ks), "dsq_set_round_k_steps")
+
+
+def dsq_set_conv3_expanded_weights(on):
+    _check(lib.dsq_set_conv3_expanded_weights(int(on)), "dsq_set_conv3_expanded_weights")
 
 
 def dsq_set_gemm_two_pass(on):

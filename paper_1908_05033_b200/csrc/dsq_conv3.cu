@@ -1039,6 +1039,78 @@ int w3_dispatch(int epi, const CUtensorMap &tb, const CUtensorMap &ta, const W3P
 
 }  // namespace
 
+// ---------------------------------------------------------------------------
+// pre-expanded weights
+// ---------------------------------------------------------------------------
+namespace {
+
+// One thread per (row, K step, packed 16-byte chunk): the chunk's OUT int8
+// chunks, in the operand's logical order (TMA applies the 128-byte swizzle when
+// it copies a tile).  Same expansion as the kernel's own (expand_word), for the
+// grid Delta (c + 1/2); bytes past the end of a weight row read as packed
+// zeros, as the kernel's TMA loads of the packed rows do.
+template <int BITS>
+__global__ void __launch_bounds__(256)
+w8_build_kernel(const uint8_t *__restrict__ packed, uint8_t *__restrict__ out, int Cout,
+                int row_bytes, int ksteps, int kpp, int xstep)
+{
+    constexpr int CH = Chunks<BITS>::CH, OUT = Chunks<BITS>::OUT;
+    const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int j = (int)(idx % CH);
+    const int ks = (int)((idx / CH) % ksteps);
+    const int64_t row = idx / ((int64_t)CH * ksteps);
+    if (row >= Cout) return;
+    const int pl = ks / kpp, kk = ks - pl * kpp;
+    const int x = kk * xstep + pl * 16 * BITS + 16 * j;        // byte offset in the packed row
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if (x < row_bytes) v = *reinterpret_cast<const uint4 *>(packed + row * row_bytes + x);
+    const uint32_t orv = 0x01010101u << (7 - BITS);
+    uint8_t *dst = out + (row * ksteps + ks) * 128;
+#pragma unroll
+    for (int c = 0; c < OUT; ++c)
+        *reinterpret_cast<uint4 *>(dst + 16 * (j * OUT + c)) =
+            make_uint4(expand_word<BITS, true>(v.x, c, orv), expand_word<BITS, true>(v.y, c, orv),
+                       expand_word<BITS, true>(v.z, c, orv), expand_word<BITS, true>(v.w, c, orv));
+}
+
+}  // namespace
+
+DsqW8Info dsq_w8_info(const dsq_conv_t *conv, int bits)
+{
+    DsqW8Info w = {0, 0, 0, 0};
+    if (!conv || conv->groups != 1 || conv->KH != 3 || conv->KW != 3 || conv->stride != 1 ||
+        conv->pad != 1 || (bits != 2 && bits != 4))
+        return w;
+    const int Cin = conv->Cin;
+    if (!(Cin == 64 || (Cin % 128 == 0 && Cin <= 1024))) return w;
+    const int npl = Cin == 64 ? 1 : Cin / 128;
+    w.enabled = 1;
+    w.ksteps = npl * (Cin == 64 ? 5 : 9);
+    const size_t packed = (size_t)conv->Cout * 9 * dsq_row_pitch(Cin, bits);
+    w.offset = (packed + 1023) / 1024 * 1024;
+    w.bytes = (size_t)conv->Cout * w.ksteps * 128;
+    return w;
+}
+
+int dsq_w8_build(void *blob, const dsq_conv_t *conv, int bits, cudaStream_t stream)
+{
+    const DsqW8Info w = dsq_w8_info(conv, bits);
+    if (!w.enabled) return DSQ_OK;
+    const int Cin = conv->Cin;
+    const int P = (int)dsq_row_pitch(Cin, bits);
+    const int kpp = Cin == 64 ? 5 : 9;
+    const int xstep = Cin == 64 ? 16 * bits : P;
+    const int64_t threads = (int64_t)conv->Cout * w.ksteps * bits;       // CH = bits
+    const unsigned blocks = (unsigned)((threads + 255) / 256);
+    const uint8_t *packed = (const uint8_t *)blob;
+    uint8_t *out = (uint8_t *)blob + w.offset;
+    if (bits == 4)
+        w8_build_kernel<4><<<blocks, 256, 0, stream>>>(packed, out, conv->Cout, 9 * P, w.ksteps, kpp, xstep);
+    else
+        w8_build_kernel<2><<<blocks, 256, 0, stream>>>(packed, out, conv->Cout, 9 * P, w.ksteps, kpp, xstep);
+    return cudaGetLastError() == cudaSuccess ? DSQ_OK : DSQ_ERR_CUDA;
+}
+
 int dsq_conv3_window(const void *act_codes, const dsq_nhwc_t *shape, int bits,
                      const void *w_packed, const dsq_conv_t *conv, const DsqEpi &e,
                      int epi_kind, int small_acc, void *workspace, cudaStream_t stream)
@@ -1088,6 +1160,10 @@ int dsq_conv3_window(const void *act_codes, const dsq_nhwc_t *shape, int bits,
     // Tiling, window and shared memory for one of the two kernel forms.
     // Transposed (tr): tiles of 256 positions x 128 output channels, A = weights.
     // Plain: 128 positions x up to 256 channels, A = window.
+    const DsqW8Info w8 = dsq_w8_info(conv, bits);
+    // (up to 64 output channels the expanded weights stay resident in shared
+    // memory for the whole CTA anyway: nothing to gain, measured slightly slower)
+    p.w8 = hooks.w8 && w8.enabled && e.half_offset && bits != 3 && Cout > 64;
     auto configure = [&](int tr) -> int {
         p.tr = tr;
         const int tile_pos = tr ? 256 : W3_BM;
@@ -1118,15 +1194,28 @@ int dsq_conv3_window(const void *act_codes, const dsq_nhwc_t *shape, int bits,
         p.b_res = 0;
         if (p.ksteps <= W3_MAX_BST) {
             for (int as = W3_MAX_AS; as >= 2; --as) {
-                const W3Smem L = w3_layout(p.apx, p.BN, bits, p.PB, as, p.ksteps, 2, p.cout_pad);
+                const int bp = p.w8 ? 0 : 2;
+                const W3Smem L = w3_layout(p.apx, p.BN, bits, p.PB, as, p.ksteps, bp, p.cout_pad);
                 if (L.total + 1024 <= 227u * 1024u) {
-                    p.b_res = 1; p.b_stages = p.ksteps; p.as_slots = as; p.bp_slots = 2;
+                    p.b_res = 1; p.b_stages = p.ksteps; p.as_slots = as; p.bp_slots = bp;
                     return 1;
                 }
             }
         }
         // {A staging slots, expanded B stages, packed B slots}: the packed ring is
         // what hides the latency of the weight loads, so it goes first
+        if (p.w8) {
+            // no packed ring: the operand ring itself hides the latency of the loads
+            for (int as = W3_MAX_AS; as >= 1; --as)
+                for (int bst = 6; bst >= 2; --bst) {
+                    const W3Smem L = w3_layout(p.apx, p.BN, bits, p.PB, as, bst, 0, p.cout_pad);
+                    if (L.total + 1024 <= 227u * 1024u) {
+                        p.as_slots = as; p.b_stages = bst; p.bp_slots = 0;
+                        return 1;
+                    }
+                }
+            return 0;
+        }
         const int tries[6][3] = {{3, 3, 4}, {2, 3, 4}, {2, 2, 4}, {2, 2, 3}, {2, 2, 2}, {1, 2, 2}};
         for (int t = 0; t < 6; ++t) {
             const W3Smem L = w3_layout(p.apx, p.BN, bits, p.PB, tries[t][0], tries[t][1],
@@ -1189,7 +1278,19 @@ int dsq_conv3_window(const void *act_codes, const dsq_nhwc_t *shape, int bits,
     DsqEncodeIm2colFn enc_i2c = dsq_encode_im2col_fn();
     if (!enc || !enc_i2c) return DSQ_ERR_CUDA;
     CUtensorMap tb, ta;
-    {
+    if (p.w8) {
+        // the blob's expanded copy: Cout rows of ksteps x 128 bytes; one box = BN
+        // rows x one K step, swizzled on the way in
+        cuuint64_t dims[2] = {(cuuint64_t)p.ksteps * 128, (cuuint64_t)Cout};
+        cuuint64_t strides[1] = {(cuuint64_t)p.ksteps * 128};
+        cuuint32_t box[2] = {128u, (cuuint32_t)p.BN};
+        cuuint32_t estr[2] = {1, 1};
+        if (enc(&tb, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2,
+                const_cast<uint8_t *>((const uint8_t *)w_packed + w8.offset), dims, strides, box,
+                estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return DSQ_ERR_CUDA;
+    } else {
         cuuint64_t dims[2] = {(cuuint64_t)9 * P, (cuuint64_t)Cout};
         cuuint64_t strides[1] = {(cuuint64_t)9 * P};
         cuuint32_t box[2] = {(cuuint32_t)(16 * bits), (cuuint32_t)p.BN};

@@ -2,6 +2,7 @@
 // (Algorithm 1 steps 1 and 3), weight quantise + pack, code pack / unpack,
 // 2x2 max-pool on codes.  All are HBM-bound streaming kernels.
 #include "dsq_common.cuh"
+#include "dsq_tc_host.h"
 
 namespace {
 
@@ -326,8 +327,12 @@ size_t dsq_packed_bytes(int64_t rows, int64_t k, int bits)
 size_t dsq_weight_bytes(const dsq_conv_t *c, int bits)
 {
     if (!c || c->Cout <= 0 || c->Cin <= 0 || c->KH <= 0 || c->KW <= 0) return 0;
-    if (c->groups == 1)
+    if (c->groups == 1) {
+        // (some geometries carry a second, pre-expanded copy behind the packed rows)
+        const DsqW8Info w8 = dsq_w8_info(c, bits);
+        if (w8.enabled) return w8.offset + w8.bytes;
         return dsq_packed_bytes((int64_t)c->Cout * c->KH * c->KW, c->Cin, bits);
+    }
     if (c->groups == c->Cin && c->Cin == c->Cout)
         return dsq_packed_bytes((int64_t)c->KH * c->KW, c->Cout, bits);
     return 0;
@@ -417,7 +422,9 @@ int dsq_pack_weights(const float *w, const dsq_conv_t *c, int bits,
                           (cudaStream_t)stream>>>(
         w, (uint32_t *)packed_out, rows, k, pw, bits, taps, dw ? 1 : 0, lo, hi,
         per_channel ? 1 : 0, (int *)workspace);
-    return dsq_launch_status();
+    int st = dsq_launch_status();
+    if (st == DSQ_OK && dense) st = dsq_w8_build(packed_out, c, bits, (cudaStream_t)stream);
+    return st;
 }
 
 int dsq_pack_codes(const int8_t *codes, int64_t rows, int64_t k, int bits,

@@ -105,7 +105,10 @@ def test_workload_1_single_3x3_conv(dsq):
                           native.pack_rows(qa.reshape(-1, 64), bits))
     blob, conv = dsq.dsq_pack_weights(T(c["w"]), bits, c["w_lo"], c["w_hi"], ws,
                                       stride=1, pad=1)
-    assert blob.numel() == 18432
+    # packed rows first (18432 bytes), then the rows expanded to int8 K step by K step
+    assert blob.numel() == 18432 + 64 * 5 * 128
+    assert np.array_equal(N(blob)[:18432].reshape(64 * 9, 32),
+                          native.pack_rows(cw.reshape(64 * 9, 64), bits))
     _, yg, accg = dsq.dsq_conv2d(act, c["x"].shape, (bits, c["act_lo"], c["act_hi"]),
                                  blob, conv, T(c["scale"]), T(c["bias"]), ws,
                                  want_f32=True, want_acc=True)
@@ -228,10 +231,11 @@ WINDOW_GEOMS = [  # N, H, W, Cin, Cout: 3x3, stride 1, pad 1 on the shared-memor
     (1, 6, 300, 128, 72), (2, 56, 56, 128, 128), (70, 5, 5, 64, 96)]
 
 
+@pytest.mark.parametrize("w8", [1, 0])
 @pytest.mark.parametrize("form", [3, 4])
 @pytest.mark.parametrize("bits", [2, 3, 4])
 @pytest.mark.parametrize("geom", WINDOW_GEOMS)
-def test_conv3x3_window_kernel(dsq, geom, bits, form):
+def test_conv3x3_window_kernel(dsq, geom, bits, form, w8):
     """3x3 stride-1 convolutions whose A operand is an expanded window of the
     input in shared memory (one constant row shift per filter tap): image sizes
     from 1x1 to wider than a window, tiles that span several images, channel
@@ -239,17 +243,21 @@ def test_conv3x3_window_kernel(dsq, geom, bits, form):
     and without a residual operand, every element against the oracle.  Both
     forms of the kernel: form 3 = transposed tiles (256 positions x 128
     channels, weights as the A operand) where the geometry allows, form 4 =
-    plain tiles only (128 positions x up to 256 channels)."""
+    plain tiles only (128 positions x up to 256 channels).  w8 = 1: weight
+    tiles of the wide layers come by TMA from the blob's pre-expanded int8 copy
+    (grid Delta (c + 1/2) only); w8 = 0: the kernel expands the packed rows."""
     n, h, w, ci, co = geom
-    if bits == 3 and form == 4:
-        pytest.skip("3-bit codes take the plain form in both settings")
+    if bits == 3 and (form == 4 or w8 == 0):
+        pytest.skip("3-bit codes take the plain form and packed weights in every setting")
     dsq.dsq_set_conv3_window(form)     # this kernel wherever the geometry allows
+    dsq.dsq_set_conv3_expanded_weights(w8)
     try:
         conv_case(dsq, n, h, w, ci, co, 3, 1, 1, bits, 0.5, residual=(n % 2 == 0),
                   seed=n + h + ci)
         conv_case(dsq, n, h, w, ci, co, 3, 1, 1, bits, 0.0, per_channel=True, seed=co)
     finally:
         dsq.dsq_set_conv3_window(1)
+        dsq.dsq_set_conv3_expanded_weights(1)
 
 
 @pytest.mark.parametrize("bits", [2, 3, 4])

@@ -43,7 +43,13 @@ def test_size_queries():
     assert dsq.dsq_row_pitch(0, 4) == 0
     assert dsq.dsq_packed_bytes(10, 64, 4) == 320
     conv = B.dsq_conv_t(64, 3, 3, 64, 1, 1, 1)
-    assert dsq.dsq_weight_bytes(conv, 4) == 64 * 9 * 32      # config 1: 18432
+    # config 1: 18432 bytes of packed rows + (3x3, stride 1, pad 1 only) the rows
+    # expanded to int8, 5 K steps of 128 bytes each
+    assert dsq.dsq_weight_bytes(conv, 4) == 64 * 9 * 32 + 64 * 5 * 128
+    assert dsq.dsq_weight_bytes(B.dsq_conv_t(64, 3, 3, 64, 2, 1, 1), 4) == 64 * 9 * 32
+    assert dsq.dsq_weight_bytes(B.dsq_conv_t(64, 3, 3, 64, 1, 1, 1), 3) == 64 * 9 * 32
+    assert dsq.dsq_weight_bytes(B.dsq_conv_t(128, 3, 3, 256, 1, 1, 1), 2) == \
+        128 * 9 * 64 + 128 * 18 * 128
     dw = B.dsq_conv_t(96, 3, 3, 96, 1, 1, 96)
     assert dsq.dsq_weight_bytes(dw, 4) == 9 * 48
     assert dsq.dsq_workspace_bytes() >= 16
