@@ -218,7 +218,7 @@ int dsq_gemm(const void *A_codes, const void *B_codes, int64_t M, int64_t N,
  * dsq_workspace_bytes() works (one fused kernel that expands the packed codes
  * tile by tile).  Given this many bytes (the status words, then room for both
  * operands as 8-bit rows: about (M + N) * K bytes), large problems (M, N, K >=
- * 1024) take two passes instead: every packed row is expanded to 8-bit lanes
+ * 1024 and M N K >= 2^35) take two passes instead: every packed row is expanded to 8-bit lanes
  * once, then an 8-bit tensor-core GEMM reads the rows by TMA.  Same results
  * bit for bit.  The area behind the first dsq_workspace_bytes() bytes is
  * scratch: its contents after the call are unspecified, and calls that may

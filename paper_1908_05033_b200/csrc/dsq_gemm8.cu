@@ -126,24 +126,30 @@ expand_rows_kernel(const uint8_t *__restrict__ A, const uint8_t *__restrict__ B,
                    int64_t N, int pitch_in, int pitch_out, uint8_t *__restrict__ A8,
                    uint8_t *__restrict__ B8)
 {
+    // lets the second pass (queued behind with programmatic dependent launch)
+    // set itself up while this grid runs; it waits for this grid to complete
+    // before its first copy
+    grid_launch_dependents();
     const int cpr = pitch_out >> 4;                       // 16-byte chunks per output row
-    const int qpr = (cpr + 3) >> 2;                       // threads per row
-    const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    const int64_t row = idx / qpr;
-    const int c0 = (int)(idx - row * qpr) * 4;
-    if (row >= M + N) return;
-    const bool is_a = row < M;                            // A: signed codes, B: unsigned
-    const uint8_t *src = is_a ? A + row * pitch_in : B + (row - M) * pitch_in;
-    uint8_t *dst = is_a ? A8 + row * pitch_out : B8 + (row - M) * pitch_out;
-    uint4 o[4];
+    const int qpr = (cpr + 3) >> 2;                       // work items per row
+    const int64_t total = (M + N) * qpr;
+    for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
+         idx += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t row = idx / qpr;
+        const int c0 = (int)(idx - row * qpr) * 4;
+        const bool is_a = row < M;                        // A: signed codes, B: unsigned
+        const uint8_t *src = is_a ? A + row * pitch_in : B + (row - M) * pitch_in;
+        uint8_t *dst = is_a ? A8 + row * pitch_out : B8 + (row - M) * pitch_out;
+        uint4 o[4];
 #pragma unroll
-    for (int j = 0; j < 4; ++j)
-        if (c0 + j < cpr)
-            o[j] = expand_chunk<BITS>(src + (c0 + j) * (2 * BITS), pitch_in - (c0 + j) * (2 * BITS),
-                                      is_a);
+        for (int j = 0; j < 4; ++j)
+            if (c0 + j < cpr)
+                o[j] = expand_chunk<BITS>(src + (c0 + j) * (2 * BITS),
+                                          pitch_in - (c0 + j) * (2 * BITS), is_a);
 #pragma unroll
-    for (int j = 0; j < 4; ++j)
-        if (c0 + j < cpr) *reinterpret_cast<uint4 *>(dst + (c0 + j) * 16) = o[j];
+        for (int j = 0; j < 4; ++j)
+            if (c0 + j < cpr) *reinterpret_cast<uint4 *>(dst + (c0 + j) * 16) = o[j];
+    }
 }
 
 // Binary operands (Eq. 1): bit 1 -> +1, bit 0 -> -1; positions past K -> 0, so
@@ -519,10 +525,13 @@ inline uint8_t *scratch_of(void *workspace)
 
 // Scratch the two-pass path needs behind the status words (0: the problem is
 // one the fused kernel keeps).
-size_t dsq_gemm8_scratch_bytes(int64_t M, int64_t N, int64_t K)
+size_t dsq_gemm8_scratch_bytes(int64_t M, int64_t N, int64_t K, int force)
 {
-    // below this the fused kernel's single launch wins (measured)
-    if (M < 1024 || N < 1024 || K < 1024) return 0;
+    // below this the fused kernel's single launch wins (measured: 2048^3 takes
+    // 22.5 us fused and 25.6 us in two passes, 4096^3 85 and 71 us)
+    if (!force && (M < 1024 || N < 1024 || K < 1024 ||
+                   (double)M * (double)N * (double)K < 34359738368.0 /* 2^35 */))
+        return 0;
     const size_t kp = round_up((size_t)K, 16);
     return round_up((size_t)M * kp, 1024) + round_up((size_t)N * kp, 1024);
 }
@@ -537,7 +546,9 @@ int dsq_gemm8_launch(const void *A_codes, const void *B_codes, int64_t M, int64_
     uint8_t *B8 = A8 + round_up((size_t)M * kp, 1024);
     const int pitch_in = (int)dsq_row_pitch(K, bits);
     const int64_t threads = (M + N) * (int64_t)((kp / 16 + 3) / 4);
-    const unsigned blocks = (unsigned)((threads + 255) / 256);
+    const int sms = dsq_sm_count() > 0 ? dsq_sm_count() : 148;
+    // whole waves of resident blocks (8 per SM), a few items per thread
+    const unsigned blocks = (unsigned)std::min<int64_t>((threads + 255) / 256, (int64_t)sms * 8);
     const uint8_t *A = (const uint8_t *)A_codes, *B = (const uint8_t *)B_codes;
     switch (bits) {
     case 2: expand_rows_kernel<2><<<blocks, 256, 0, stream>>>(A, B, M, N, pitch_in, (int)kp, A8, B8); break;

@@ -48,7 +48,9 @@ int dsq_set_conv3_window(int mode);
 int dsq_set_conv3_expanded_weights(int on);
 
 /* dsq_gemm with a workspace large enough for the expanded operands: 1 = take
- * the two-pass path (default), 0 = always the fused kernel. */
+ * the two-pass path where it is the faster one (default: M, N, K >= 1024 and
+ * M N K >= 2^35), 0 = always the fused kernel, 2 = two passes whatever the
+ * size (dsq_gemm_workspace_bytes answers accordingly). */
 int dsq_set_gemm_two_pass(int on);
 
 /* Test hook: in every later launch the thread that issues the TMA copies of

@@ -65,17 +65,35 @@ __global__ void __launch_bounds__(256) soft_fwd_kernel(const float *__restrict__
     for (int64_t i = 4 * n4 + tid; i < n; i += stride) y[i] = soft_fwd_one(x[i], p);
 }
 
+// tanh(z) and sech^2(z) from one exponential and one reciprocal (the special
+// function unit's ex2 and rcp, each good to about 2^-22 relative):
+//   e = exp(2 z), r = 1/(e + 1):  tanh = 1 - 2 r,  sech^2 = 4 e r^2
+// sech^2 has no cancellation (relative error ~1e-6); tanh is good to ~1e-6
+// absolute, and it only enters sums next to terms of order one.  z -> +inf:
+// e = inf, r = 0, tanh = 1 and sech^2 is forced to 0; z -> -inf: e = 0.
+__device__ __forceinline__ void tanh_sech2(float z, float &t, float &sech2)
+{
+    float e, r;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(z * 2.885390081777927f));   // 2 log2(e)
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(e + 1.0f));
+    t = fmaf(-2.0f, r, 1.0f);
+    sech2 = r == 0.0f ? 0.0f : 4.0f * e * r * r;
+}
+
 // one element of the backward pass: returns dL/dx, adds this element's terms
-// of dL/dalpha, dL/dl, dL/du (times g) to the accumulators
-__device__ __forceinline__ float soft_bwd_one(float x, float g, const SoftP &p, double &aa,
-                                              double &al, double &au)
+// of dL/dalpha, dL/dl, dL/du (times g) to the accumulators (binary32 partial
+// sums of a few elements; the caller folds them into binary64)
+__device__ __forceinline__ float soft_bwd_one(float x, float g, const SoftP &p, float &aa,
+                                              float &al, float &au)
 {
     if (x != x) return x;
-    if (x < p.lo) { al += (double)g; return 0.0f; }
-    if (x > p.hi) { au += (double)g; return 0.0f; }
-    float fi, t, xm;
-    soft_core(x, p, fi, t, xm);
-    const float sech2 = fmaf(-t, t, 1.0f);
+    if (x < p.lo) { al += g; return 0.0f; }
+    if (x > p.hi) { au += g; return 0.0f; }
+    const float xc = x;
+    const float fi = fminf(fmaxf(floorf((xc - p.lo) * p.inv_delta), 0.0f), (float)p.imax);
+    const float xm = xc - fmaf(fi + 0.5f, p.delta, p.lo);
+    float t, sech2;
+    tanh_sech2(p.k * xm, t, sech2);
     const float q = fi + fmaf(0.5f * p.s, t, 0.5f);                  // Eq. 13
     // Eq. 10: (Delta/2) (ds/da tanh + s sech^2 (x - m) dk/da)
     const float da = 0.5f * p.delta * fmaf(p.ds_da, t, p.s * sech2 * xm * p.dk_da);
@@ -86,9 +104,9 @@ __device__ __forceinline__ float soft_bwd_one(float x, float g, const SoftP &p, 
     const float dphi_du = ssech * (-p.k_over_delta * p.dd_du * xm - p.k * dm_du);
     const float dl = 1.0f + fmaf(q, p.dd_dl, 0.5f * p.delta * dphi_dl);
     const float du = fmaf(q, p.dd_du, 0.5f * p.delta * dphi_du);
-    aa += (double)(g * da);
-    al += (double)(g * dl);
-    au += (double)(g * du);
+    aa = fmaf(g, da, aa);
+    al = fmaf(g, dl, al);
+    au = fmaf(g, du, au);
     return g * p.half_dsk * sech2;
 }
 
@@ -105,14 +123,19 @@ __global__ void __launch_bounds__(256) soft_bwd_kernel(const float *__restrict__
         const float4 v = ld_stream(reinterpret_cast<const float4 *>(x) + i);
         const float4 g = ld_stream(reinterpret_cast<const float4 *>(gy) + i);
         float4 o;
-        o.x = soft_bwd_one(v.x, g.x, p, aa, al, au);
-        o.y = soft_bwd_one(v.y, g.y, p, aa, al, au);
-        o.z = soft_bwd_one(v.z, g.z, p, aa, al, au);
-        o.w = soft_bwd_one(v.w, g.w, p, aa, al, au);
+        float fa = 0.0f, fl = 0.0f, fu = 0.0f;          // this vector's four terms
+        o.x = soft_bwd_one(v.x, g.x, p, fa, fl, fu);
+        o.y = soft_bwd_one(v.y, g.y, p, fa, fl, fu);
+        o.z = soft_bwd_one(v.z, g.z, p, fa, fl, fu);
+        o.w = soft_bwd_one(v.w, g.w, p, fa, fl, fu);
+        aa += (double)fa; al += (double)fl; au += (double)fu;
         __stcs(reinterpret_cast<float4 *>(gx) + i, o);
     }
-    for (int64_t i = 4 * n4 + tid; i < n; i += stride)
-        gx[i] = soft_bwd_one(x[i], gy[i], p, aa, al, au);
+    for (int64_t i = 4 * n4 + tid; i < n; i += stride) {
+        float fa = 0.0f, fl = 0.0f, fu = 0.0f;
+        gx[i] = soft_bwd_one(x[i], gy[i], p, fa, fl, fu);
+        aa += (double)fa; al += (double)fl; au += (double)fu;
+    }
     // the three sums: warp shuffles, one shared-memory pass per block, one
     // double-precision atomic add per block and sum
 #pragma unroll

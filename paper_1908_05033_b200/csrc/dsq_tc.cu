@@ -1732,7 +1732,8 @@ static int gemm_check_args(const void *A_codes, const void *B_codes, int64_t M, 
 size_t dsq_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int bits)
 {
     if (bits < 2 || bits > 4 || M <= 0 || N <= 0 || K <= 0) return DSQ_WS_BYTES;
-    const size_t need = dsq_gemm8_scratch_bytes(M, N, K);
+    const int mode = g_two_pass.load();
+    const size_t need = mode ? dsq_gemm8_scratch_bytes(M, N, K, mode == 2) : 0;
     return need ? DSQ_WS_BYTES + 1024 + need : DSQ_WS_BYTES;
 }
 
@@ -1744,7 +1745,8 @@ int dsq_set_conv3_expanded_weights(int on)
 
 int dsq_set_gemm_two_pass(int on)
 {
-    g_two_pass = on ? 1 : 0;
+    if (on < 0 || on > 2) return DSQ_ERR_SHAPE;
+    g_two_pass = on;
     return DSQ_OK;
 }
 
@@ -1761,7 +1763,8 @@ int dsq_gemm(const void *A_codes, const void *B_codes, int64_t M, int64_t N, int
     // large problems, when the caller's workspace has room for the expanded
     // operands (dsq_gemm_workspace_bytes): expand every row once, then an
     // 8-bit GEMM fed by TMA alone
-    const size_t scratch_need = g_two_pass.load() ? dsq_gemm8_scratch_bytes(M, N, K) : 0;
+    const int two_pass = g_two_pass.load();
+    const size_t scratch_need = two_pass ? dsq_gemm8_scratch_bytes(M, N, K, two_pass == 2) : 0;
     if (scratch_need) {
         const uintptr_t w0 = reinterpret_cast<uintptr_t>(workspace);
         const uintptr_t s0 = (w0 + DSQ_WS_BYTES + 1023u) & ~(uintptr_t)1023u;

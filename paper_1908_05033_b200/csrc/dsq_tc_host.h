@@ -48,10 +48,11 @@ DSQ_HIDDEN int dsq_conv3_window(const void *act_codes, const dsq_nhwc_t *shape, 
 
 // Two-pass GEMM (dsq_gemm8.cu): every packed row is expanded to int8 once
 // into caller-provided scratch, then an 8-bit GEMM reads it by TMA.
-// dsq_gemm8_scratch_bytes: scratch the path needs (0: not a problem it takes).
+// dsq_gemm8_scratch_bytes: scratch the path needs (0: not a problem it takes;
+// force: whatever the size).
 // dsq_gemm8_launch: arguments as dsq_gemm after validation, `scratch`
 // 1024-byte aligned and at least that large.
-DSQ_HIDDEN size_t dsq_gemm8_scratch_bytes(int64_t M, int64_t N, int64_t K);
+DSQ_HIDDEN size_t dsq_gemm8_scratch_bytes(int64_t M, int64_t N, int64_t K, int force);
 DSQ_HIDDEN int dsq_gemm8_launch(const void *A_codes, const void *B_codes, int64_t M, int64_t N,
                                 int64_t K, int bits, int32_t *C_i32, const float *row_scale,
                                 float *D_f32, void *workspace, void *scratch,

@@ -93,19 +93,23 @@ def run_two_pass(dsq, A, B, rs, bits, want_i32=True):
     """dsq_gemm with a workspace that has room for the expanded operands."""
     M, K = A.shape
     Nn = B.shape[0]
-    assert dsq.dsq_gemm_workspace_bytes(M, Nn, K, bits) > dsq.dsq_workspace_bytes()
-    ws = dsq.new_gemm_workspace(M, Nn, K, bits)
-    Ap, Bp = dsq.dsq_pack_codes(T(A), bits), dsq.dsq_pack_codes(T(B), bits)
-    Cg, Dg = dsq.dsq_gemm(Ap, Bp, M, Nn, K, bits, ws, row_scale=T(rs), want_i32=want_i32)
-    assert dsq.dsq_workspace_status(ws) == 0
+    dsq.dsq_set_gemm_two_pass(2)          # two passes whatever the size
+    try:
+        assert dsq.dsq_gemm_workspace_bytes(M, Nn, K, bits) > dsq.dsq_workspace_bytes()
+        ws = dsq.new_gemm_workspace(M, Nn, K, bits)
+        Ap, Bp = dsq.dsq_pack_codes(T(A), bits), dsq.dsq_pack_codes(T(B), bits)
+        Cg, Dg = dsq.dsq_gemm(Ap, Bp, M, Nn, K, bits, ws, row_scale=T(rs), want_i32=want_i32)
+        assert dsq.dsq_workspace_status(ws) == 0
+    finally:
+        dsq.dsq_set_gemm_two_pass(1)
     return (N(Cg) if want_i32 else None), N(Dg)
 
 
 # the two-pass path (rows expanded to 8-bit once, then an 8-bit GEMM): whole
 # tiles, ragged M / N / K, an N that is not a multiple of 8 (scalar stores), a K
 # that is not a multiple of 16
-TWO_PASS_SIZES = [(1024, 1024, 1024), (1100, 1030, 1050), (1024, 1027, 1031),
-                  (1281, 1536, 2048)]
+TWO_PASS_SIZES = [(1, 1, 1), (130, 70, 200), (300, 257, 1000), (1024, 1024, 1024),
+                  (1100, 1030, 1050), (1024, 1027, 1031), (1281, 1536, 2048)]
 
 
 @pytest.mark.parametrize("bits", [2, 3, 4])

@@ -93,7 +93,12 @@ def test_validation_status_codes_without_a_gpu():
     assert lib.dsq_gemm_workspace_bytes(512, 4096, 4096, 4) == lib.dsq_workspace_bytes()
     assert lib.dsq_gemm_workspace_bytes(4096, 4096, 4096, 7) == lib.dsq_workspace_bytes()
     assert lib.dsq_gemm_workspace_bytes(4096, 4096, 4096, 4) == 256 + 1024 + 2 * 4096 * 4096
+    assert lib.dsq_gemm_workspace_bytes(2048, 2048, 2048, 4) == lib.dsq_workspace_bytes()
+    assert lib.dsq_gemm_workspace_bytes(4100, 4099, 2049, 2) >= 256 + 1024 + (4100 + 4099) * 2064
+    assert lib.dsq_set_gemm_two_pass(2) == 0
     assert lib.dsq_gemm_workspace_bytes(1025, 1030, 1031, 2) >= 256 + 1024 + (1025 + 1030) * 1040
+    assert lib.dsq_gemm_workspace_bytes(3, 5, 7, 4) > lib.dsq_workspace_bytes()
+    assert lib.dsq_set_gemm_two_pass(1) == 0 and lib.dsq_set_gemm_two_pass(3) == -4
     # the no-workspace variant rejects bad arguments before it looks up its
     # scratch or enqueues anything (so this works without a GPU)
     assert lib.dsq_gemm_static_ws(None, fake, 128, 128, 128, 4, fake, None, None, 1, None) == -1
