@@ -97,6 +97,9 @@ struct W3Params {
     int tap_stride;                    // slot rows between two filter rows
     int as_slots, bp_slots, b_stages, b_res;
     int w8;                            // weight K steps come expanded, by TMA, into the operand ring
+    int dup;                           // transposed tiles, <= 64 output channels: the 128 A rows hold the
+                                       // weight rows twice; lanes 64..127 of the accumulator repeat lanes
+                                       // 0..63 and their epilogue warps take the other half of the columns
     int cout_pad;                      // Cout rounded up to the N tiling
     int tr;                            // transposed tiles (kernel form TR)
     int mstep;                         // M tiles between two tiles of a CTA
@@ -362,6 +365,9 @@ dsq_win3_kernel(const __grid_constant__ CUtensorMap tmap_b,
                 mbar_arrive_expect_tx(bar_b_full(s), b_stage_bytes);
                 tma_load_2d(smem_u32(smem + L.b_tiles + s * b_stage_bytes), &tmap_b, x, y,
                             bar_b_full(s));
+                if (p.dup)     // the map's box is 64 rows: the same rows again behind them
+                    tma_load_2d(smem_u32(smem + L.b_tiles + s * b_stage_bytes + 64 * 128), &tmap_b,
+                                x, y, bar_b_full(s));
                 ++issued;
                 x += 128;
                 if (x == p.ksteps * 128) x = 0;
@@ -694,11 +700,15 @@ dsq_win3_kernel(const __grid_constant__ CUtensorMap tmap_b,
             constexpr uint32_t MASK = (1u << BITS) - 1u;
             const DsqEpi &e = p.e;
             const float *lut = reinterpret_cast<const float *>(smem + L.lut);
-            const int ch = n_tile * 128 + quarter * 32 + lane;
+            // (dup: lanes 64..127 repeat channels 0..63; quarters 2, 3 take columns 128..255)
+            const int chq = p.dup ? (quarter & 1) * 32 : quarter * 32;
+            const int colbase = p.dup ? 128 * (quarter >> 1) + 32 * k : 64 * k;
+            const int units = p.dup ? 2 : 4;
+            const int ch = n_tile * 128 + chq + lane;
             // a warp has work while its first code word lies inside the output row:
             // channels past Cout are padding lanes of the packed row and get zeros
             // (warp-uniform)
-            const bool warp_live = (n_tile * 128 + quarter * 32) * BITS / 8 < p.out_pitch;
+            const bool warp_live = (n_tile * 128 + chq) * BITS / 8 < p.out_pitch;
             float sc = 0.f, bi = 0.f;
             if (ch < p.Ncols) {
                 sc = __ldg(e.scale + ch);
@@ -706,14 +716,15 @@ dsq_win3_kernel(const __grid_constant__ CUtensorMap tmap_b,
                 bi = __ldg(e.bias + ch);
             }
             const int pw = p.out_pitch / 4;                  // words of an output pixel
-            const int cg = (n_tile * 128 + quarter * 32 + (lane & ~(E - 1))) / E;   // this lane group's word
+            const int cg = (n_tile * 128 + chq + (lane & ~(E - 1))) / E;   // this lane group's word
             const uint32_t *res32 = reinterpret_cast<const uint32_t *>(e.residual);
             uint32_t *y32 = reinterpret_cast<uint32_t *>(e.y_codes);
-            // output pixel (or -1) of the warp's 64 columns: lane L follows columns
-            // 64 k + 2 L and 64 k + 2 L + 1; the others get them by shuffle
+            // output pixel (or -1) of the warp's columns: lane L follows columns
+            // colbase + 2 L and colbase + 2 L + 1; the others get them by shuffle
+            // (dup: a warp has 32 columns and only asks lanes 0..15)
             W3Pos pos0, pos1;
             {
-                const int g0 = m_first * TP + 64 * k + 2 * lane;
+                const int g0 = m_first * TP + colbase + 2 * lane;
                 pos0.n = g0 / img_positions;
                 const int rem = g0 - pos0.n * img_positions;
                 pos0.h = rem / p.Wp;
@@ -734,8 +745,8 @@ dsq_win3_kernel(const __grid_constant__ CUtensorMap tmap_b,
                 tc_fence_after_sync();
                 const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + as * 256;
 #pragma unroll 1
-                for (int u = 0; warp_live && u < 4; ++u) {
-                    const int col0 = 64 * k + 16 * u;
+                for (int u = 0; warp_live && u < units; ++u) {
+                    const int col0 = colbase + 16 * u;
                     uint32_t r[16], cw[CWU], resT[CWU];
                     int mp[CWU];
                     __syncwarp();
@@ -1127,11 +1138,13 @@ int dsq_conv3_window(const void *act_codes, const dsq_nhwc_t *shape, int bits,
     if (shape->W + 2 > 32000 || shape->H + 2 > 32000) return DSQ_ERR_UNSUPPORTED;
     // Which kernel (hook value 1 = automatic; measured on the ResNet-18- and
     // VGG-16-shaped layers, per layer, 20 launches back to back):
-    //  * more than 64 output channels: transposed tiles wherever they fit, except
-    //    7x7-sized images with >= 512 input channels (a handful of tiles with very
-    //    long K loops, where the im2col kernel's CTA pairs are faster);
-    //  * up to 64 output channels (half of a transposed tile's 128 weight rows
-    //    would be idle): plain tiles.
+    //  * transposed tiles wherever they fit, except 7x7-sized images with >= 512
+    //    input channels (a handful of tiles with very long K loops, where the
+    //    im2col kernel is as fast or faster).  With up to 64 output channels the
+    //    transposed form needs the weight rows twice in its A operand (`dup`),
+    //    which it only gets from the blob's expanded copy: 64->64 at 56x56 runs
+    //    in 18 us against 22.5 us on plain tiles;
+    //  * otherwise plain tiles.
     const bool tiny_deep = shape->H * shape->W <= 64 && Cin >= 512;
     if (hooks.window3 == 1 && tiny_deep) return DSQ_ERR_UNSUPPORTED;
     // the lean codes epilogue wants the requantiser range to start at 0, the
@@ -1161,11 +1174,17 @@ int dsq_conv3_window(const void *act_codes, const dsq_nhwc_t *shape, int bits,
     // Transposed (tr): tiles of 256 positions x 128 output channels, A = weights.
     // Plain: 128 positions x up to 256 channels, A = window.
     const DsqW8Info w8 = dsq_w8_info(conv, bits);
-    // (up to 64 output channels the expanded weights stay resident in shared
-    // memory for the whole CTA anyway: nothing to gain, measured slightly slower)
-    p.w8 = hooks.w8 && w8.enabled && e.half_offset && bits != 3 && Cout > 64;
+    // (plain tiles with up to 64 output channels keep the expanded weights resident in
+    // shared memory for the whole CTA anyway: nothing to gain, measured slightly slower)
+    const bool w8_ok = hooks.w8 && w8.enabled && e.half_offset && bits != 3;
     auto configure = [&](int tr) -> int {
         p.tr = tr;
+        // transposed tiles for <= 64 output channels: the weight rows twice in the
+        // A operand (two TMA boxes of the expanded copy), so that all 128 lanes of
+        // the accumulator, and all epilogue warps, carry data
+        p.dup = tr && Cout <= 64;
+        if (p.dup && !w8_ok) return 0;
+        p.w8 = w8_ok && (Cout > 64 || p.dup);
         const int tile_pos = tr ? 256 : W3_BM;
         p.m_tiles = (int)((G + tile_pos - 1) / tile_pos);
         p.BN = tr ? 128 : (Cout >= 256 ? 256 : ((Cout + 63) / 64) * 64);
@@ -1228,7 +1247,7 @@ int dsq_conv3_window(const void *act_codes, const dsq_nhwc_t *shape, int bits,
         return 0;
     };
     int found = 0;
-    const bool want_tr = hooks.window3 == 3 || (hooks.window3 == 1 && Cout > 64);
+    const bool want_tr = hooks.window3 == 3 || hooks.window3 == 1;
     if (bits != 3 && want_tr) found = configure(1);
     if (!found) found = configure(0);
     if (!found) return DSQ_ERR_UNSUPPORTED;
@@ -1283,7 +1302,7 @@ int dsq_conv3_window(const void *act_codes, const dsq_nhwc_t *shape, int bits,
         // rows x one K step, swizzled on the way in
         cuuint64_t dims[2] = {(cuuint64_t)p.ksteps * 128, (cuuint64_t)Cout};
         cuuint64_t strides[1] = {(cuuint64_t)p.ksteps * 128};
-        cuuint32_t box[2] = {128u, (cuuint32_t)p.BN};
+        cuuint32_t box[2] = {128u, (cuuint32_t)(p.dup ? 64 : p.BN)};
         cuuint32_t estr[2] = {1, 1};
         if (enc(&tb, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2,
                 const_cast<uint8_t *>((const uint8_t *)w_packed + w8.offset), dims, strides, box,
