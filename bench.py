@@ -38,7 +38,7 @@ import dsq_inputs  # noqa: E402
 # DRAM traffic of the tensor-core convolution kernels per launch in this
 # workload, from one ncu capture (profiles/bench_launch_list.txt); valid only
 # for the kernel sources it was taken on (checked by hash)
-TRAFFIC = {"bytes_per_launch": 4726885, "sources_sha256": "29b376070cc6976455d295b3d50e21a9d3187d1ed26eafb01c642c6828775896"}
+TRAFFIC = {"bytes_per_launch": 4790865, "sources_sha256": "65c0234e31d3b55b9d963fc3904cfe39c344c53146a14df273f3364e45b0c6ab"}
 
 WORKLOAD = "resnet18-shaped stack, 4-bit W/A, batch 64, 56x56x64 stem output, 19 convs"
 METRIC = "4-bit ResNet-18 conv-stack throughput (effective low-bit conv TOPS alongside)"

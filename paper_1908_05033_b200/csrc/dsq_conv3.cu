@@ -83,6 +83,11 @@ constexpr int W3_MAX_BST = 10;         // expanded B stages (resident: all K ste
 constexpr int W3_BAND_PX = 136;        // pixels of a band (three-band staging)
 constexpr int W3_MAX_WINDOW_PX = 416;
 
+// byte offsets of the kernel's shared-memory regions (w3_layout)
+struct W3Smem {
+    uint32_t a_slots, b_tiles, a_stage, b_packed, epi, lut, a_tab, bars, tmem_slot, abort_flag, total;
+};
+
 struct W3Params {
     // geometry
     int N, H, W, Hp, Wp;               // Hp = H + 2, Wp = W + 2
@@ -118,12 +123,10 @@ struct W3Params {
     uint32_t orv;
     const uint8_t *act;                // input codes and pixel pitch (general weight offset: S_a)
     int P;
+    W3Smem L;                          // shared-memory layout (host-made: w3_layout)
     int *ws;
 };
 
-struct W3Smem {
-    uint32_t a_slots, b_tiles, a_stage, b_packed, epi, lut, a_tab, bars, tmem_slot, abort_flag, total;
-};
 
 __host__ __device__ inline W3Smem w3_layout(int apx, int BN, int bits, int PB, int as_slots,
                                             int b_stages, int bp_slots, int cout_pad)
@@ -246,11 +249,13 @@ dsq_win3_kernel(const __grid_constant__ CUtensorMap tmap_b,
     constexpr int TP = TR ? 256 : W3_BM;       // positions of a tile
     static_assert(!TR || BITS != 3, "transposed tiles: 2- and 4-bit codes");
     extern __shared__ __align__(1024) uint8_t smem_raw[];
+    if ((threadIdx.x >> 5) == 1) W3_STAMP(13, 0);
     uint8_t *smem = reinterpret_cast<uint8_t *>(
         (reinterpret_cast<uintptr_t>(smem_raw) + 1023u) & ~(uintptr_t)1023u);
     const int BN = p.BN;
-    const W3Smem L = w3_layout(p.apx, BN, BITS, p.PB, p.as_slots, p.b_stages, p.bp_slots,
-                               p.cout_pad);
+    // (the layout comes ready-made: every warp's first instructions are on the
+    // critical path of a launch)
+    const W3Smem &L = p.L;
     if ((uint32_t)(smem - smem_raw) + L.total > (uint32_t)p.smem_bytes) {
         grid_dependency_wait();
         if (threadIdx.x == 0) atomicCAS(p.ws + DSQ_WS_STATUS, 0, (int)DSQ_ERR_UNSUPPORTED);
@@ -260,8 +265,8 @@ dsq_win3_kernel(const __grid_constant__ CUtensorMap tmap_b,
     const int lane = threadIdx.x & 31;
     // CTA c works on N tile c % n_tiles and on the M tiles m_first, m_first +
     // mstep, ... (the grid is a multiple of n_tiles)
-    const int n_tile = (int)blockIdx.x % p.n_tiles;
-    const int m_first = (int)blockIdx.x / p.n_tiles;
+    const int n_tile = p.n_tiles == 1 ? 0 : (int)blockIdx.x % p.n_tiles;
+    const int m_first = p.n_tiles == 1 ? (int)blockIdx.x : (int)blockIdx.x / p.n_tiles;
     const int my_tiles = m_first < p.m_tiles ? (p.m_tiles - 1 - m_first) / p.mstep + 1 : 0;
     const uint32_t n_b_fills =
         my_tiles == 0 ? 0u : (p.b_res ? (uint32_t)p.ksteps : (uint32_t)my_tiles * p.ksteps);
@@ -291,6 +296,7 @@ dsq_win3_kernel(const __grid_constant__ CUtensorMap tmap_b,
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + L.tmem_slot);
     Ctl ctl{reinterpret_cast<volatile int *>(smem + L.abort_flag), p.ws, p.wait_ns};
 
+    if (warp == 0) W3_STAMP(13, 9);
     if (threadIdx.x == 0) {
         for (int s = 0; s < W3_A_SLOTS; ++s) {
             mbar_init(bar_a_full(s), W3_NUM_A_WARPS);
@@ -314,11 +320,15 @@ dsq_win3_kernel(const __grid_constant__ CUtensorMap tmap_b,
         }
         mbar_init(bar_drain, 1);
         *ctl.abort_flag = 0;
+        W3_STAMP(13, 10);
         mbar_init_fence();
+        W3_STAMP(13, 11);
     }
     if (warp == W3_WARP_MMA) {
+        W3_STAMP(13, 5);
         tmem_alloc(smem_u32((const void *)tmem_slot), 512);
         tmem_relinquish();
+        W3_STAMP(13, 6);
         // A descriptor offsets (16-byte units from the start of a slot) of the
         // four instructions of every K step of a plane; 0xFFFFFFFF = no
         // instruction (the half-empty last K step of a 64-channel input)
@@ -340,14 +350,18 @@ dsq_win3_kernel(const __grid_constant__ CUtensorMap tmap_b,
         const int q = threadIdx.x - 64;
         reinterpret_cast<float *>(smem + L.lut)[q] = __fmaf_rn((float)q, p.e.res_delta, p.e.res_lo);
     }
+    if (warp == W3_WARP_MMA) W3_STAMP(13, 7);
+    if (warp == W3_WARP_E0) W3_STAMP(13, 8);
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = __shfl_sync(0xffffffffu, *tmem_slot, 0);
     // everything above touched no global data; nothing below starts before the
     // kernels ahead of this one in the stream have completed
+    W3_STAMP(13, 1);
     grid_launch_dependents();
     grid_dependency_wait();
+    W3_STAMP(13, 2);
 
     if (warp == W3_WARP_TMA_B) {
         // ---------------- producer: packed B rows of one K step ------------------
@@ -741,7 +755,9 @@ dsq_win3_kernel(const __grid_constant__ CUtensorMap tmap_b,
                                    ? (pos1.n * p.H + pos1.h) * p.W + pos1.w : -1;
                 pos0 = w3_add(pos0, p.t_dn, p.t_dh, p.t_dw, p.Hp, p.Wp);
                 pos1 = w3_add(pos1, p.t_dn, p.t_dh, p.t_dw, p.Hp, p.Wp);
+                if (warp == W3_WARP_E0) W3_STAMP(7, it);
                 if (!(ok = wait_bar_warp(bar_acc_full(as), (it >> 1) & 1u, ctl, 8))) break;
+                if (warp == W3_WARP_E0) W3_STAMP(8, it);
                 tc_fence_after_sync();
                 const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + as * 256;
 #pragma unroll 1
@@ -830,6 +846,7 @@ dsq_win3_kernel(const __grid_constant__ CUtensorMap tmap_b,
                 tc_fence_before_sync();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_acc_empty(as));
+                if (warp == W3_WARP_E0) W3_STAMP(9, it);
             }
         } else {
         const int row_in_tile = quarter * 32 + lane;
@@ -986,10 +1003,12 @@ dsq_win3_kernel(const __grid_constant__ CUtensorMap tmap_b,
     // ---------------- teardown ------------------------------------------------------
     tc_fence_before_sync();
     __syncthreads();
+    if (warp == 0) W3_STAMP(13, 3);
     if (warp == W3_WARP_MMA) {
         __syncwarp();
         tc_fence_after_sync();
         tmem_dealloc(tmem_base, 512);
+        W3_STAMP(13, 4);
     }
 }
 
@@ -1251,8 +1270,8 @@ int dsq_conv3_window(const void *act_codes, const dsq_nhwc_t *shape, int bits,
     if (bits != 3 && want_tr) found = configure(1);
     if (!found) found = configure(0);
     if (!found) return DSQ_ERR_UNSUPPORTED;
-    p.smem_bytes = (int)w3_layout(p.apx, p.BN, bits, p.PB, p.as_slots, p.b_stages, p.bp_slots,
-                                  p.cout_pad).total + 1024;
+    p.L = w3_layout(p.apx, p.BN, bits, p.PB, p.as_slots, p.b_stages, p.bp_slots, p.cout_pad);
+    p.smem_bytes = (int)p.L.total + 1024;
     // grid: a multiple of n_tiles; CTA c takes N tile c % n_tiles and every
     // mstep-th M tile
     const int sms = dsq_sm_count();
