@@ -350,6 +350,17 @@ dsq_win3_kernel(const __grid_constant__ CUtensorMap tmap_b,
         const int q = threadIdx.x - 64;
         reinterpret_cast<float *>(smem + L.lut)[q] = __fmaf_rn((float)q, p.e.res_delta, p.e.res_lo);
     }
+    // the window producer's first position (two divisions on one lane), worked out
+    // here, where the warp would otherwise only wait for the slower warps at the
+    // barrier: it is on the critical path of a launch
+    W3Pos a_base0 = {0, 0, 0};
+    if (warp == W3_WARP_TMA_A && lane == 0) {
+        const int g0 = m_first * TP;
+        a_base0.n = g0 / img_positions;
+        const int rem = g0 - a_base0.n * img_positions;
+        a_base0.h = rem / p.Wp;
+        a_base0.w = rem - a_base0.h * p.Wp;
+    }
     if (warp == W3_WARP_MMA) W3_STAMP(13, 7);
     if (warp == W3_WARP_E0) W3_STAMP(13, 8);
     tc_fence_before_sync();
@@ -360,7 +371,8 @@ dsq_win3_kernel(const __grid_constant__ CUtensorMap tmap_b,
     // kernels ahead of this one in the stream have completed
     W3_STAMP(13, 1);
     grid_launch_dependents();
-    grid_dependency_wait();
+    // (the window producer first works out its coordinates, then waits)
+    if (warp != W3_WARP_TMA_A) grid_dependency_wait();
     W3_STAMP(13, 2);
 
     if (warp == W3_WARP_TMA_B) {
@@ -419,48 +431,59 @@ dsq_win3_kernel(const __grid_constant__ CUtensorMap tmap_b,
         }
     } else if (warp == W3_WARP_TMA_A) {
         // ---------------- producer: packed window of a tile and plane ------------
+        if (lane != 0) grid_dependency_wait();
         if (lane == 0) {
             uint32_t issued = 0, ph = 0;
             const int AS = p.as_slots;
             const int nld = p.nbands * p.a_nload;
             int s = 0, pl = 0;
-            // first position of the CTA's first tile (the only division)
-            W3Pos base;
-            {
-                const int g0 = m_first * TP;
-                base.n = g0 / img_positions;
-                const int rem = g0 - base.n * img_positions;
-                base.h = rem / p.Wp;
-                base.w = rem - base.h * p.Wp;
-            }
+            // The start coordinates of a fill's loads are worked out one fill ahead
+            // (the first before anything can be issued), so that between the
+            // moment a slot is free and the copies only the issue itself remains.
+            // Loads that start behind the last image hold nothing a valid output
+            // reads: they are left out (and not counted).  An im2col load must
+            // start inside the map's bounding box (0 <= h < Hp, 0 <= w < Wp, n >= 0,
+            // which the position arithmetic guarantees): a position outside it is
+            // never issued - the roles then run into their wait limit and the
+            // kernel reports the failure.
+            W3Pos base = a_base0;
+            W3Pos q[3];
+            int nl = 0;
+            bool bad = false;
+            auto prepare = [&]() {
+                nl = 0;
+                bad = false;
+#pragma unroll
+                for (int i = 0; i < 3; ++i) {
+                    if (i >= nld) break;
+                    q[i] = w3_add(base, p.ld_dn[i], p.ld_dh[i], p.ld_dw[i], p.Hp, p.Wp);
+                    if (q[i].n < p.N) {
+                        ++nl;
+                        bad |= q[i].n < 0 || q[i].h < 0 || q[i].h >= p.Hp || q[i].w < 0 || q[i].w >= p.Wp;
+                    }
+                }
+            };
+            prepare();
+            grid_dependency_wait();
 #pragma unroll 1
             for (uint32_t g = 0; g < n_a_fills; ++g) {
                 if (!wait_bar(bar_as_empty(s), ph ^ 1u, ctl, 11)) break;
-                // loads that start behind the last image hold nothing a valid
-                // output reads: they are left out (and not counted)
-                int nl = 0;
-                for (int i = 0; i < nld; ++i)
-                    nl += w3_add(base, p.ld_dn[i], p.ld_dh[i], p.ld_dw[i], p.Hp, p.Wp).n < p.N;
+                if (bad) {
+                    if (atomicCAS(p.ws + DSQ_WS_STATUS, 0, (int)DSQ_ERR_SHAPE) == 0)
+                        p.ws[DSQ_WS_DETAIL] = 16;
+                    *ctl.abort_flag = 1;
+                    break;
+                }
                 mbar_arrive_expect_tx(bar_as_full(s), (uint32_t)(nl * p.a_box * p.PB));
                 const uint32_t dst0 = smem_u32(smem + L.a_stage) + s * a_stage_bytes;
-                for (int i = 0; i < nld; ++i) {
-                    // (start coordinates always lie inside the map's bounding box:
-                    // 0 <= q.h < Hp, 0 <= q.w < Wp, q.n < N)
-                    const W3Pos q = w3_add(base, p.ld_dn[i], p.ld_dh[i], p.ld_dw[i], p.Hp, p.Wp);
-                    if (q.n >= p.N) continue;
-                    // an im2col load must start inside the map's bounding box: a
-                    // position outside it is never issued (the roles then run into
-                    // their wait limit and the kernel reports the failure)
-                    if (q.n < 0 || q.h < 0 || q.h >= p.Hp || q.w < 0 || q.w >= p.Wp) {
-                        if (atomicCAS(p.ws + DSQ_WS_STATUS, 0, (int)DSQ_ERR_SHAPE) == 0)
-                            p.ws[DSQ_WS_DETAIL] = 16;
-                        *ctl.abort_flag = 1;
-                        continue;
-                    }
+#pragma unroll
+                for (int i = 0; i < 3; ++i) {
+                    if (i >= nld) break;
+                    if (q[i].n >= p.N) continue;
                     // bounding box = image grown by one pixel: base positions
                     // -2 .. W-1 / -2 .. H-1, filter offset (1, 1)
                     tma_load_im2col_4d(dst0 + (uint32_t)(i * p.a_box * p.PB), &tmap_a, pl * p.PB,
-                                       q.w - 2, q.h - 2, q.n, (uint16_t)1, (uint16_t)1,
+                                       q[i].w - 2, q[i].h - 2, q[i].n, (uint16_t)1, (uint16_t)1,
                                        bar_as_full(s));
                 }
                 ++issued;
@@ -468,6 +491,7 @@ dsq_win3_kernel(const __grid_constant__ CUtensorMap tmap_b,
                 if (++pl == p.npl) {
                     pl = 0;
                     base = w3_add(base, p.t_dn, p.t_dh, p.t_dw, p.Hp, p.Wp);
+                    prepare();
                 }
                 if (++s == AS) { s = 0; ph ^= 1u; }
             }
