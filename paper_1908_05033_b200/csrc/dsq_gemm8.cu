@@ -14,7 +14,7 @@
 //           touches an operand byte.  CTA pairs on 256 x 256 tiles
 //           (tcgen05.mma cta_group::2, kind::i8, both operands through
 //           shared-memory descriptors: at N = 256 a descriptor-fed instruction
-//           runs at the pipe's full rate), a ring of six 32 KB stages per CTA,
+//           runs at the pipe's full rate), a ring of seven 32 KB stages per CTA,
 //           and TWO 256-column accumulators in tensor memory, so the epilogue
 //           of a tile (eight warps per CTA) overlaps the next tile's
 //           instructions.
