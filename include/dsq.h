@@ -149,6 +149,13 @@ int dsq_workspace_status(void *workspace, void *stream);
  *              signed codes at the activation pixel pitch
  *              dsq_row_pitch(Cin, bits).  Depthwise: KH*KW packed rows of C
  *              signed codes.  Treat as opaque; dsq_unpack can read it.
+ *              For dense 3x3 stride-1 pad-1 convolutions at 2 or 4 bits with
+ *              64 or a multiple of 128 input channels the buffer is larger:
+ *              behind the packed rows (1024-byte aligned) it holds the same
+ *              rows already expanded to the 8-bit operand bytes of the grid
+ *              Delta (c + 1/2), which dsq_conv2d then copies to the tensor
+ *              core's shared-memory operand without expanding them again
+ *              (dsq_weight_bytes includes that copy).
  * A clip range with hi <= lo or a non-finite bound cannot be seen from the
  * host: the kernel writes code 0 for that channel and records DSQ_ERR_RANGE
  * in the workspace. */
