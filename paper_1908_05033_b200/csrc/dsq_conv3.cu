@@ -779,6 +779,29 @@ dsq_win3_kernel(const __grid_constant__ CUtensorMap tmap_b,
                                    ? (pos1.n * p.H + pos1.h) * p.W + pos1.w : -1;
                 pos0 = w3_add(pos0, p.t_dn, p.t_dh, p.t_dw, p.Hp, p.Wp);
                 pos1 = w3_add(pos1, p.t_dn, p.t_dh, p.t_dw, p.Hp, p.Wp);
+                // Word w of a unit covers E positions; lane i of a channel group owns
+                // position i of them: it stores that position's word at the end, and it
+                // fetches that position's residual word - one unit ahead, the first
+                // unit's before the wait for the accumulator, so that the loads'
+                // latency is off the path.  The same transpose that turns "E positions
+                // of my channel" into "E channels of my position" is its own inverse,
+                // so it also turns the fetched words into "residual codes of my channel
+                // at E positions".
+                int mpn[CWU];
+                uint32_t wordn[CWU];
+                auto fetch = [&](int u) {
+#pragma unroll
+                    for (int w = 0; w < CWU; ++w) {
+                        const int cpos = 16 * u + w * E + (lane & (E - 1));   // column of the warp
+                        const int mp_a = __shfl_sync(0xffffffffu, m0, cpos >> 1);
+                        const int mp_b = __shfl_sync(0xffffffffu, m1, cpos >> 1);
+                        mpn[w] = (cpos & 1) ? mp_b : mp_a;
+                        wordn[w] = 0u;
+                        if (EPI != DSQ_EPI_CODES && e.residual && mpn[w] >= 0 && 4 * cg < p.out_pitch)
+                            wordn[w] = __ldg(res32 + (int64_t)mpn[w] * pw + cg);
+                    }
+                };
+                if (warp_live) fetch(0);
                 if (warp == W3_WARP_E0) W3_STAMP(7, it);
                 if (!(ok = wait_bar_warp(bar_acc_full(as), (it >> 1) & 1u, ctl, 8))) break;
                 if (warp == W3_WARP_E0) W3_STAMP(8, it);
@@ -791,23 +814,14 @@ dsq_win3_kernel(const __grid_constant__ CUtensorMap tmap_b,
                     int mp[CWU];
                     __syncwarp();
                     tmem_ld_32x16(taddr + col0, r);
-                    // Word w of the unit covers E positions; lane i of a channel group
-                    // owns position i of them: it stores that position's word at the
-                    // end, and it fetches that position's residual word now.  The same
-                    // transpose that turns "E positions of my channel" into "E channels
-                    // of my position" is its own inverse, so it also turns the fetched
-                    // words into "residual codes of my channel at E positions".
+                    uint32_t word[CWU];
+#pragma unroll
+                    for (int w = 0; w < CWU; ++w) { mp[w] = mpn[w]; word[w] = wordn[w]; }
+                    if (u + 1 < units) fetch(u + 1);
 #pragma unroll
                     for (int w = 0; w < CWU; ++w) {
-                        const int cpos = 16 * u + w * E + (lane & (E - 1));   // column of the warp
-                        const int mp_a = __shfl_sync(0xffffffffu, m0, cpos >> 1);
-                        const int mp_b = __shfl_sync(0xffffffffu, m1, cpos >> 1);
-                        mp[w] = (cpos & 1) ? mp_b : mp_a;
-                        uint32_t word = 0u;
-                        if (EPI != DSQ_EPI_CODES && e.residual && mp[w] >= 0 && 4 * cg < p.out_pitch)
-                            word = __ldg(res32 + (int64_t)mp[w] * pw + cg);
                         resT[w] = 0u;
-                        if (EPI != DSQ_EPI_CODES) resT[w] = w3_transpose_fields<BITS>(word, lane);
+                        if (EPI != DSQ_EPI_CODES) resT[w] = w3_transpose_fields<BITS>(word[w], lane);
                         cw[w] = 0u;
                     }
                     tmem_ld_wait();
