@@ -38,7 +38,7 @@ import dsq_inputs  # noqa: E402
 # DRAM traffic of the tensor-core convolution kernels per launch in this
 # workload, from one ncu capture (profiles/bench_launch_list.txt); valid only
 # for the kernel sources it was taken on (checked by hash)
-TRAFFIC = {"bytes_per_launch": 4787456, "sources_sha256": "d575c13524f2c9fc86079e096577b783345c970da376a59616326ac4442925fc"}
+TRAFFIC = {"bytes_per_launch": 4788042, "sources_sha256": "585f1a5645589bf21d02a3907c39fa0f79a688af8ef574aeb29a2ef435337442"}
 
 WORKLOAD = "resnet18-shaped stack, 4-bit W/A, batch 64, 56x56x64 stem output, 19 convs"
 METRIC = "4-bit ResNet-18 conv-stack throughput (effective low-bit conv TOPS alongside)"
